@@ -1,0 +1,387 @@
+#!/usr/bin/env python
+"""Benchmark of the W4A16 layer on B200: the batch sweep on one large layer.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Workload (config 2 of this build): K = N = 8192, group size 128, M in {1,2,4,8,16,32,64,128};
+A ~ fp16 N(0,1), codes uniform 0..15 (zero point 8), scales uniform in [0.005, 0.02]; synthetic.
+One step = one pass of the layer at every M of the sweep (pack is offline and not in the step).
+Weights are cold: every launch reads the next of several packed copies whose total size exceeds
+twice the L2 capacity.
+
+Prints ONE JSON line.  `value` = packed weight bytes (codes + scales) streamed per second over the
+whole step, inputs resident in HBM, timed with CUDA events around a CUDA graph of K steps.
+`e2e` = the same metric with A copied from pinned host memory and C copied back inside the timed
+region (weights stay resident: they are the model).  `roofline` compares the algorithmic bytes
+(weights + scales + A + C, each once) per second with the measured HBM peak.  `per_m` lists each
+batch size: time, weight GB/s, TFLOP/s, fraction of its roofline, speedup over a cuBLAS fp16 GEMM
+of the same shape (torch.matmul).  `cpu_baseline` times the CPU oracle on a bounded sample.
+
+N > 1: the layer does not shard in this build (replicas only): every rank runs the same sweep on
+its own GPU; `value` sums the ranks, time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2408_11743_b200 import inputs, roofline  # noqa: E402
+
+K_DIM, N_DIM, GROUP = 8192, 8192, 128
+SWEEP = (1, 2, 4, 8, 16, 32, 64, 128)
+METRIC = "w4a16_gemm_weight_stream_rate_batch_sweep_M1-128_K8192_N8192_g128"
+UNIT = "GB/s"
+CPU_SAMPLE_MS = (16, 64)      # cpu_baseline leg of the GPU arm
+REFERENCE_SAMPLE_MS = (16,)   # one step of --impl reference
+
+
+def launches_for(M: int) -> int:
+    return (M + 31) // 32  # one kernel per slab of 32 rows
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while a region runs (read-only queries)."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self):
+        if self.proc is None:
+            return
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+
+    def summary(self, t0: float, t1: float):
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        rows = [r for t, r in self.rows if t0 - 0.05 <= t <= t1 + 0.05] or [r for _, r in self.rows]
+        for r in rows:
+            parts = [p.strip() for p in r.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(smax), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle leg
+# ------------------------------------------------------------------------------------------------
+def time_oracle_sample(case_cache, Ms=CPU_SAMPLE_MS):
+    """The oracle as it stands, on the host cores, on the full layer at a few batch sizes of the sweep."""
+    import oracle
+    oracle.build()
+    t = 0.0
+    wbytes = 0
+    for M in Ms:
+        case = case_cache(M)
+        t0 = time.perf_counter()
+        oracle.gemm(case.A, case.q_kpacked, case.S, case.G)
+        t += time.perf_counter() - t0
+        wbytes += roofline.weight_bytes(K_DIM, N_DIM, GROUP)
+    return wbytes / t / 1e9, t, oracle.num_threads()
+
+
+def make_case_cache():
+    cache = {}
+    base = inputs.make_dense(max(SWEEP), K_DIM, N_DIM, GROUP, inputs.case_seed(2, 0, 0))
+
+    def get(M):
+        if M not in cache:
+            cache[M] = inputs.DenseCase(np.ascontiguousarray(base.A[:M]), base.q_kpacked, base.S, M, K_DIM, N_DIM,
+                                        GROUP, base.seed)
+        return cache[M]
+    return get
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    get = make_case_cache()
+    vals = []
+    for i in range(args.warmup + args.steps):
+        v, t, cores = time_oracle_sample(get, REFERENCE_SAMPLE_MS)
+        if i >= args.warmup:
+            vals.append((v, t))
+    value = sum(v for v, _ in vals) / len(vals)
+    ms = 1e3 * sum(t for _, t in vals) / len(vals)
+    sample = f"full layer at M in {list(REFERENCE_SAMPLE_MS)} per step (1 of the 8 batch sizes of the sweep)"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "batch sweep K=8192 N=8192 g128 (CPU oracle on a bounded sample)", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------
+# GPU leg
+# ------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2408_11743_b200 as marlin
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a GPU: this library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    marlin.lib()
+    dev = torch.device("cuda", local_rank)
+    props = torch.cuda.get_device_properties(dev)
+    l2 = getattr(props, "L2_cache_size", 126 * 1024 * 1024)
+
+    get = make_case_cache()
+    base = get(max(SWEEP))
+    wbytes = roofline.weight_bytes(K_DIM, N_DIM, GROUP)
+    copies = max(2, int(np.ceil(2.0 * l2 / wbytes)) + 1)
+    q_dev = torch.from_numpy(base.q_kpacked.view(np.int32)).to(dev)
+    s_dev = torch.from_numpy(base.S).to(dev)
+    w0, s0 = marlin.pack(q_dev, s_dev, GROUP)
+    packed = [(w0.clone(), s0.clone()) for _ in range(copies)]
+    del q_dev
+    A_dev = {M: torch.from_numpy(get(M).A).to(dev) for M in SWEEP}
+    C_dev = {M: torch.empty((M, N_DIM), dtype=torch.float16, device=dev) for M in SWEEP}
+    ws = marlin.new_workspace(max(SWEEP), K_DIM, N_DIM, device=dev)
+    stream = torch.cuda.Stream(device=dev)
+    rot = [0]
+
+    def one_gemm(M):
+        w, s = packed[rot[0] % copies]
+        rot[0] += 1
+        marlin.gemm(A_dev[M], w, s, K_DIM, N_DIM, GROUP, ws, out=C_dev[M], stream=stream)
+
+    def one_step():
+        for M in SWEEP:
+            one_gemm(M)
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    # warm-up (also sets kernel attributes before any capture)
+    with torch.cuda.stream(stream):
+        for _ in range(max(3, args.warmup)):
+            one_step()
+    torch.cuda.synchronize(dev)
+    if marlin.read_status(ws, stream=stream) != 0:
+        raise RuntimeError("device-side wait expired during warm-up")
+
+    def capture(fn, reps):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for _ in range(reps):
+                fn()
+        return g
+
+    def time_graph(g, replays=1):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            e0.record(stream)
+            for _ in range(replays):
+                g.replay()
+            e1.record(stream)
+        e1.synchronize()
+        return e0.elapsed_time(e1) * 1e-3
+
+    # ---- main timed region: K steps, device time, max over ranks ----
+    g_steps = capture(one_step, args.steps)
+    with torch.cuda.stream(stream):
+        g_steps.replay()  # instantiate / upload outside the timed region
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    barrier()
+    t_wall0 = time.time()
+    elapsed = time_graph(g_steps)
+    # keep the same load running a little longer so that the 50 ms clock sampler sees it
+    t_extra_end = time.time() + 0.6
+    while time.time() < t_extra_end:
+        time_graph(g_steps)
+    t_wall1 = time.time()
+    barrier()
+    sampler.stop()
+    clocks = sampler.summary(t_wall0, t_wall1)
+    if world > 1:
+        t = torch.tensor([elapsed], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed = float(t.item())
+    step_s = elapsed / args.steps
+    step_wbytes = wbytes * len(SWEEP)
+    value = world * step_wbytes / step_s / 1e9
+    step_alg_bytes = sum(roofline.algorithmic_bytes(M, K_DIM, N_DIM, GROUP) for M in SWEEP)
+    launches_per_step = sum(launches_for(M) for M in SWEEP)
+
+    line = None
+    if rank == 0:
+        peaks = roofline.load_peaks(ROOT)
+        # ---- per batch size: our kernel and cuBLAS fp16 on cold weights ----
+        reps = 4 * copies
+        W16 = [torch.randn((K_DIM, N_DIM), dtype=torch.float16, device=dev) * 0.05
+               for _ in range(max(2, int(np.ceil(2.0 * l2 / (2 * K_DIM * N_DIM))) + 1))]
+        rot16 = [0]
+        per_m = []
+        for M in SWEEP:
+            g = capture(lambda: one_gemm(M), reps)
+            time_graph(g)
+            t_ours = min(time_graph(g) for _ in range(5)) / reps
+            out16 = torch.empty((M, N_DIM), dtype=torch.float16, device=dev)
+
+            def fp16_gemm():
+                torch.matmul(A_dev[M], W16[rot16[0] % len(W16)], out=out16)
+                rot16[0] += 1
+            with torch.cuda.stream(stream):
+                for _ in range(3):
+                    fp16_gemm()
+            torch.cuda.synchronize(dev)
+            g16 = capture(fp16_gemm, 2 * len(W16))
+            time_graph(g16)
+            t_fp16 = min(time_graph(g16) for _ in range(5)) / (2 * len(W16))
+            t_roof = roofline.roofline_seconds(M, K_DIM, N_DIM, GROUP, peaks)
+            per_m.append({
+                "M": M, "us": round(t_ours * 1e6, 3), "weight_gbs": round(wbytes / t_ours / 1e9, 1),
+                "tflops": round(roofline.flops(M, K_DIM, N_DIM) / t_ours / 1e12, 2),
+                "roofline_us": round(t_roof * 1e6, 3), "roofline_frac": round(t_roof / t_ours, 4),
+                "cublas_fp16_us": round(t_fp16 * 1e6, 3), "speedup_vs_fp16": round(t_fp16 / t_ours, 3),
+                "launches": launches_for(M),
+            })
+            del g, g16
+        del W16
+
+        # ---- end to end: host buffers, copies inside the timed region ----
+        A_host = {M: torch.from_numpy(get(M).A).pin_memory() for M in SWEEP}
+        C_host = {M: torch.empty((M, N_DIM), dtype=torch.float16).pin_memory() for M in SWEEP}
+
+        def e2e_step():
+            for M in SWEEP:
+                A_dev[M].copy_(A_host[M], non_blocking=True)
+                one_gemm(M)
+                C_host[M].copy_(C_dev[M], non_blocking=True)
+
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                e2e_step()
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            e0.record(stream)
+            for _ in range(args.steps):
+                e2e_step()
+            e1.record(stream)
+        e1.synchronize()
+        e2e_s = e0.elapsed_time(e1) * 1e-3 / args.steps
+        h2d = sum(2 * M * K_DIM for M in SWEEP)
+        d2h = sum(2 * M * N_DIM for M in SWEEP)
+
+        if marlin.read_status(ws, stream=stream) != 0:
+            raise RuntimeError("device-side wait expired during the benchmark")
+
+        # ---- CPU oracle on a bounded sample ----
+        cpu_v, cpu_t, cores = time_oracle_sample(get)
+
+        achieved = step_alg_bytes / step_s / 1e9
+        line = {
+            "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": round(step_s * 1e3, 5), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f16 x int4 -> f32 accumulate -> f16",
+            "data": "synthetic",
+            "config": {"workload": "config 2: batch sweep M in {1,2,4,8,16,32,64,128} on K=8192 N=8192 g128",
+                       "step": "one marlin_gemm per batch size (8 calls)", "cold_weights":
+                       f"{copies} rotating packed copies ({copies * wbytes / 2**20:.0f} MiB > 2 x L2)",
+                       "timing": "CUDA graph of K steps between CUDA events on the launch stream",
+                       "multi_gpu": "replicas only"},
+            "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": round(achieved / peaks["hbm_gbs"], 4), "traffic": None,
+                         "peak_source": peaks["source"], "kernel": "gemm_dense_kernel",
+                         "per_launch_us": round(step_s * 1e6 / launches_per_step, 3),
+                         "algorithmic_bytes_per_step": step_alg_bytes},
+            "per_m": per_m,
+            "cpu_baseline": {"value": round(cpu_v, 4), "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": f"full layer at M in {list(CPU_SAMPLE_MS)} ({cpu_t:.1f} s)"},
+            "e2e": {"value": round(world * step_wbytes / e2e_s / 1e9, 2), "unit": UNIT,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_s * 1e3, 5)},
+            "gpu_launches": launches_per_step * args.steps,
+            "clocks": clocks,
+        }
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if line is not None:
+        print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,146 @@
+/*
+ * marlin_b200 -- W4A16 linear layer for NVIDIA B200 (sm_100a), C ABI.
+ *
+ *     C[M x N] (fp16) = A[M x K] (fp16) . dequant(Wq[K x N] int4, fp16 scales),  fp32 accumulation
+ *     dequant:  W[k][n] = (Q[k][n] - 8) * S[k / G][n],  Q in 0..15
+ *
+ * The operation is the mixed-precision layer of the MARLIN paper (arxiv 2408.11743), Section 3.4
+ * "Kernel Design": A in fp16, B a K x N INT4 matrix, symmetrically quantised, with one fp16 scale per
+ * output column or per G consecutive weights of a column (ceil(K/G) * N scales).  The 2:4 variant is
+ * Section 4 ("The Sparse-MARLIN Kernel"): groups of four along K, two values kept, 2-bit positions.
+ *
+ * General rules
+ *   - Every pointer named *device* is a CUDA device pointer owned by the caller, 16-byte aligned,
+ *     valid on the current device until the work queued on `stream` has finished.  Host pointers
+ *     are said to be host pointers.  Buffers of one call must not overlap.
+ *   - Calls are asynchronous on `stream`; nothing synchronises, nothing is allocated, nothing throws.
+ *     Every function that can fail returns a marlin_status; 0 is success.
+ *   - There is no CPU path and no other-architecture path: on a device that is not compute
+ *     capability 10.x the calls return MARLIN_ERR_ARCH.
+ *   - Shapes: K % 128 == 0, N % 64 == 0, M >= 1.  group_size is a multiple of 128 that divides K,
+ *     or K itself (also written -1): one scale per column.
+ *   - The packed device layout is opaque (documented in the design doc); only marlin_pack* writes it and
+ *     only marlin_unpack* / marlin_gemm* read it.
+ */
+#ifndef MARLIN_B200_H_
+#define MARLIN_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define MARLIN_API __attribute__((visibility("default")))
+#else
+#define MARLIN_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  MARLIN_OK = 0,
+  MARLIN_ERR_NULL = 1,           /* a required pointer is NULL                                  */
+  MARLIN_ERR_SHAPE = 2,          /* M, K or N out of range or not a multiple of the tile sizes  */
+  MARLIN_ERR_GROUP = 3,          /* group_size not supported for this K                         */
+  MARLIN_ERR_ALIGN = 4,          /* a device pointer is not 16-byte aligned                     */
+  MARLIN_ERR_WORKSPACE = 5,      /* workspace smaller than marlin_workspace_bytes()             */
+  MARLIN_ERR_ARCH = 6,           /* current device is not sm_100                                */
+  MARLIN_ERR_CUDA = 7,           /* a CUDA runtime call or the launch failed                    */
+  MARLIN_ERR_DEVICE_TIMEOUT = 8  /* a bounded wait inside a kernel expired (see marlin_read_status) */
+} marlin_status;
+
+/* A CUDA stream handle (cudaStream_t) passed as an opaque pointer; NULL is the default stream. */
+typedef void* marlin_stream;
+
+MARLIN_API const char* marlin_status_string(int status);
+
+/* ---- sizes (host arithmetic only; valid without a GPU) ------------------------------------- */
+
+/* Bytes of the packed weight buffer: K*N/2 dense; K*N/4 when sparse24 != 0.  0 on a bad shape. */
+MARLIN_API size_t marlin_packed_weight_bytes(int K, int N, int sparse24);
+/* Bytes of the packed scale buffer: 2 * (K/G) * N.  0 on a bad shape or group size. */
+MARLIN_API size_t marlin_packed_scale_bytes(int K, int N, int group_size);
+/* Bytes of the packed 2:4 metadata buffer: K*N/8 (2 bits per kept value). */
+MARLIN_API size_t marlin_packed_meta_bytes(int K, int N);
+/* Bytes of the workspace marlin_gemm* needs for any M <= max_M on this K x N layer.
+ * The workspace holds a status word, per-column-tile arrival counters and the fp32 partial tiles
+ * of the stripe fix-up (Section 3.4 "Striped Partitioning": the paper's "small extra lock buffer").
+ * The caller zeroes it ONCE after allocation (cudaMemset); every call leaves the counters zero.
+ * One workspace must not be used by two calls that can run at the same time. */
+MARLIN_API size_t marlin_workspace_bytes(int max_M, int K, int N);
+
+/* ---- offline re-layout (Section 3.4 "Maximizing Loading Bandwidth", "Dequantization and Tensor
+ *      Cores": weights are static, so they are reshuffled once into the order the kernel streams) -- */
+
+/* Dense pack.
+ *   q_kpacked  device, uint32 [K/8][N]: canonical codes, nibble j of word (kb, n) = Q[8*kb + j][n]
+ *   scales     device, fp16   [K/G][N] row-major
+ *   w_packed   device, out, marlin_packed_weight_bytes(K, N, 0) bytes
+ *   s_packed   device, out, marlin_packed_scale_bytes(K, N, G) bytes
+ * Integer-only permutation; unpack(pack(x)) == x bit for bit. */
+MARLIN_API int marlin_pack(const uint32_t* q_kpacked, const void* scales, void* w_packed, void* s_packed,
+                int K, int N, int group_size, marlin_stream stream);
+
+/* Inverse of marlin_pack: writes the canonical forms back. */
+MARLIN_API int marlin_unpack(const void* w_packed, const void* s_packed, uint32_t* q_kpacked, void* scales,
+                  int K, int N, int group_size, marlin_stream stream);
+
+/* ---- the layer (Section 3.4, all paragraphs: weight streaming, dequantisation, tensor-core
+ *      product, striped partition with global reduction) ----------------------------------------- */
+
+/* C = A . dequant(W).
+ *   A          device, fp16 [M][K] row-major
+ *   w_packed, s_packed   device, from marlin_pack with the same K, N, group_size
+ *   C          device, out, fp16 [M][N] row-major, every element written
+ *   workspace  device, at least marlin_workspace_bytes(M, K, N) bytes, zeroed once by the caller
+ * Accumulation is fp32 (also across stripes); the result is rounded once to fp16 (nearest even).
+ * Results are deterministic: the same inputs give the same bits on every call.
+ * M > 32 is processed as consecutive slabs of rows.
+ * Errors: argument checks return before anything is queued.  A kernel whose bounded waits expire
+ * sets the workspace status word; read it with marlin_read_status. */
+MARLIN_API int marlin_gemm(const void* A, const void* w_packed, const void* s_packed, void* C,
+                int M, int K, int N, int group_size,
+                void* workspace, size_t workspace_bytes, marlin_stream stream);
+
+/* ---- 2:4 structured-sparse variant (Section 4: values structure + metadata indices) ------------ */
+
+/* Pack the compressed form.
+ *   qc_kpacked device, uint32 [K/16][N]: kept codes Qc[K/2][N], nibble j of word (r, n) = Qc[8r+j][n]
+ *   idx        device, uint8  [K/2][N]: position 0..3 of kept value t inside group t/2 of four rows
+ *              along K; idx[2u][n] < idx[2u+1][n]
+ *   scales     device, fp16 [K/G][N], groups over the ORIGINAL K
+ *   outputs    w_packed (K*N/4 bytes), meta_packed (K*N/8 bytes), s_packed (2*(K/G)*N bytes) */
+MARLIN_API int marlin_pack_sparse24(const uint32_t* qc_kpacked, const uint8_t* idx, const void* scales,
+                         void* w_packed, void* meta_packed, void* s_packed,
+                         int K, int N, int group_size, marlin_stream stream);
+
+MARLIN_API int marlin_unpack_sparse24(const void* w_packed, const void* meta_packed, const void* s_packed,
+                           uint32_t* qc_kpacked, uint8_t* idx, void* scales,
+                           int K, int N, int group_size, marlin_stream stream);
+
+/* C = A . dequant(expand(W)) with the pruned positions contributing zero. */
+MARLIN_API int marlin_gemm_sparse24(const void* A, const void* w_packed, const void* meta_packed,
+                         const void* s_packed, void* C, int M, int K, int N, int group_size,
+                         void* workspace, size_t workspace_bytes, marlin_stream stream);
+
+/* Synchronises `stream`, then returns the device-side status word of `workspace`
+ * (MARLIN_OK, or MARLIN_ERR_DEVICE_TIMEOUT if a kernel gave up a bounded wait), or
+ * MARLIN_ERR_CUDA if the stream reports an error.  The status word is sticky until the
+ * workspace is zeroed again. */
+MARLIN_API int marlin_read_status(const void* workspace, marlin_stream stream);
+
+/* ---- host-side planning, exposed for inspection and tests (no GPU needed) ----------------------- */
+
+/* The striped partition of Section 3.4 "Striped Partitioning": the (column tile, 128-row k-block)
+ * units of the weight matrix are numbered column by column, top to bottom, and worker i of
+ * `workers` owns units [bounds[i], bounds[i+1]).  Fills n_tile (columns per tile: 64, 128 or 256),
+ * workers (<= sm_count) and bounds[0..workers] (host pointers; `cap` entries available in bounds).
+ * Returns MARLIN_ERR_SHAPE if cap is too small or the shape is invalid. */
+MARLIN_API int marlin_plan_stripes(int M, int K, int N, int sm_count, int* n_tile, int* workers,
+                        int64_t* bounds, int cap);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MARLIN_B200_H_ */

@@ -1,0 +1,42 @@
+"""CPU restatement of the device weight layout -- TEST INFRASTRUCTURE ONLY.
+
+Written from the layout description in DESIGN.md ("Packed layout"), not from the CUDA source;
+used only to compare bytes with what ``marlin_pack`` writes on the GPU.  Nothing in the product
+imports this file.
+
+Dense layout: the packed buffer is a sequence of uint32 words,
+    word index = (((kb * (N/64) + nb) * 8 + i) * 32 + lane) * 4 + t
+with i = 4*h + j and lane = 4*g + c, and nibble p (bits 4p..4p+3) of that word holds the code at
+    column n = 64*nb + 16*j + g + 8*(p & 1)
+    row    k = 128*kb + 64*h + 16*c + 4*t + 2*((p >> 1) & 1) + (p >> 2)
+Scales: inside every run of 64 columns, packed position 8*g + 2*j + b holds column 16*j + 8*b + g.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+
+def pack_dense_weights(Q: np.ndarray) -> np.ndarray:
+    """Codes Q[K, N] (uint8, 0..15) -> packed uint32 words (1-D, K*N/8)."""
+    K, N = Q.shape
+    assert K % 128 == 0 and N % 64 == 0
+    kb, nb, h, j, g, c, t, p = np.meshgrid(
+        np.arange(K // 128), np.arange(N // 64), np.arange(2), np.arange(4), np.arange(8), np.arange(4),
+        np.arange(4), np.arange(8), indexing="ij")
+    n = 64 * nb + 16 * j + g + 8 * (p & 1)
+    k = 128 * kb + 64 * h + 16 * c + 4 * t + 2 * ((p >> 1) & 1) + (p >> 2)
+    codes = Q[k, n].astype(np.uint32)  # [kb, nb, h, j, g, c, t, p]: already in word order
+    words = np.zeros(codes.shape[:-1], dtype=np.uint32)
+    for pp in range(8):
+        words |= codes[..., pp] << np.uint32(4 * pp)
+    return words.reshape(-1)
+
+
+def pack_scales(S: np.ndarray) -> np.ndarray:
+    """Scales S[K/G, N] fp16 -> packed order (same shape)."""
+    R, N = S.shape
+    assert N % 64 == 0
+    pos = np.arange(64)
+    g, j, b = pos >> 3, (pos >> 1) & 3, pos & 1
+    src = 16 * j + 8 * b + g
+    return S.reshape(R, N // 64, 64)[:, :, src].reshape(R, N)

@@ -1,0 +1,246 @@
+"""ctypes binding of libmarlin_b200.so: same names as the C ABI, argument marshalling only.
+
+Every step of the layer (re-layout, streaming, dequantisation, tensor-core product, stripe
+fix-up) runs inside the library's CUDA kernels.  torch is used for device memory and streams.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libmarlin_b200.so")
+_lib = None
+
+EXPORTS = [
+    "marlin_status_string", "marlin_packed_weight_bytes", "marlin_packed_scale_bytes", "marlin_packed_meta_bytes",
+    "marlin_workspace_bytes", "marlin_pack", "marlin_unpack", "marlin_gemm", "marlin_pack_sparse24",
+    "marlin_unpack_sparse24", "marlin_gemm_sparse24", "marlin_read_status", "marlin_plan_stripes",
+]
+
+
+class MarlinError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        msg = lib().marlin_status_string(status).decode()
+        super().__init__(f"{what}: marlin status {status} ({msg})")
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def lib():
+    """Loads the shared library (once).  Raises if it has not been built: no fallback exists."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise RuntimeError(
+            f"{_LIB_PATH} is missing: build it with `python -m paper_2408_11743_b200.build` "
+            "(this package has no CPU or eager path)")
+    L = ctypes.CDLL(_LIB_PATH)
+    c = ctypes
+    vp, i, sz = c.c_void_p, c.c_int, c.c_size_t
+    L.marlin_status_string.restype = c.c_char_p
+    L.marlin_status_string.argtypes = [i]
+    L.marlin_packed_weight_bytes.restype = sz
+    L.marlin_packed_weight_bytes.argtypes = [i, i, i]
+    L.marlin_packed_scale_bytes.restype = sz
+    L.marlin_packed_scale_bytes.argtypes = [i, i, i]
+    L.marlin_packed_meta_bytes.restype = sz
+    L.marlin_packed_meta_bytes.argtypes = [i, i]
+    L.marlin_workspace_bytes.restype = sz
+    L.marlin_workspace_bytes.argtypes = [i, i, i]
+    L.marlin_pack.argtypes = [vp, vp, vp, vp, i, i, i, vp]
+    L.marlin_unpack.argtypes = [vp, vp, vp, vp, i, i, i, vp]
+    L.marlin_gemm.argtypes = [vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
+    L.marlin_pack_sparse24.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, vp]
+    L.marlin_unpack_sparse24.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, vp]
+    L.marlin_gemm_sparse24.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
+    L.marlin_read_status.argtypes = [vp, vp]
+    L.marlin_plan_stripes.argtypes = [i, i, i, i, vp, vp, vp, i]
+    for name in ("marlin_pack", "marlin_unpack", "marlin_gemm", "marlin_pack_sparse24", "marlin_unpack_sparse24",
+                 "marlin_gemm_sparse24", "marlin_read_status", "marlin_plan_stripes"):
+        getattr(L, name).restype = i
+    _lib = L
+    return L
+
+
+def _torch():
+    import torch
+    return torch
+
+
+def _stream_ptr(stream=None) -> int:
+    torch = _torch()
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(s.cuda_stream)
+
+
+def _dev(t, dtype, name):
+    torch = _torch()
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError(f"{name} must be a CUDA tensor")
+    if t.dtype != dtype:
+        raise TypeError(f"{name} must have dtype {dtype}, got {t.dtype}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    return t
+
+
+def _check(status: int, what: str):
+    if status != 0:
+        raise MarlinError(status, what)
+
+
+def workspace_bytes(max_M: int, K: int, N: int) -> int:
+    n = int(lib().marlin_workspace_bytes(max_M, K, N))
+    if n == 0:
+        raise MarlinError(2, "marlin_workspace_bytes")
+    return n
+
+
+def new_workspace(max_M: int, K: int, N: int, device="cuda"):
+    """Allocates the workspace with torch and zeroes it once, as the C ABI requires."""
+    torch = _torch()
+    return torch.zeros(workspace_bytes(max_M, K, N), dtype=torch.uint8, device=device)
+
+
+def pack(q_kpacked, scales, group_size: int, stream=None):
+    """marlin_pack: canonical codes uint32(int32) [K/8, N] + fp16 scales [K/G, N] -> (w_packed, s_packed)."""
+    torch = _torch()
+    q = _dev(q_kpacked, torch.int32, "q_kpacked")
+    s = _dev(scales, torch.float16, "scales")
+    K, N = q.shape[0] * 8, q.shape[1]
+    L = lib()
+    wb, sb = L.marlin_packed_weight_bytes(K, N, 0), L.marlin_packed_scale_bytes(K, N, group_size)
+    if wb == 0:
+        raise MarlinError(2, "marlin_pack")
+    if sb == 0:
+        raise MarlinError(3, "marlin_pack")
+    if s.numel() * 2 != sb:
+        raise ValueError(f"scales has {s.numel()} elements, expected {sb // 2}")
+    w_packed = torch.empty(wb, dtype=torch.uint8, device=q.device)
+    s_packed = torch.empty(sb, dtype=torch.uint8, device=q.device)
+    _check(L.marlin_pack(q.data_ptr(), s.data_ptr(), w_packed.data_ptr(), s_packed.data_ptr(), K, N, group_size,
+                         _stream_ptr(stream)), "marlin_pack")
+    return w_packed, s_packed
+
+
+def unpack(w_packed, s_packed, K: int, N: int, group_size: int, stream=None):
+    """marlin_unpack: the inverse of pack; returns (q_kpacked int32 [K/8, N], scales fp16 [K/G, N])."""
+    torch = _torch()
+    w = _dev(w_packed, torch.uint8, "w_packed")
+    s = _dev(s_packed, torch.uint8, "s_packed")
+    L = lib()
+    sb = L.marlin_packed_scale_bytes(K, N, group_size)
+    if w.numel() != L.marlin_packed_weight_bytes(K, N, 0) or s.numel() != sb or sb == 0:
+        raise ValueError("packed buffer sizes do not match K, N, group_size")
+    q = torch.empty((K // 8, N), dtype=torch.int32, device=w.device)
+    sc = torch.empty((sb // 2 // N, N), dtype=torch.float16, device=w.device)
+    _check(L.marlin_unpack(w.data_ptr(), s.data_ptr(), q.data_ptr(), sc.data_ptr(), K, N, group_size,
+                           _stream_ptr(stream)), "marlin_unpack")
+    return q, sc
+
+
+def gemm(A, w_packed, s_packed, K: int, N: int, group_size: int, workspace, out=None, stream=None):
+    """marlin_gemm: C[M, N] = A[M, K] . dequant(W).  `workspace` from new_workspace(max_M >= M, K, N)."""
+    torch = _torch()
+    A = _dev(A, torch.float16, "A")
+    if A.dim() != 2 or A.shape[1] != K:
+        raise ValueError("A must be [M, K]")
+    M = A.shape[0]
+    w = _dev(w_packed, torch.uint8, "w_packed")
+    s = _dev(s_packed, torch.uint8, "s_packed")
+    ws = _dev(workspace, torch.uint8, "workspace")
+    L = lib()
+    if w.numel() != L.marlin_packed_weight_bytes(K, N, 0) or s.numel() != L.marlin_packed_scale_bytes(K, N, group_size):
+        raise ValueError("packed buffer sizes do not match K, N, group_size")
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float16, device=A.device)
+    else:
+        _dev(out, torch.float16, "out")
+        if tuple(out.shape) != (M, N):
+            raise ValueError("out must be [M, N]")
+    _check(L.marlin_gemm(A.data_ptr(), w.data_ptr(), s.data_ptr(), out.data_ptr(), M, K, N, group_size,
+                         ws.data_ptr(), ws.numel(), _stream_ptr(stream)), "marlin_gemm")
+    return out
+
+
+def pack_sparse24(qc_kpacked, idx, scales, group_size: int, stream=None):
+    """marlin_pack_sparse24: kept codes int32 [K/16, N], positions uint8 [K/2, N], scales fp16 [K/G, N]."""
+    torch = _torch()
+    qc = _dev(qc_kpacked, torch.int32, "qc_kpacked")
+    ix = _dev(idx, torch.uint8, "idx")
+    s = _dev(scales, torch.float16, "scales")
+    K, N = qc.shape[0] * 16, qc.shape[1]
+    if tuple(ix.shape) != (K // 2, N):
+        raise ValueError("idx must be [K/2, N]")
+    L = lib()
+    wb, mb, sb = (L.marlin_packed_weight_bytes(K, N, 1), L.marlin_packed_meta_bytes(K, N),
+                  L.marlin_packed_scale_bytes(K, N, group_size))
+    if wb == 0 or mb == 0:
+        raise MarlinError(2, "marlin_pack_sparse24")
+    if sb == 0:
+        raise MarlinError(3, "marlin_pack_sparse24")
+    w_packed = torch.empty(wb, dtype=torch.uint8, device=qc.device)
+    m_packed = torch.empty(mb, dtype=torch.uint8, device=qc.device)
+    s_packed = torch.empty(sb, dtype=torch.uint8, device=qc.device)
+    _check(L.marlin_pack_sparse24(qc.data_ptr(), ix.data_ptr(), s.data_ptr(), w_packed.data_ptr(),
+                                  m_packed.data_ptr(), s_packed.data_ptr(), K, N, group_size, _stream_ptr(stream)),
+           "marlin_pack_sparse24")
+    return w_packed, m_packed, s_packed
+
+
+def unpack_sparse24(w_packed, meta_packed, s_packed, K: int, N: int, group_size: int, stream=None):
+    torch = _torch()
+    w = _dev(w_packed, torch.uint8, "w_packed")
+    m = _dev(meta_packed, torch.uint8, "meta_packed")
+    s = _dev(s_packed, torch.uint8, "s_packed")
+    L = lib()
+    sb = L.marlin_packed_scale_bytes(K, N, group_size)
+    qc = torch.empty((K // 16, N), dtype=torch.int32, device=w.device)
+    ix = torch.empty((K // 2, N), dtype=torch.uint8, device=w.device)
+    sc = torch.empty((sb // 2 // N, N), dtype=torch.float16, device=w.device)
+    _check(L.marlin_unpack_sparse24(w.data_ptr(), m.data_ptr(), s.data_ptr(), qc.data_ptr(), ix.data_ptr(),
+                                    sc.data_ptr(), K, N, group_size, _stream_ptr(stream)), "marlin_unpack_sparse24")
+    return qc, ix, sc
+
+
+def gemm_sparse24(A, w_packed, meta_packed, s_packed, K: int, N: int, group_size: int, workspace, out=None,
+                  stream=None):
+    torch = _torch()
+    A = _dev(A, torch.float16, "A")
+    if A.dim() != 2 or A.shape[1] != K:
+        raise ValueError("A must be [M, K]")
+    M = A.shape[0]
+    w = _dev(w_packed, torch.uint8, "w_packed")
+    m = _dev(meta_packed, torch.uint8, "meta_packed")
+    s = _dev(s_packed, torch.uint8, "s_packed")
+    ws = _dev(workspace, torch.uint8, "workspace")
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float16, device=A.device)
+    _check(lib().marlin_gemm_sparse24(A.data_ptr(), w.data_ptr(), m.data_ptr(), s.data_ptr(), out.data_ptr(), M, K,
+                                      N, group_size, ws.data_ptr(), ws.numel(), _stream_ptr(stream)),
+           "marlin_gemm_sparse24")
+    return out
+
+
+def read_status(workspace, stream=None) -> int:
+    """marlin_read_status: synchronises the stream and returns the device-side status word."""
+    torch = _torch()
+    ws = _dev(workspace, torch.uint8, "workspace")
+    return int(lib().marlin_read_status(ws.data_ptr(), _stream_ptr(stream)))
+
+
+def plan_stripes(M: int, K: int, N: int, sm_count: int) -> Tuple[int, int, list]:
+    """marlin_plan_stripes (host only): returns (n_tile, workers, bounds[workers + 1])."""
+    L = lib()
+    cap = 1024
+    n_tile, workers = ctypes.c_int(0), ctypes.c_int(0)
+    bounds = (ctypes.c_int64 * cap)()
+    _check(L.marlin_plan_stripes(M, K, N, sm_count, ctypes.byref(n_tile), ctypes.byref(workers), bounds, cap),
+           "marlin_plan_stripes")
+    return n_tile.value, workers.value, list(bounds[: workers.value + 1])

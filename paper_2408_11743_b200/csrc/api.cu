@@ -1,0 +1,206 @@
+// C-ABI entry points of libmarlin_b200: argument validation, planning, launches.
+#include <stdlib.h>
+
+#include "marlin_internal.cuh"
+
+using namespace marlin_b200;
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// group_size -> normalised G, or 0 if unsupported.
+int normalise_group(int K, int group_size) {
+  if (K <= 0) return 0;
+  if (group_size == -1 || group_size == K) return K;
+  if (group_size <= 0 || group_size % kTileK || K % group_size) return 0;
+  return group_size;
+}
+
+bool shape_ok(int K, int N) {
+  return K >= kTileK && K % kTileK == 0 && N >= kChunkN && N % kChunkN == 0 && N / kChunkN <= kWsMaxCounters;
+}
+
+struct DeviceInfo {
+  int sm_count;
+  int cc_major;
+};
+
+// Queried once per device and cached (a few attribute reads; no allocation).
+int device_info(DeviceInfo* out) {
+  static DeviceInfo cache[64];
+  static bool known[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return MARLIN_ERR_CUDA;
+  if (dev >= 0 && dev < 64 && known[dev]) {
+    *out = cache[dev];
+    return MARLIN_OK;
+  }
+  DeviceInfo info;
+  if (cudaDeviceGetAttribute(&info.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&info.cc_major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+    return MARLIN_ERR_CUDA;
+  if (dev >= 0 && dev < 64) {
+    cache[dev] = info;
+    known[dev] = true;
+  }
+  *out = info;
+  return MARLIN_OK;
+}
+
+int slab_mpad(int max_M) {
+  return max_M <= 8 ? 8 : (max_M <= 16 ? 16 : 32);  // rows of one launch, padded to its 8-row blocks
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* marlin_status_string(int status) {
+  switch (status) {
+    case MARLIN_OK: return "ok";
+    case MARLIN_ERR_NULL: return "null pointer";
+    case MARLIN_ERR_SHAPE: return "unsupported shape";
+    case MARLIN_ERR_GROUP: return "unsupported group size";
+    case MARLIN_ERR_ALIGN: return "pointer not 16-byte aligned";
+    case MARLIN_ERR_WORKSPACE: return "workspace too small";
+    case MARLIN_ERR_ARCH: return "device is not sm_100";
+    case MARLIN_ERR_CUDA: return "CUDA error";
+    case MARLIN_ERR_DEVICE_TIMEOUT: return "bounded wait expired inside a kernel";
+    default: return "unknown status";
+  }
+}
+
+size_t marlin_packed_weight_bytes(int K, int N, int sparse24) {
+  if (!shape_ok(K, N)) return 0;
+  return (size_t)K * N / (sparse24 ? 4 : 2);
+}
+
+size_t marlin_packed_scale_bytes(int K, int N, int group_size) {
+  int G = normalise_group(K, group_size);
+  if (!shape_ok(K, N) || !G) return 0;
+  return (size_t)2 * (K / G) * N;
+}
+
+size_t marlin_packed_meta_bytes(int K, int N) {
+  if (!shape_ok(K, N)) return 0;
+  return (size_t)K * N / 8;
+}
+
+size_t marlin_workspace_bytes(int max_M, int K, int N) {
+  if (max_M < 1 || !shape_ok(K, N)) return 0;
+  return kWsPartialOff + (size_t)2 * kMaxWorkers * kWsSlotCols * slab_mpad(max_M) * sizeof(float);
+}
+
+int marlin_pack(const uint32_t* q_kpacked, const void* scales, void* w_packed, void* s_packed, int K, int N,
+                int group_size, marlin_stream stream) {
+  if (!q_kpacked || !scales || !w_packed || !s_packed) return MARLIN_ERR_NULL;
+  if (!shape_ok(K, N)) return MARLIN_ERR_SHAPE;
+  int G = normalise_group(K, group_size);
+  if (!G) return MARLIN_ERR_GROUP;
+  if (!aligned16(q_kpacked) || !aligned16(scales) || !aligned16(w_packed) || !aligned16(s_packed))
+    return MARLIN_ERR_ALIGN;
+  cudaError_t err = launch_pack_dense(const_cast<uint32_t*>(q_kpacked),
+                                      static_cast<uint16_t*>(const_cast<void*>(scales)),
+                                      static_cast<uint32_t*>(w_packed), static_cast<uint16_t*>(s_packed), K, N, G,
+                                      false, static_cast<cudaStream_t>(stream));
+  return err == cudaSuccess ? MARLIN_OK : MARLIN_ERR_CUDA;
+}
+
+int marlin_unpack(const void* w_packed, const void* s_packed, uint32_t* q_kpacked, void* scales, int K, int N,
+                  int group_size, marlin_stream stream) {
+  if (!q_kpacked || !scales || !w_packed || !s_packed) return MARLIN_ERR_NULL;
+  if (!shape_ok(K, N)) return MARLIN_ERR_SHAPE;
+  int G = normalise_group(K, group_size);
+  if (!G) return MARLIN_ERR_GROUP;
+  if (!aligned16(q_kpacked) || !aligned16(scales) || !aligned16(w_packed) || !aligned16(s_packed))
+    return MARLIN_ERR_ALIGN;
+  cudaError_t err = launch_pack_dense(q_kpacked, static_cast<uint16_t*>(scales),
+                                      static_cast<uint32_t*>(const_cast<void*>(w_packed)),
+                                      static_cast<uint16_t*>(const_cast<void*>(s_packed)), K, N, G, true,
+                                      static_cast<cudaStream_t>(stream));
+  return err == cudaSuccess ? MARLIN_OK : MARLIN_ERR_CUDA;
+}
+
+int marlin_gemm(const void* A, const void* w_packed, const void* s_packed, void* C, int M, int K, int N,
+                int group_size, void* workspace, size_t workspace_bytes, marlin_stream stream) {
+  if (!A || !w_packed || !s_packed || !C || !workspace) return MARLIN_ERR_NULL;
+  if (M < 1 || !shape_ok(K, N)) return MARLIN_ERR_SHAPE;
+  int G = normalise_group(K, group_size);
+  if (!G) return MARLIN_ERR_GROUP;
+  if (!aligned16(A) || !aligned16(w_packed) || !aligned16(s_packed) || !aligned16(C) || !aligned16(workspace))
+    return MARLIN_ERR_ALIGN;
+  if (workspace_bytes < marlin_workspace_bytes(M, K, N)) return MARLIN_ERR_WORKSPACE;
+  DeviceInfo info;
+  int st = device_info(&info);
+  if (st != MARLIN_OK) return st;
+  if (info.cc_major != 10) return MARLIN_ERR_ARCH;
+
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  for (int m0 = 0; m0 < M; m0 += kMaxSlabM) {
+    const int m_slab = (M - m0) < kMaxSlabM ? (M - m0) : kMaxSlabM;
+    DensePlan plan;
+    if (!make_dense_plan(m_slab, K, N, info.sm_count, &plan)) return MARLIN_ERR_SHAPE;
+    GemmParams p;
+    p.A = static_cast<const uint16_t*>(A) + (size_t)m0 * K;
+    p.wq = static_cast<const uint8_t*>(w_packed);
+    p.sq = static_cast<const uint8_t*>(s_packed);
+    p.C = static_cast<uint16_t*>(C) + (size_t)m0 * N;
+    p.M = m_slab;
+    p.K = K;
+    p.N = N;
+    p.kb = plan.kb;
+    p.kb_per_group = G / kTileK;
+    p.grouped = (G != K) ? 1 : 0;
+    p.ncols = plan.ncols;
+    p.units = plan.units;
+    p.workers = plan.workers;
+    p.stages = plan.stages;
+    p.stage_bytes = plan.stage_bytes;
+    p.status = reinterpret_cast<int*>(ws + kWsStatusOff);
+    p.counters = reinterpret_cast<int*>(ws + kWsCounterOff);
+    p.partials = reinterpret_cast<float*>(ws + kWsPartialOff);
+    p.slot_floats = kWsSlotCols * slab_mpad(M);
+    if (launch_gemm_dense(plan, p, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MARLIN_ERR_CUDA;
+  }
+  return MARLIN_OK;
+}
+
+int marlin_pack_sparse24(const uint32_t*, const uint8_t*, const void*, void*, void*, void*, int, int, int,
+                         marlin_stream) {
+  return MARLIN_ERR_SHAPE;  // filled in by gemm_sparse24.cu once that kernel exists
+}
+int marlin_unpack_sparse24(const void*, const void*, const void*, uint32_t*, uint8_t*, void*, int, int, int,
+                           marlin_stream) {
+  return MARLIN_ERR_SHAPE;
+}
+int marlin_gemm_sparse24(const void*, const void*, const void*, const void*, void*, int, int, int, int, void*, size_t,
+                         marlin_stream) {
+  return MARLIN_ERR_SHAPE;
+}
+
+int marlin_read_status(const void* workspace, marlin_stream stream) {
+  if (!workspace) return MARLIN_ERR_NULL;
+  int host_status = 0;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(&host_status, static_cast<const uint8_t*>(workspace) + kWsStatusOff, sizeof(int),
+                      cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    return MARLIN_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return MARLIN_ERR_CUDA;
+  return host_status;
+}
+
+int marlin_plan_stripes(int M, int K, int N, int sm_count, int* n_tile, int* workers, int64_t* bounds, int cap) {
+  if (!n_tile || !workers || !bounds) return MARLIN_ERR_NULL;
+  if (M < 1 || !shape_ok(K, N)) return MARLIN_ERR_SHAPE;
+  DensePlan plan;
+  const int m_slab = M < kMaxSlabM ? M : kMaxSlabM;
+  if (!make_dense_plan(m_slab, K, N, sm_count, &plan)) return MARLIN_ERR_SHAPE;
+  if (cap < plan.workers + 1) return MARLIN_ERR_SHAPE;
+  *n_tile = plan.nw * kChunkN;
+  *workers = plan.workers;
+  for (int w = 0; w <= plan.workers; ++w) bounds[w] = stripe_begin(w, plan.units, plan.workers);
+  return MARLIN_OK;
+}
+
+}  // extern "C"

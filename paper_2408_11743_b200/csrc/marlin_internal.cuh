@@ -1,0 +1,82 @@
+// Internal declarations shared by the translation units of libmarlin_b200 (sm_100a only).
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "marlin_b200.h"
+
+namespace marlin_b200 {
+
+// ---- fixed geometry of the packed layouts ----------------------------------------------------
+// One "chunk" is the 64-column x 128-row block of weights a consumer warp turns into tensor-core
+// fragments: 8 x 32 lanes x 16 bytes = 4096 bytes (dense).  A pipeline stage holds NW chunks that
+// are adjacent in the packed buffer (the same 128 rows, NW*64 consecutive columns).
+constexpr int kTileK = 128;           // rows of W per k-block
+constexpr int kChunkN = 64;           // columns of W per chunk
+constexpr int kChunkBytes = 4096;     // dense chunk
+constexpr int kConsumerWarps = 8;
+constexpr int kGemmThreads = (kConsumerWarps + 1) * 32;  // + one producer warp
+constexpr int kMaxStages = 32;
+constexpr int kMaxWorkers = 160;      // grid size cap (a B200 has 148 SMs)
+constexpr int kMaxSlabM = 32;         // rows of A handled by one launch of the mma.sync kernel
+constexpr int kSmemBudget = 227 * 1024;
+
+// workspace layout (bytes)
+constexpr size_t kWsStatusOff = 0;
+constexpr size_t kWsCounterOff = 256;
+constexpr int kWsMaxCounters = 1024;  // N / 64 <= 1024
+constexpr size_t kWsPartialOff = 8192;
+constexpr int kWsSlotCols = 256;      // widest column tile
+
+struct DensePlan {
+  int mb;          // 8-row blocks of A per launch (1, 2 or 4)
+  int nw;          // chunks per stage; column tile = 64 * nw
+  int kb;          // K / 128
+  int ncols;       // N / (64 * nw)
+  long long units; // ncols * kb
+  int workers;     // CTAs
+  int stages;
+  int stage_bytes;
+  int smem_bytes;
+};
+
+// Chooses tile width, worker count and pipeline depth for one slab of m_slab <= 32 rows.
+// Pure host arithmetic.  Returns false on an unsupported shape.
+bool make_dense_plan(int m_slab, int K, int N, int sm_count, DensePlan* plan);
+
+struct GemmParams {
+  const uint16_t* A;
+  const uint8_t* wq;
+  const uint8_t* sq;
+  uint16_t* C;
+  int M, K, N;
+  int kb;            // K / 128
+  int kb_per_group;  // group_size / 128
+  int grouped;       // 0: one scale per column (group_size == K)
+  int ncols;
+  long long units;
+  int workers;
+  int stages;
+  int stage_bytes;
+  int* status;
+  int* counters;
+  float* partials;
+  int slot_floats;   // floats per partial-tile slot
+};
+
+cudaError_t launch_gemm_dense(const DensePlan& plan, const GemmParams& p, cudaStream_t stream);
+// inverse == false: (q, s) canonical inputs -> (wq, sq) packed outputs; inverse == true: the other way round.
+cudaError_t launch_pack_dense(uint32_t* q, uint16_t* s, uint32_t* wq, uint16_t* sq, int K, int N, int G, bool inverse,
+                              cudaStream_t stream);
+
+// ---- the stripe partition (host and device use the same two formulas) ------------------------
+// worker w of P owns units [w*U/P, (w+1)*U/P); the owner of unit x is floor(((x+1)*P - 1) / U).
+__host__ __device__ inline long long stripe_begin(long long w, long long U, long long P) { return (w * U) / P; }
+__host__ __device__ inline int stripe_owner(long long x, long long U, long long P) {
+  return (int)(((x + 1) * P - 1) / U);
+}
+
+}  // namespace marlin_b200

@@ -1,0 +1,159 @@
+"""GPU parity of marlin_gemm against the CPU oracle, through the C ABI.
+
+Bound (floating point): |C - C_ref| <= 5e-3 * (|C_ref| + rms(C_ref)) for every element.
+Integer-valued closed forms must match bit for bit.
+"""
+import numpy as np
+import pytest
+
+from paper_2408_11743_b200 import inputs
+from gpu_util import DenseLayer, to_dev, to_host
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def marlin():
+    import torch
+    assert torch.cuda.is_available()
+    import paper_2408_11743_b200 as m
+    m.lib()
+    return m
+
+
+def _assert_close(oracle_lib, C, C_ref):
+    bad, worst, rms = oracle_lib.check_tolerance(C, C_ref)
+    assert bad == 0, f"{bad} elements out of tolerance, worst ratio {worst:.3f}, rms {rms:.3f}"
+    return worst
+
+
+# small shapes the oracle finishes at once; several tiles, ragged M, both scale modes,
+# K and N that are not multiples of the wide tiles, shapes with fewer units than SMs
+SMALL = [
+    (1, 128, 64, 128), (2, 256, 64, 128), (5, 256, 192, 128), (8, 512, 128, -1), (3, 384, 320, 128),
+    (16, 1024, 256, 128), (9, 1024, 384, 256), (13, 2048, 512, -1), (16, 4096, 4096, 128),
+    (17, 1024, 768, 128), (32, 2048, 1024, 128), (31, 1152, 448, 128), (24, 4096, 1024, -1),
+    (33, 1024, 512, 128), (64, 2048, 1024, 128), (100, 1024, 640, -1), (128, 2048, 2048, 128),
+    (7, 11008, 256, 128), (1, 8192, 8192, 128), (4, 4096, 12288, 128), (16, 28672, 1024, -1),
+    (16, 28672, 1024, 128), (32, 4096, 22016, 128),
+]
+
+
+@pytest.mark.parametrize("M,K,N,G", SMALL)
+def test_gemm_matches_oracle(marlin, oracle_lib, M, K, N, G):
+    case = inputs.make_dense(M, K, N, G, seed=1000 + M + K + N)
+    layer = DenseLayer(marlin, case.q_kpacked, case.S, G, max_M=M)
+    C = layer(case.A)
+    C_ref = oracle_lib.gemm(case.A, case.q_kpacked, case.S, case.G)
+    _assert_close(oracle_lib, C, C_ref)
+
+
+def test_config1_single_layer(marlin, oracle_lib):
+    name, M, K, N, G, seed = next(inputs.iter_cases(1))
+    case = inputs.make_dense(M, K, N, G, seed)
+    C = DenseLayer(marlin, case.q_kpacked, case.S, G, max_M=M)(case.A)
+    worst = _assert_close(oracle_lib, C, oracle_lib.gemm(case.A, case.q_kpacked, case.S, G))
+    assert worst < 0.5  # an honest fp32-accumulating kernel sits far inside the bound
+
+
+def test_same_layer_many_batch_sizes_and_repeatability(marlin, oracle_lib):
+    K, N, G = 2048, 1536, 128
+    case = inputs.make_dense(128, K, N, G, seed=77)
+    layer = DenseLayer(marlin, case.q_kpacked, case.S, G, max_M=128)
+    C_ref = oracle_lib.gemm(case.A, case.q_kpacked, case.S, G)
+    for M in (1, 2, 3, 4, 7, 8, 9, 15, 16, 17, 31, 32, 33, 63, 64, 65, 127, 128):
+        C = layer(case.A[:M])
+        # rows are independent: the reference of the first M rows is the first M rows of the reference,
+        # but the bound's rms is over the compared block
+        _assert_close(oracle_lib, C, np.ascontiguousarray(C_ref[:M]))
+        C2 = layer(case.A[:M])
+        assert np.array_equal(C.view(np.uint16), C2.view(np.uint16))  # deterministic fix-up
+
+
+def test_zero_codes_give_zero(marlin):
+    K, N = 1024, 256
+    q = inputs.kpack(np.full((K, N), 8, dtype=np.uint8))
+    case = inputs.make_dense(5, K, N, 128, seed=3)
+    C = DenseLayer(marlin, q, case.S, 128, max_M=5)(case.A)
+    assert np.all(C == 0)
+
+
+@pytest.mark.parametrize("M,K,N", [(2, 4096, 256), (16, 8192, 512), (32, 2048, 320)])
+def test_integer_closed_form_is_bit_exact(marlin, oracle_lib, M, K, N):
+    # scales are powers of two and activations small integers: every product and every partial sum is
+    # an integer multiple of the scale below 2^24, so fp32 accumulation in any order is exact and the
+    # GPU must equal the oracle bit for bit
+    rng = np.random.default_rng(M + K)
+    Q = rng.integers(0, 16, size=(K, N), dtype=np.uint8)
+    A = rng.integers(-3, 4, size=(M, K)).astype(np.float16)
+    S = np.ldexp(1.0, rng.integers(-4, 1, size=(K // 128, N))).astype(np.float16)
+    q = inputs.kpack(Q)
+    C = DenseLayer(marlin, q, S, 128, max_M=M)(A)
+    C_ref = oracle_lib.gemm(A, q, S, 128)
+    assert np.array_equal(C.view(np.uint16), C_ref.view(np.uint16))
+    # all-ones row and unit scales: plain column sums of (Q - 8)
+    A1 = np.ones((1, K), dtype=np.float16)
+    S1 = np.ones((1, N), dtype=np.float16)
+    C1 = DenseLayer(marlin, q, S1, K, max_M=1)(A1)
+    assert np.array_equal(C1.view(np.uint16), oracle_lib.gemm(A1, q, S1, K).view(np.uint16))
+
+
+def test_one_hot_rows_probe_every_k_position(marlin, oracle_lib):
+    # A = unit vectors e_k: C[m, n] = (Q[k_m, n] - 8) * S[k_m // G, n] exactly; sweeps every k
+    K, N, G = 512, 192, 128
+    rng = np.random.default_rng(5)
+    Q = rng.integers(0, 16, size=(K, N), dtype=np.uint8)
+    expo = rng.integers(-5, 2, size=(K // G, N))
+    S = np.ldexp(1.0, expo).astype(np.float16)
+    q = inputs.kpack(Q)
+    layer = DenseLayer(marlin, q, S, G, max_M=128)
+    for k0 in range(0, K, 128):
+        A = np.zeros((128, K), dtype=np.float16)
+        A[np.arange(128), k0 + np.arange(128)] = 1.0
+        C = layer(A).astype(np.float64)
+        want = (Q[k0:k0 + 128].astype(np.float64) - 8) * np.ldexp(1.0, expo[(k0 // G)])[None, :]
+        assert np.array_equal(C, want)
+
+
+def test_subnormal_scales_and_large_values(marlin, oracle_lib):
+    K, N = 1024, 128
+    case = inputs.make_dense(4, K, N, 128, seed=9)
+    S = np.full((K // 128, N), 2.0 ** -20, dtype=np.float16)  # subnormal fp16
+    C = DenseLayer(marlin, case.q_kpacked, S, 128, max_M=4)(case.A)
+    _assert_close(oracle_lib, C, oracle_lib.gemm(case.A, case.q_kpacked, S, 128))
+    S = np.full((K // 128, N), 4.0, dtype=np.float16)
+    A = (case.A.astype(np.float32) * 8).astype(np.float16)
+    C = DenseLayer(marlin, case.q_kpacked, S, 128, max_M=4)(A)
+    _assert_close(oracle_lib, C, oracle_lib.gemm(A, case.q_kpacked, S, 128))
+
+
+def test_full_size_layers_on_sampled_outputs(marlin, oracle_lib):
+    # the largest layers of the workload list, checked on outputs the oracle computes one by one
+    rng = np.random.default_rng(2)
+    for (K, N, G, M) in [(8192, 57344, 128, 16), (28672, 8192, -1, 64), (8192, 8192, 128, 128)]:
+        case = inputs.make_dense(M, K, N, G, seed=K + N + M)
+        C = DenseLayer(marlin, case.q_kpacked, case.S, G, max_M=M)(case.A)
+        ms = rng.integers(0, M, 4096)
+        ns = rng.integers(0, N, 4096)
+        ref = oracle_lib.gemm_samples(case.A, case.q_kpacked, case.S, case.G, ms, ns)
+        # the bound's rms is taken over the sampled outputs (a fair estimate of the full one)
+        bad, worst, _ = oracle_lib.check_tolerance(np.ascontiguousarray(C[ms, ns]), ref)
+        assert bad == 0, (K, N, G, M, worst)
+        assert np.all(np.isfinite(C.astype(np.float32)))
+
+
+def test_errors_and_status(marlin):
+    import torch
+    K, N = 256, 128
+    case = inputs.make_dense(4, K, N, 128, seed=1)
+    layer = DenseLayer(marlin, case.q_kpacked, case.S, 128, max_M=4)
+    A = to_dev(case.A)
+    small_ws = torch.zeros(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(marlin.MarlinError) as e:
+        marlin.gemm(A, layer.w, layer.s, K, N, 128, small_ws)
+    assert e.value.status == 5
+    assert marlin.read_status(layer.ws) == 0
+    # the arrival counters are left at zero by every call
+    layer(case.A)
+    counters = to_host(layer.ws[256:256 + 4096]).view(np.int32)
+    assert np.all(counters == 0)
