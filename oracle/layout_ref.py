@@ -4,8 +4,11 @@ Written from the layout description in DESIGN.md ("Packed layout"), not from the
 used only to compare bytes with what ``marlin_pack`` writes on the GPU.  Nothing in the product
 imports this file.
 
-Dense layout: the packed buffer is a sequence of uint32 words,
-    word index = (((kb * (N/64) + nb) * 8 + i) * 32 + lane) * 4 + t
+Dense layout: the packed buffer is a sequence of 4096-byte chunks, one per (k-block kb = k/128,
+64-column block nb = n/64), ordered by super-columns of four chunks:
+    chunk index = (nb/4) * 4 * (K/128) + kb * cs + nb % 4,   cs = min(4, N/64 - 4*(nb/4))
+Inside a chunk
+    word index = (i * 32 + lane) * 4 + t
 with i = 4*h + j and lane = 4*g + c, and nibble p (bits 4p..4p+3) of that word holds the code at
     column n = 64*nb + 16*j + g + 8*(p & 1)
     row    k = 128*kb + 64*h + 16*c + 4*t + 2*((p >> 1) & 1) + (p >> 2)
@@ -29,7 +32,15 @@ def pack_dense_weights(Q: np.ndarray) -> np.ndarray:
     words = np.zeros(codes.shape[:-1], dtype=np.uint32)
     for pp in range(8):
         words |= codes[..., pp] << np.uint32(4 * pp)
-    return words.reshape(-1)
+    chunks = words.reshape(K // 128, N // 64, 1024)  # [kb, nb, words of the chunk]
+    KB, NB = K // 128, N // 64
+    out = np.empty((KB * NB, 1024), dtype=np.uint32)
+    for nb_ in range(NB):
+        sc = nb_ // 4
+        cs = min(4, NB - 4 * sc)
+        idx = sc * 4 * KB + np.arange(KB) * cs + nb_ % 4
+        out[idx] = chunks[:, nb_, :]
+    return out.reshape(-1)
 
 
 def pack_scales(S: np.ndarray) -> np.ndarray:

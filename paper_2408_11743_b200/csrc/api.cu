@@ -18,7 +18,9 @@ int normalise_group(int K, int group_size) {
 }
 
 bool shape_ok(int K, int N) {
-  return K >= kTileK && K % kTileK == 0 && N >= kChunkN && N % kChunkN == 0 && N / kChunkN <= kWsMaxCounters;
+  // the device's 32-bit stripe arithmetic needs (N/64) * (K/128) * workers < 2^32
+  return K >= kTileK && K % kTileK == 0 && K <= (1 << 20) && N >= kChunkN && N % kChunkN == 0 &&
+         N / kChunkN <= kWsMaxCounters;
 }
 
 struct DeviceInfo {
@@ -149,12 +151,12 @@ int marlin_gemm(const void* A, const void* w_packed, const void* s_packed, void*
     p.M = m_slab;
     p.K = K;
     p.N = N;
-    p.kb = plan.kb;
+    p.kb = (uint32_t)plan.kb;
     p.kb_per_group = G / kTileK;
     p.grouped = (G != K) ? 1 : 0;
     p.ncols = plan.ncols;
-    p.units = plan.units;
-    p.workers = plan.workers;
+    p.units = (uint32_t)plan.units;
+    p.workers = (uint32_t)plan.workers;
     p.stages = plan.stages;
     p.stage_bytes = plan.stage_bytes;
     p.status = reinterpret_cast<int*>(ws + kWsStatusOff);

@@ -1,20 +1,26 @@
 // Dense W4A16 layer for sm_100a, decode batch sizes (one launch handles up to 32 rows of A).
 //
 // Structure of one CTA (one per SM, persistent over its stripe of work units):
-//   warp 8        producer: one elected lane issues bulk-async copies (cp.async.bulk + mbarrier
-//                 complete_tx) of the packed weight chunks, the group scales and the A rows of one
-//                 k-block into a ring of shared-memory stages; weights carry an L2 evict-first policy
-//                 (each byte is read once), activations evict-last (re-read by every column tile).
+//   warp 8        producer: per k-block ONE bulk-async copy (cp.async.bulk + mbarrier complete_tx) of
+//                 the contiguous packed weights of the column tile and one TMA tensor-tile copy per
+//                 64-wide half of the A tile (128-byte swizzle, rows beyond M zero-filled by the
+//                 hardware) into a ring of shared-memory stages.  Weights carry an L2 evict-first
+//                 policy (each byte is read once), activations evict-last (re-read by every tile).
+//                 Issuing a bulk copy costs the producer on the order of a hundred cycles whatever
+//                 its size, so the design keeps copies few and large.
 //   warps 0..7    consumers, arranged as SK groups of NW warps.  Stage number `it` of the CTA is
 //                 consumed by group it % SK; inside a group warp wn owns 64 output columns.  A warp
 //                 reads its 16-byte weight vectors, converts the 4-bit codes to fp16 (q - 8) with the
 //                 exponent-bias trick, and feeds mma.sync.m16n8k16 with the WEIGHTS as the 16-wide
 //                 operand and the batch on the 8-wide one, so that batch sizes 1..8 cost one MMA per
 //                 256 weights.  The group scale is not applied to the weights: each group of k
-//                 accumulates into `tmp`, and `acc += s * tmp` in fp32 when the group ends.
+//                 accumulates into `tmp`, and `acc += s * tmp` in fp32 when the group ends; the
+//                 scales themselves are read straight from global memory (one 16-byte load per lane
+//                 and group, issued a whole stage before its use).
 //   end of a column segment: tree reduction of the SK groups through shared memory, then the stripe
 //                 fix-up across CTAs: partial tiles go to the workspace in fp32, an arrival counter
-//                 tells the last CTA of a column tile to add them in stripe order and write fp16 C.
+//                 (acq_rel atomic) tells the last CTA of a column tile to add them in stripe order,
+//                 with all its threads and all loads in flight at once, and write fp16 C.
 //                 Nobody spins on another CTA.
 //
 // Paper correspondence (Section 3.4): weight streaming and evict-first ("Maximizing Loading
@@ -23,6 +29,9 @@
 // ("Dequantization and Tensor Cores"), scales ("Groups and Instruction Ordering"), stripes and the
 // global reduction ("Striped Partitioning").  What differs from the paper's Ampere design is listed
 // in the design document of this repository.
+#include <cuda.h>
+#include <stdlib.h>
+
 #include "marlin_internal.cuh"
 
 namespace marlin_b200 {
@@ -101,6 +110,20 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
       ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(pol)
       : "memory");
 }
+// One box of a 2-D tensor map -> shared memory (no multicast: every CTA fetches its own copy).
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar,
+                                            uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%2, %3}], [%4], %5;"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(pol)
+      : "memory");
+}
+__device__ __forceinline__ int atom_add_acq_rel_gpu(int* addr, int v) {
+  int old;
+  asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(addr), "r"(v) : "memory");
+  return old;
+}
 __device__ __forceinline__ void named_bar_sync(int id, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
@@ -139,7 +162,7 @@ __device__ __forceinline__ void dequant8(uint32_t w, uint32_t (&a)[4]) {
 }
 
 __device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
+  asm(
       "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
@@ -150,37 +173,41 @@ __device__ __forceinline__ float4 ld_cg_f4(const float4* p) { return __ldcg(p); 
 // ---------------------------------------------------------------------------------------------
 // shared memory map
 // ---------------------------------------------------------------------------------------------
-constexpr int kBarBytes = 1024;  // full[32], empty[32], flags
-constexpr int kARowBytes = kTileK * 2 + 16;  // 272: rows 16 bytes apart modulo 128 -> conflict-free 16-byte reads
+constexpr int kBarBytes = 1024;  // full[32] at 0, empty[32] at 256, flags at 512
 
 template <int MB, int NW>
 struct Geometry {
-  static constexpr int SK = kConsumerWarps / NW;
+  static constexpr int SK = kConsumerWarps / NW;             // groups of warps that split K
   static constexpr int MPAD = MB * 8;
-  static constexpr int NT = NW * 64;
+  static constexpr int NT = NW * kChunkN;
+  static constexpr int A_HALF_BYTES = MPAD * 128;            // one 64-wide half of the A tile: MPAD rows x 128 B
+  static constexpr int A_BYTES = 2 * A_HALF_BYTES;
   static constexpr int W_BYTES = NW * kChunkBytes;
-  static constexpr int S_BYTES = NW * 128;
-  static constexpr int A_OFF = W_BYTES + S_BYTES;
+  static constexpr int STAGE_BYTES = A_BYTES + W_BYTES;      // multiple of 1024
   static constexpr int FRAG_F4 = MB * 4;                     // float4 accumulator registers per thread
-  static constexpr int TILE_FLOATS = NW * 32 * FRAG_F4 * 4;  // one partial tile
-  static constexpr int RED_BYTES = (SK / 2) * TILE_FLOATS * 4;
+  static constexpr int TILE_F4 = NW * FRAG_F4 * 32;          // float4s of one partial tile
+  static constexpr int RED_BYTES = (SK / 2) * TILE_F4 * 16;
   static constexpr int CST_STRIDE = NT + 8;                  // halves
-  static constexpr int CST_BYTES = ((MPAD * CST_STRIDE * 2 + 127) / 128) * 128;
-  static constexpr int STAGE_BYTES = ((A_OFF + MPAD * kARowBytes + 127) / 128) * 128;
-  static constexpr int FIXED_BYTES = kBarBytes + RED_BYTES + CST_BYTES;
+  static constexpr int CST_BYTES = MPAD * CST_STRIDE * 2;
+  static constexpr int FIXED_BYTES = ((kBarBytes + RED_BYTES + CST_BYTES + 1023) / 1024) * 1024;
+  static constexpr int ALIGN_SLACK = 1024;                   // the stage ring is placed on a 1024-byte boundary
 };
 
 // ---------------------------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------------------------
 template <int MB, int NW>
-__global__ void __launch_bounds__(kGemmThreads, 1) gemm_dense_kernel(const GemmParams p) {
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a) {
   using G = Geometry<MB, NW>;
   constexpr int SK = G::SK;
-  extern __shared__ __align__(128) uint8_t smem[];
+  constexpr int kConsumerThreads = kConsumerWarps * 32;
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  // 128-byte-swizzled TMA tiles need their shared address aligned to the 1024-byte swizzle period
+  uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   uint64_t* full = reinterpret_cast<uint64_t*>(smem);
-  uint64_t* empty = full + kMaxStages;
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + 2 * kMaxStages * 8);
+  uint64_t* empty = reinterpret_cast<uint64_t*>(smem + 256);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + 512);
   volatile int* last_flag = abort_flag + 1;
   float4* red = reinterpret_cast<float4*>(smem + kBarBytes);
   uint16_t* cst = reinterpret_cast<uint16_t*>(smem + kBarBytes + G::RED_BYTES);
@@ -188,53 +215,55 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_dense_kernel(const GemmP
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int worker = blockIdx.x;
-  const long long U = p.units, P = p.workers;
-  const long long u0 = stripe_begin(worker, U, P), u1 = stripe_begin(worker + 1, U, P);
-  const int KB = p.kb;
+  const uint32_t worker = blockIdx.x;
+  const uint32_t U = p.units, P = p.workers, KB = p.kb;
+  const uint32_t u0 = stripe_begin32(worker, U, P), u1 = stripe_begin32(worker + 1, U, P);
   const int nstages = p.stages;
 
+  if ((int)threadIdx.x < nstages) {
+    mbar_init(&full[threadIdx.x], 1);
+    mbar_init(&empty[threadIdx.x], NW);
+  }
   if (threadIdx.x == 0) {
-    for (int s = 0; s < nstages; ++s) {
-      mbar_init(&full[s], 1);
-      mbar_init(&empty[s], NW);
-    }
     *abort_flag = 0;
     *last_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // rows of the A tile at or beyond M are never copied; give them a defined value once
-  for (int s = 0; s < nstages; ++s) {
-    uint4* arows = reinterpret_cast<uint4*>(stage0 + (size_t)s * G::STAGE_BYTES + G::A_OFF);
-    for (int x = threadIdx.x; x < G::MPAD * kARowBytes / 16; x += kGemmThreads) arows[x] = make_uint4(0, 0, 0, 0);
-  }
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   __syncthreads();
 
   if (warp == kConsumerWarps) {
     // ------------------------------- producer ---------------------------------------------
+    if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
     const uint64_t pol_w = policy_evict_first();
     const uint64_t pol_a = policy_evict_last();
-    const uint32_t tx_bytes = G::W_BYTES + (p.grouped ? G::S_BYTES : 0) + p.M * (kTileK * 2);
-    const int nb64 = p.N / 64;
+    constexpr uint32_t tx_bytes = G::W_BYTES + G::A_BYTES;  // out-of-range rows of the box count too
+    const uint32_t nb64 = p.N / kChunkN;
     int s = 0;
     uint32_t ph = 0;
-    int col = (int)(u0 / KB), kb = (int)(u0 % KB);
-    for (long long u = u0; u < u1; ++u) {
+    uint32_t col = u0 / KB, kb = u0 % KB;
+    // weights of (kb, col): super-columns of four chunks, k-blocks contiguous inside a super-column
+    uint32_t nb = col * NW;
+    uint32_t sc = nb >> 2, cs = min(4u, nb64 - 4u * sc);
+    const uint8_t* wsrc = p.wq + ((size_t)sc * 4u * KB + (size_t)kb * cs + (nb & 3u)) * kChunkBytes;
+    for (uint32_t u = u0; u < u1; ++u) {
       mbar_wait(&empty[s], ph ^ 1u, abort_flag, p.status);
       uint8_t* st = stage0 + (size_t)s * G::STAGE_BYTES;
-      if (lane == 0) mbar_expect_tx(&full[s], tx_bytes);
+      if (lane == 0) {
+        mbar_expect_tx(&full[s], tx_bytes);
+        bulk_g2s(st + G::A_BYTES, wsrc, G::W_BYTES, &full[s], pol_w);
+      }
       __syncwarp();
-      if (lane == 0)
-        bulk_g2s(st, p.wq + ((size_t)kb * nb64 + (size_t)col * NW) * kChunkBytes, G::W_BYTES, &full[s], pol_w);
-      if (lane == 1 && p.grouped)
-        bulk_g2s(st + G::W_BYTES, p.sq + ((size_t)(kb / p.kb_per_group) * p.N + (size_t)col * G::NT) * 2, G::S_BYTES,
-                 &full[s], pol_w);
-      for (int m = lane; m < p.M; m += 32)
-        bulk_g2s(st + G::A_OFF + m * kARowBytes, p.A + (size_t)m * p.K + (size_t)kb * kTileK, kTileK * 2, &full[s],
-                 pol_a);
+      if (lane < 2) tma_load_2d(st + lane * G::A_HALF_BYTES, &tmap_a, (int)(kb * kTileK + lane * 64), 0, &full[s], pol_a);
       if (++s == nstages) { s = 0; ph ^= 1u; }
-      if (++kb == KB) { kb = 0; ++col; }
+      wsrc += (size_t)cs * kChunkBytes;
+      if (++kb == KB) {
+        kb = 0;
+        ++col;
+        nb = col * NW;
+        sc = nb >> 2;
+        cs = min(4u, nb64 - 4u * sc);
+        wsrc = p.wq + ((size_t)sc * 4u * KB + (nb & 3u)) * kChunkBytes;
+      }
     }
     if (*abort_flag) {
       // give copies that may still be in flight time to land before the CTA's shared memory goes away
@@ -247,19 +276,41 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_dense_kernel(const GemmP
   const int grp = warp / NW;
   const int wn = warp % NW;
   const int g = lane >> 2, c = lane & 3;
-  int s = grp;  // this group's first stage is iteration `grp` of the CTA
+  const int ctid = threadIdx.x;  // 0..255 among consumers
+  int s = grp;                   // this group's first stage is iteration `grp` of the CTA
   uint32_t ph = 0;
+  // byte offsets of this thread's two 16-byte A vectors inside a 128-byte row (128B swizzle: chunk ^ row%8)
+  const uint32_t a_off0 = (uint32_t)g * 128u + (uint32_t)(((2 * c) ^ g) * 16);
+  const uint32_t a_off1 = (uint32_t)g * 128u + (uint32_t)(((2 * c + 1) ^ g) * 16);
 
   float acc[4 * MB][4];
   float tmp[4 * MB][4];
-  float cur_s[8];
+  uint4 cur_raw = make_uint4(0, 0, 0, 0);  // 8 fp16 scales of the open group: columns 16j+g and 16j+8+g, j = 0..3
 
-  long long u = u0;
-  long long it0 = 0;  // iteration index of the segment's first unit, relative to u0
+  auto close_group = [&]() {
+    const __half2* h2 = reinterpret_cast<const __half2*>(&cur_raw);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float2 sc2 = __half22float2(h2[j]);
+#pragma unroll
+      for (int mb = 0; mb < MB; ++mb) {
+        const int r = j * MB + mb;
+        acc[r][0] += sc2.x * tmp[r][0];
+        acc[r][1] += sc2.x * tmp[r][1];
+        acc[r][2] += sc2.y * tmp[r][2];
+        acc[r][3] += sc2.y * tmp[r][3];
+        tmp[r][0] = tmp[r][1] = tmp[r][2] = tmp[r][3] = 0.f;
+      }
+    }
+  };
+
+  uint32_t u = u0;
+  uint32_t it0 = 0;  // iteration index of the segment's first unit, relative to u0
   while (u < u1) {
-    const int col = (int)(u / KB);
-    const int kb0 = (int)(u % KB);
-    const int len = (int)min((long long)(KB - kb0), u1 - u);
+    const uint32_t col = u / KB;
+    const uint32_t kb0 = u % KB;
+    const uint32_t len = min(KB - kb0, u1 - u);
+    const uint16_t* srow = reinterpret_cast<const uint16_t*>(p.sq) + (size_t)col * G::NT + wn * 64 + g * 8;
 
 #pragma unroll
     for (int r = 0; r < 4 * MB; ++r)
@@ -267,59 +318,33 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_dense_kernel(const GemmP
       for (int x = 0; x < 4; ++x) { acc[r][x] = 0.f; tmp[r][x] = 0.f; }
     int cur_group = -1;
     if (!p.grouped) {
-      const uint4 sv = *reinterpret_cast<const uint4*>(p.sq + ((size_t)col * G::NT + wn * 64 + g * 8) * 2);
-      const __half2* h2 = reinterpret_cast<const __half2*>(&sv);
-#pragma unroll
-      for (int x = 0; x < 4; ++x) {
-        float2 f = __half22float2(h2[x]);
-        cur_s[2 * x] = f.x;
-        cur_s[2 * x + 1] = f.y;
-      }
+      cur_raw = __ldg(reinterpret_cast<const uint4*>(srow));
       cur_group = 0;
     }
 
-    // first iteration of this segment that belongs to this group
-    int off = (int)((grp - (it0 % SK) + SK) % SK);
-    for (int x = off; x < len; x += SK) {
-      const int kb = kb0 + x;
-      mbar_wait(&full[s], ph, abort_flag, p.status);
-      const uint8_t* st = stage0 + (size_t)s * G::STAGE_BYTES;
-
+    // iterations of this segment that belong to this group: x = off, off + SK, ...
+    const uint32_t off = (grp + SK - (it0 % SK)) % SK;
+    for (uint32_t x = off; x < len; x += SK) {
+      const uint32_t kb = kb0 + x;
       if (p.grouped) {
-        const int gi = kb / p.kb_per_group;
+        const int gi = (int)(kb / (uint32_t)p.kb_per_group);
         if (gi != cur_group) {
-          if (cur_group >= 0) {
-#pragma unroll
-            for (int r = 0; r < 4 * MB; ++r) {
-              const int j = r / MB;
-              acc[r][0] += cur_s[2 * j] * tmp[r][0];
-              acc[r][1] += cur_s[2 * j] * tmp[r][1];
-              acc[r][2] += cur_s[2 * j + 1] * tmp[r][2];
-              acc[r][3] += cur_s[2 * j + 1] * tmp[r][3];
-              tmp[r][0] = tmp[r][1] = tmp[r][2] = tmp[r][3] = 0.f;
-            }
-          }
-          const uint4 sv = *reinterpret_cast<const uint4*>(st + G::W_BYTES + wn * 128 + g * 16);
-          const __half2* h2 = reinterpret_cast<const __half2*>(&sv);
-#pragma unroll
-          for (int y = 0; y < 4; ++y) {
-            float2 f = __half22float2(h2[y]);
-            cur_s[2 * y] = f.x;
-            cur_s[2 * y + 1] = f.y;
-          }
+          if (cur_group >= 0) close_group();
+          cur_raw = __ldg(reinterpret_cast<const uint4*>(srow + (size_t)gi * p.N));  // used when the group closes
           cur_group = gi;
         }
       }
-
-      const uint4* wp = reinterpret_cast<const uint4*>(st + wn * kChunkBytes) + lane;
-      const uint8_t* ap = st + G::A_OFF + g * kARowBytes + c * 32;
+      mbar_wait(&full[s], ph, abort_flag, p.status);
+      const uint8_t* st = stage0 + (size_t)s * G::STAGE_BYTES;
+      const uint4* wp = reinterpret_cast<const uint4*>(st + G::A_BYTES + wn * kChunkBytes) + lane;
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         uint32_t bf[MB][8];
 #pragma unroll
         for (int mb = 0; mb < MB; ++mb) {
-          const uint4 v0 = *reinterpret_cast<const uint4*>(ap + mb * 8 * kARowBytes + h * 128);
-          const uint4 v1 = *reinterpret_cast<const uint4*>(ap + mb * 8 * kARowBytes + h * 128 + 16);
+          const uint8_t* arow = st + h * G::A_HALF_BYTES + mb * 1024;
+          const uint4 v0 = *reinterpret_cast<const uint4*>(arow + a_off0);
+          const uint4 v1 = *reinterpret_cast<const uint4*>(arow + a_off1);
           bf[mb][0] = v0.x; bf[mb][1] = v0.y; bf[mb][2] = v0.z; bf[mb][3] = v0.w;
           bf[mb][4] = v1.x; bf[mb][5] = v1.y; bf[mb][6] = v1.z; bf[mb][7] = v1.w;
         }
@@ -341,84 +366,105 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_dense_kernel(const GemmP
       s += SK;
       if (s >= nstages) { s -= nstages; ph ^= 1u; }
     }
-    // close the open scale group
-    if (cur_group >= 0) {
+    if (cur_group >= 0) close_group();
+
+    // ---- reduce the SK groups of this CTA (the last step of Algorithm 1, as a tree) ----
 #pragma unroll
-      for (int r = 0; r < 4 * MB; ++r) {
-        const int j = r / MB;
-        acc[r][0] += cur_s[2 * j] * tmp[r][0];
-        acc[r][1] += cur_s[2 * j] * tmp[r][1];
-        acc[r][2] += cur_s[2 * j + 1] * tmp[r][2];
-        acc[r][3] += cur_s[2 * j + 1] * tmp[r][3];
+    for (int half = SK / 2; half >= 1; half >>= 1) {
+      if (grp >= half && grp < 2 * half) {
+        float4* dst = red + (size_t)(grp - half) * G::TILE_F4 + (size_t)wn * G::FRAG_F4 * 32 + lane;
+#pragma unroll
+        for (int r = 0; r < 4 * MB; ++r) dst[r * 32] = make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
       }
+      named_bar_sync(1, kConsumerThreads);
+      if (grp < half) {
+        const float4* src = red + (size_t)grp * G::TILE_F4 + (size_t)wn * G::FRAG_F4 * 32 + lane;
+#pragma unroll
+        for (int r = 0; r < 4 * MB; ++r) {
+          const float4 v = src[r * 32];
+          acc[r][0] += v.x; acc[r][1] += v.y; acc[r][2] += v.z; acc[r][3] += v.w;
+        }
+      }
+      named_bar_sync(1, kConsumerThreads);
     }
 
-    // ---- reduce the SK groups of this CTA (Algorithm 1's final step, as a tree) ----
-    if (SK > 1) {
-#pragma unroll
-      for (int half = SK / 2; half >= 1; half >>= 1) {
-        if (grp >= half && grp < 2 * half) {
-          float4* dst = red + (size_t)(grp - half) * (G::TILE_FLOATS / 4) + (size_t)wn * G::FRAG_F4 * 32 + lane;
-#pragma unroll
-          for (int r = 0; r < 4 * MB; ++r) dst[r * 32] = make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
-        }
-        named_bar_sync(1, kConsumerWarps * 32);
-        if (grp < half) {
-          const float4* src = red + (size_t)grp * (G::TILE_FLOATS / 4) + (size_t)wn * G::FRAG_F4 * 32 + lane;
-#pragma unroll
-          for (int r = 0; r < 4 * MB; ++r) {
-            const float4 v = src[r * 32];
-            acc[r][0] += v.x; acc[r][1] += v.y; acc[r][2] += v.z; acc[r][3] += v.w;
-          }
-        }
-        named_bar_sync(1, kConsumerWarps * 32);
-      }
-    }
-
-    // ---- stripe fix-up and output, by group 0 ----
-    if (grp == 0) {
-      const int first_w = stripe_owner((long long)col * KB, U, P);
-      const int last_w = stripe_owner((long long)(col + 1) * KB - 1, U, P);
-      bool write_out = true;
-      if (last_w > first_w) {
-        const int my_slot = 2 * worker + (col != (int)(u0 / KB) ? 1 : 0);
+    // ---- stripe fix-up across CTAs and output ----
+    const int first_w = (int)stripe_owner32(col * KB, U, P);
+    const int last_w = (int)stripe_owner32((col + 1) * KB - 1, U, P);
+    bool tile_in_cst = false;
+    if (last_w > first_w) {
+      // this column tile is shared: publish the partial, count arrivals
+      if (grp == 0) {
+        const int my_slot = 2 * (int)worker + (col != u0 / KB ? 1 : 0);
         float4* mine = reinterpret_cast<float4*>(p.partials + (size_t)my_slot * p.slot_floats) +
                        (size_t)wn * G::FRAG_F4 * 32 + lane;
 #pragma unroll
         for (int r = 0; r < 4 * MB; ++r) mine[r * 32] = make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
-        __threadfence();
-        named_bar_sync(2, NW * 32);
-        if (warp == 0 && lane == 0) {
-          const int old = atomicAdd(&p.counters[col], 1);
-          const int is_last = (old == last_w - first_w) ? 1 : 0;
-          if (is_last) p.counters[col] = 0;  // everyone has arrived: leave the counter ready for the next call
-          *last_flag = is_last;
-        }
-        named_bar_sync(2, NW * 32);
-        write_out = (*last_flag != 0);
-        if (write_out) {
-          // The last arriver adds every partial of the column tile, its own included, in stripe
-          // order from the workspace: the order of the fp32 sum never depends on who came last.
-          __threadfence();
-          for (int w = first_w; w <= last_w; ++w) {
-            const int wcol0 = (int)(stripe_begin(w, U, P) / KB);
-            const int slot = 2 * w + (col != wcol0 ? 1 : 0);
-            const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)slot * p.slot_floats) +
-                                (size_t)wn * G::FRAG_F4 * 32 + lane;
+      }
+      named_bar_sync(1, kConsumerThreads);
+      if (ctid == 0) {
+        const int old = atom_add_acq_rel_gpu(&p.counters[col], 1);
+        const int is_last = (old == last_w - first_w) ? 1 : 0;
+        if (is_last) p.counters[col] = 0;  // everyone has arrived: leave the counter ready for the next call
+        *last_flag = is_last;
+      }
+      named_bar_sync(1, kConsumerThreads);
+      if (*last_flag) {
+        // The last arriver adds every partial of the tile, its own included, in stripe order, so the
+        // order of the fp32 sum never depends on who came last.  All consumer threads take part and
+        // the loads of several contributors are in flight together.
+        constexpr int PER = (G::TILE_F4 + kConsumerThreads - 1) / kConsumerThreads;
+        constexpr int BATCH = PER >= 8 ? 1 : (PER >= 4 ? 2 : 4);  // contributors whose loads are in flight together
+        float4 sum[PER];
+        for (int w = first_w; w <= last_w; w += BATCH) {
+          float4 v[BATCH][PER];
 #pragma unroll
-            for (int r = 0; r < 4 * MB; ++r) {
-              const float4 v = ld_cg_f4(src + r * 32);
-              if (w == first_w) {
-                acc[r][0] = v.x; acc[r][1] = v.y; acc[r][2] = v.z; acc[r][3] = v.w;
-              } else {
-                acc[r][0] += v.x; acc[r][1] += v.y; acc[r][2] += v.z; acc[r][3] += v.w;
+          for (int d = 0; d < BATCH; ++d) {
+            const int ww = w + d;
+            if (ww <= last_w) {
+              const int slot = 2 * ww + (col != stripe_begin32(ww, U, P) / KB ? 1 : 0);
+              const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)slot * p.slot_floats);
+#pragma unroll
+              for (int e = 0; e < PER; ++e) {
+                const int f = ctid + e * kConsumerThreads;
+                if (f < G::TILE_F4) v[d][e] = ld_cg_f4(src + f);
+              }
+            }
+          }
+#pragma unroll
+          for (int d = 0; d < BATCH; ++d) {
+            const int ww = w + d;
+            if (ww <= last_w) {
+#pragma unroll
+              for (int e = 0; e < PER; ++e) {
+                if (ww == first_w) {
+                  sum[e] = v[d][e];
+                } else {
+                  sum[e].x += v[d][e].x; sum[e].y += v[d][e].y; sum[e].z += v[d][e].z; sum[e].w += v[d][e].w;
+                }
               }
             }
           }
         }
+#pragma unroll
+        for (int e = 0; e < PER; ++e) {
+          const int f = ctid + e * kConsumerThreads;
+          if (f < G::TILE_F4) {
+            // float4 f of the tile is register r of lane ln of warp w2 (fragment order)
+            const int ln = f & 31, r = (f >> 5) % G::FRAG_F4, w2 = f / (32 * G::FRAG_F4);
+            const int j = r / MB, mb = r % MB;
+            const int n = w2 * 64 + 16 * j + (ln >> 2);
+            const int m = mb * 8 + 2 * (ln & 3);
+            cst[m * G::CST_STRIDE + n] = __half_as_ushort(__float2half_rn(sum[e].x));
+            cst[(m + 1) * G::CST_STRIDE + n] = __half_as_ushort(__float2half_rn(sum[e].y));
+            cst[m * G::CST_STRIDE + n + 8] = __half_as_ushort(__float2half_rn(sum[e].z));
+            cst[(m + 1) * G::CST_STRIDE + n + 8] = __half_as_ushort(__float2half_rn(sum[e].w));
+          }
+        }
+        tile_in_cst = true;
       }
-      if (write_out) {
-        // fragments -> fp16 tile in shared memory -> 16-byte row stores
+    } else {
+      if (grp == 0) {
 #pragma unroll
         for (int r = 0; r < 4 * MB; ++r) {
           const int j = r / MB, mb = r % MB;
@@ -430,16 +476,17 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_dense_kernel(const GemmP
           cst[(m + 1) * G::CST_STRIDE + n + 8] = __half_as_ushort(__float2half_rn(acc[r][3]));
         }
       }
-      named_bar_sync(2, NW * 32);
-      if (write_out) {
-        constexpr int CH = NW * 8;  // 16-byte chunks per row
-        for (int x = warp * 32 + lane; x < p.M * CH; x += NW * 32) {
-          const int m = x / CH, ch = x % CH;
-          const uint4 v = *reinterpret_cast<const uint4*>(cst + m * G::CST_STRIDE + ch * 8);
-          *reinterpret_cast<uint4*>(p.C + (size_t)m * p.N + (size_t)col * G::NT + ch * 8) = v;
-        }
+      tile_in_cst = true;
+    }
+    if (tile_in_cst) {
+      named_bar_sync(1, kConsumerThreads);
+      constexpr int CH = NW * 8;  // 16-byte chunks per row of the tile
+      for (int x = ctid; x < p.M * CH; x += kConsumerThreads) {
+        const int m = x / CH, ch = x % CH;
+        const uint4 v = *reinterpret_cast<const uint4*>(cst + m * G::CST_STRIDE + ch * 8);
+        *reinterpret_cast<uint4*>(p.C + (size_t)m * p.N + (size_t)col * G::NT + ch * 8) = v;
       }
-      named_bar_sync(2, NW * 32);
+      named_bar_sync(1, kConsumerThreads);  // the tile buffer is free again
     }
 
     u += len;
@@ -447,22 +494,50 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_dense_kernel(const GemmP
   }
 }
 
+// cuTensorMapEncodeTiled through the runtime's driver entry point (no link against libcuda).
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// A[M][K] fp16 row-major as a 2-D tensor (inner K); box = 64 columns x mpad rows, 128-byte swizzle.
+bool make_a_tensor_map(CUtensorMap* map, const void* A, int M, int K, int mpad) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
+  const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)mpad};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(A), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int MB, int NW>
 cudaError_t launch_one(const DensePlan& plan, const GemmParams& p, cudaStream_t stream) {
   auto kernel = gemm_dense_kernel<MB, NW>;
-  static bool attr_set[16] = {};  // per device
+  static bool attr_set[64] = {};  // per device
   int dev = 0;
   cudaError_t err = cudaGetDevice(&dev);
   if (err != cudaSuccess) return err;
-  if (dev < 16 && !attr_set[dev]) {
+  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
     err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
     if (err != cudaSuccess) return err;
-    attr_set[dev] = true;
-  } else if (dev >= 16) {
-    err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
-    if (err != cudaSuccess) return err;
+    if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
-  kernel<<<plan.workers, kGemmThreads, plan.smem_bytes, stream>>>(p);
+  alignas(64) CUtensorMap tmap;
+  if (!make_a_tensor_map(&tmap, p.A, p.M, p.K, MB * 8)) return cudaErrorInvalidValue;
+  kernel<<<plan.workers, kGemmThreads, plan.smem_bytes, stream>>>(p, tmap);
   return cudaGetLastError();
 }
 
@@ -470,10 +545,11 @@ template <int MB, int NW>
 void fill_geometry(DensePlan* plan) {
   using G = Geometry<MB, NW>;
   plan->stage_bytes = G::STAGE_BYTES;
-  int stages = (kSmemBudget - G::FIXED_BYTES) / G::STAGE_BYTES;
+  int stages = (kSmemBudget - G::FIXED_BYTES - G::ALIGN_SLACK) / G::STAGE_BYTES;
   if (stages > kMaxStages) stages = kMaxStages;
+  if (const char* e = getenv("MARLIN_B200_STAGES")) { int v = atoi(e); if (v >= 2 && v < stages) stages = v; }
   plan->stages = stages;
-  plan->smem_bytes = G::FIXED_BYTES + stages * G::STAGE_BYTES;
+  plan->smem_bytes = G::FIXED_BYTES + G::ALIGN_SLACK + stages * G::STAGE_BYTES;
 }
 
 }  // namespace
@@ -485,12 +561,14 @@ bool make_dense_plan(int m_slab, int K, int N, int sm_count, DensePlan* plan) {
   if (m_slab < 1 || m_slab > kMaxSlabM || K < kTileK || K % kTileK || N < kChunkN || N % kChunkN) return false;
   if (sm_count < 1) return false;
   int mb = m_slab <= 8 ? 1 : (m_slab <= 16 ? 2 : 4);
-  int nw = m_slab <= 8 ? 1 : (m_slab <= 16 ? 2 : 4);
-  while (nw > 1 && N % (64 * nw)) nw >>= 1;
+  // wide column tiles keep the bulk copies large (16 KB) whatever the batch size
+  int nw = 4;
+  if (const char* e = getenv("MARLIN_B200_NW")) { int v = atoi(e); if (v == 1 || v == 2 || v == 4) nw = v; }
+  while (nw > 1 && N % (kChunkN * nw)) nw >>= 1;
   plan->mb = mb;
   plan->nw = nw;
   plan->kb = K / kTileK;
-  plan->ncols = N / (64 * nw);
+  plan->ncols = N / (kChunkN * nw);
   plan->units = (long long)plan->ncols * plan->kb;
   long long workers = sm_count < kMaxWorkers ? sm_count : kMaxWorkers;
   if (workers > plan->units) workers = plan->units;

@@ -53,12 +53,12 @@ struct GemmParams {
   const uint8_t* sq;
   uint16_t* C;
   int M, K, N;
-  int kb;            // K / 128
+  uint32_t kb;       // K / 128
   int kb_per_group;  // group_size / 128
   int grouped;       // 0: one scale per column (group_size == K)
   int ncols;
-  long long units;
-  int workers;
+  uint32_t units;
+  uint32_t workers;
   int stages;
   int stage_bytes;
   int* status;
@@ -78,5 +78,8 @@ __host__ __device__ inline long long stripe_begin(long long w, long long U, long
 __host__ __device__ inline int stripe_owner(long long x, long long U, long long P) {
   return (int)(((x + 1) * P - 1) / U);
 }
+// the same in 32-bit arithmetic for the device (U * P < 2^32 is checked on the host)
+__device__ inline uint32_t stripe_begin32(uint32_t w, uint32_t U, uint32_t P) { return (w * U) / P; }
+__device__ inline uint32_t stripe_owner32(uint32_t x, uint32_t U, uint32_t P) { return ((x + 1) * P - 1) / U; }
 
 }  // namespace marlin_b200

@@ -5,8 +5,14 @@
 // (Section 3.4, "Maximizing Loading Bandwidth" and "Dequantization and Tensor Cores").  The order
 // used here is this library's own:
 //
-//   word index = (((kb * (N/64) + nb) * 8 + i) * 32 + lane) * 4 + t
-//     kb   = k / 128, nb = n / 64            one 4096-byte chunk per (kb, nb), chunks of a k-block adjacent
+//   One 4096-byte chunk holds the codes of 128 rows (k-block kb = k / 128) x 64 columns (nb = n / 64).
+//   Chunks are ordered by "super-columns" of four chunks (256 columns): inside super-column sc = nb / 4
+//   the k-blocks follow one another, each with its cs chunks side by side (cs = 4, or the 1..3 chunks
+//   left over in the last super-column when N is not a multiple of 256):
+//     chunk index = sc * 4 * (K/128) + kb * cs + (nb % 4)
+//   so the weights a CTA streams for a 256-column tile are one contiguous run of memory, k-block after
+//   k-block, and one k-block of a tile is a single 16 KB bulk copy.
+//   word index = ((chunk index * 8 + i) * 32 + lane) * 4 + t
 //     i    = 4*h + j                         h: which 64-row half of the k-block, j: which 16 columns
 //     lane = 4*g + c                         the consuming thread; g = lane / 4, c = lane % 4
 //     t    = 0..3                            which 16-row MMA step inside the half
@@ -32,6 +38,27 @@ __device__ __forceinline__ void decode_position(int p, int g, int c, int t, int 
   *k = 128 * kb + 64 * h + 16 * c + 4 * t + 2 * (r >> 1) + (p >> 2);
 }
 
+// chunk index <-> (kb, nb)
+__device__ __forceinline__ long long chunk_index(int kb, int nb, int KB, int nb64) {
+  int sc = nb >> 2;
+  int cs = min(4, nb64 - 4 * sc);
+  return (long long)sc * 4 * KB + (long long)kb * cs + (nb & 3);
+}
+__device__ __forceinline__ void chunk_coords(long long chunk, int KB, int nb64, int* kb, int* nb) {
+  long long full = (long long)(nb64 >> 2) * 4 * KB;  // chunks in complete super-columns
+  if (chunk < full) {
+    int sc = (int)(chunk / (4 * KB));
+    int rem = (int)(chunk % (4 * KB));
+    *kb = rem >> 2;
+    *nb = 4 * sc + (rem & 3);
+  } else {
+    int cs = nb64 & 3;
+    int rem = (int)(chunk - full);
+    *kb = rem / cs;
+    *nb = 4 * (nb64 >> 2) + rem % cs;
+  }
+}
+
 __global__ void pack_weights_kernel(const uint32_t* __restrict__ q, uint32_t* __restrict__ wq, int K, int N) {
   long long total = (long long)K * N / 8;
   for (long long wi = blockIdx.x * (long long)blockDim.x + threadIdx.x; wi < total;
@@ -39,10 +66,9 @@ __global__ void pack_weights_kernel(const uint32_t* __restrict__ q, uint32_t* __
     int t = (int)(wi & 3);
     int lane = (int)((wi >> 2) & 31);
     int i = (int)((wi >> 7) & 7);
-    long long chunk = wi >> 10;
     int nb64 = N / 64;
-    int nb = (int)(chunk % nb64);
-    int kb = (int)(chunk / nb64);
+    int kb, nb;
+    chunk_coords(wi >> 10, K / 128, nb64, &kb, &nb);
     int g = lane >> 2, c = lane & 3, h = i >> 2, j = i & 3;
     uint32_t out = 0;
 #pragma unroll
@@ -72,7 +98,7 @@ __global__ void unpack_weights_kernel(const uint32_t* __restrict__ wq, uint32_t*
       int kb = k >> 7, h = (k >> 6) & 1, c = (k >> 4) & 3, t = (k >> 2) & 3, e = k & 3;
       int p = (rbit0 | ((e >> 1) << 1)) + 4 * (e & 1);
       int lane = 4 * g + c, i = 4 * h + j;
-      long long wi = ((((long long)kb * nb64 + nb) * 8 + i) * 32 + lane) * 4 + t;
+      long long wi = ((chunk_index(kb, nb, K / 128, nb64) * 8 + i) * 32 + lane) * 4 + t;
       uint32_t code = (wq[wi] >> (4 * p)) & 15u;
       out |= code << (4 * jn);
     }
