@@ -39,14 +39,16 @@ def needs_build() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not needs_build():
+def build(force: bool = False, verbose: bool = False, extra_flags=(), out: str = LIB) -> str:
+    """Compiles every .cu of the library and links `out`.  `extra_flags` (for example -DMARLIN_TIMING)
+    and a different `out` give an instrumented variant beside the product library."""
+    if not force and out == LIB and not needs_build():
         return LIB
     objs = []
     procs = []
     for src in SOURCES:
-        obj = os.path.join(CSRC, src.replace(".cu", ".o"))
-        cmd = [_nvcc(), *NVCC_FLAGS, "-I", os.path.join(_ROOT, "include"), "-I", CSRC, "-c",
+        obj = os.path.join(CSRC, src.replace(".cu", ".o" if out == LIB else ".variant.o"))
+        cmd = [_nvcc(), *NVCC_FLAGS, *extra_flags, "-I", os.path.join(_ROOT, "include"), "-I", CSRC, "-c",
                os.path.join(CSRC, src), "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas")
@@ -56,16 +58,16 @@ def build(force: bool = False, verbose: bool = False) -> str:
         objs.append(obj)
     failed = False
     for src, proc in procs:
-        out, _ = proc.communicate()
+        log, _ = proc.communicate()
         if proc.returncode != 0 or verbose:
-            sys.stderr.write(out)
+            sys.stderr.write(log)
         failed |= proc.returncode != 0
     if failed:
         raise RuntimeError("nvcc failed")
-    link = [_nvcc(), "-shared", "-o", LIB, *objs, "-cudart", "static",
+    link = [_nvcc(), "-shared", "-o", out, *objs, "-cudart", "static",
             "-gencode", "arch=compute_100a,code=sm_100a"]
     subprocess.run(link, check=True)
-    return LIB
+    return out
 
 
 if __name__ == "__main__":

@@ -153,6 +153,9 @@ int marlin_gemm(const void* A, const void* w_packed, const void* s_packed, void*
     p.N = N;
     p.kb = (uint32_t)plan.kb;
     p.kb_per_group = G / kTileK;
+    p.group_shift = -1;
+    for (int sh = 0; sh < 31; ++sh)
+      if ((1 << sh) == p.kb_per_group) p.group_shift = sh;
     p.grouped = (G != K) ? 1 : 0;
     p.ncols = plan.ncols;
     p.units = (uint32_t)plan.units;

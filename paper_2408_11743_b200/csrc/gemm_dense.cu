@@ -168,16 +168,39 @@ __device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4],
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+// Register re-allocation between warpgroups (all four warps of a warpgroup execute it together).
+template <int N>
+__device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N>
+__device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+
+// Programmatic dependent launch: let the next kernel of the stream start its prologue while this
+// one drains, and wait for the previous kernel's memory before touching anything it may have written.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait_prior_grids() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ float4 ld_cg_f4(const float4* p) { return __ldcg(p); }
+
+// Optional per-CTA cycle stamps for tuning (built only with -DMARLIN_TIMING; not part of the library).
+#ifdef MARLIN_TIMING
+__device__ long long g_timing[kMaxWorkers][16];
+#define MARLIN_STAMP(slot) do { if (lane == 0) g_timing[blockIdx.x][slot] = (long long)global_timer_ns(); } while (0)
+#else
+#define MARLIN_STAMP(slot) do { } while (0)
+#endif
 
 // ---------------------------------------------------------------------------------------------
 // shared memory map
 // ---------------------------------------------------------------------------------------------
 constexpr int kBarBytes = 1024;  // full[32] at 0, empty[32] at 256, flags at 512
 
-template <int MB, int NW>
+// Consumer warps per CTA.  Eight everywhere: a sixteen-warp variant of the one-block kernel (batch <= 8)
+// raised "unspecified launch failure" on long-K layers, was no faster, and is not built.
+constexpr int consumer_warps_for(int /*mb*/) { return 8; }
+
+template <int MB, int NW, int CW>
 struct Geometry {
-  static constexpr int SK = kConsumerWarps / NW;             // groups of warps that split K
+  static constexpr int SK = CW / NW;             // groups of warps that split K
   static constexpr int MPAD = MB * 8;
   static constexpr int NT = NW * kChunkN;
   static constexpr int A_HALF_BYTES = MPAD * 128;            // one 64-wide half of the A tile: MPAD rows x 128 B
@@ -196,12 +219,16 @@ struct Geometry {
 // ---------------------------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------------------------
-template <int MB, int NW>
-__global__ void __launch_bounds__(kGemmThreads, 1)
+template <int MB, int NW, int CW>
+__global__ void __launch_bounds__((CW + 4) * 32, 1)
 gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a) {
-  using G = Geometry<MB, NW>;
+  using G = Geometry<MB, NW, CW>;
   constexpr int SK = G::SK;
-  constexpr int kConsumerThreads = kConsumerWarps * 32;
+  constexpr int kConsumerWarps = CW;
+  constexpr int kConsumerThreads = CW * 32;
+  // register budget: (CW + 4) * 32 threads share 64K registers; the producer warpgroup keeps 40
+  constexpr int kBaseRegs = (65536 / ((CW + 4) * 32)) / 8 * 8;
+  constexpr int kConsumerRegs = (kBaseRegs + (kBaseRegs - kProducerRegs) * 4 / CW) / 8 * 8;
   extern __shared__ __align__(128) uint8_t smem_raw[];
   // 128-byte-swizzled TMA tiles need their shared address aligned to the 1024-byte swizzle period
   uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -220,6 +247,8 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
   const uint32_t u0 = stripe_begin32(worker, U, P), u1 = stripe_begin32(worker + 1, U, P);
   const int nstages = p.stages;
 
+  pdl_launch_dependents();
+  if (warp == 0) MARLIN_STAMP(10);
   if ((int)threadIdx.x < nstages) {
     mbar_init(&full[threadIdx.x], 1);
     mbar_init(&empty[threadIdx.x], NW);
@@ -230,22 +259,55 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
   }
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   __syncthreads();
+  if (warp == 0) MARLIN_STAMP(0);
 
-  if (warp == kConsumerWarps) {
-    // ------------------------------- producer ---------------------------------------------
+  if (warp >= kConsumerWarps) {
+    // ------------------------------- producers --------------------------------------------
+    // The third warpgroup gives most of its registers to the two consumer warpgroups.  Its warps
+    // take the stages round-robin: issuing a bulk or tensor copy occupies a warp for a few hundred
+    // cycles whatever the size of the copy, so several warps issue in parallel.
+    const int pw = warp - kConsumerWarps;
     if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
     const uint64_t pol_w = policy_evict_first();
     const uint64_t pol_a = policy_evict_last();
     constexpr uint32_t tx_bytes = G::W_BYTES + G::A_BYTES;  // out-of-range rows of the box count too
     const uint32_t nb64 = p.N / kChunkN;
-    int s = 0;
-    uint32_t ph = 0;
-    uint32_t col = u0 / KB, kb = u0 % KB;
     // weights of (kb, col): super-columns of four chunks, k-blocks contiguous inside a super-column
-    uint32_t nb = col * NW;
-    uint32_t sc = nb >> 2, cs = min(4u, nb64 - 4u * sc);
-    const uint8_t* wsrc = p.wq + ((size_t)sc * 4u * KB + (size_t)kb * cs + (nb & 3u)) * kChunkBytes;
-    for (uint32_t u = u0; u < u1; ++u) {
+    auto weight_src = [&](uint32_t col, uint32_t kb) -> const uint8_t* {
+      const uint32_t nb = col * NW;
+      const uint32_t sc = nb >> 2, cs = min(4u, nb64 - 4u * sc);
+      return p.wq + ((size_t)sc * 4u * KB + (size_t)kb * cs + (nb & 3u)) * kChunkBytes;
+    };
+    // First pass over the ring: the packed weights do not depend on the previous kernel of the
+    // stream, so their copies go out before the dependency wait and HBM keeps streaming across the
+    // kernel boundary; the A tiles follow once the previous kernel's memory is visible.
+    uint32_t u = u0 + pw;
+    int s = pw;
+    if (lane == 0) {
+      for (; u < u1 && s < nstages; u += kProducerWarps, s += kProducerWarps) {
+        const uint32_t col = u / KB, kb = u - col * KB;
+        mbar_expect_tx(&full[s], tx_bytes);
+        bulk_g2s(stage0 + (size_t)s * G::STAGE_BYTES + G::A_BYTES, weight_src(col, kb), G::W_BYTES, &full[s], pol_w);
+      }
+    }
+    __syncwarp();
+    MARLIN_STAMP(1 + (pw & 1));
+    setmaxnreg_dec<kProducerRegs>();
+    pdl_wait_prior_grids();
+    u = u0 + pw;
+    s = pw;
+    for (; u < u1 && s < nstages; u += kProducerWarps, s += kProducerWarps) {
+      const uint32_t col = u / KB, kb = u - col * KB;
+      if (lane < 2)
+        tma_load_2d(stage0 + (size_t)s * G::STAGE_BYTES + lane * G::A_HALF_BYTES, &tmap_a,
+                    (int)(kb * kTileK + lane * 64), 0, &full[s], pol_a);
+    }
+    // steady state: a stage is refilled as soon as its consumers have released it
+    uint32_t ph = 1;
+    s -= nstages;
+    for (; u < u1; u += kProducerWarps) {
+      const uint32_t col = u / KB, kb = u - col * KB;
+      const uint8_t* wsrc = weight_src(col, kb);
       mbar_wait(&empty[s], ph ^ 1u, abort_flag, p.status);
       uint8_t* st = stage0 + (size_t)s * G::STAGE_BYTES;
       if (lane == 0) {
@@ -254,17 +316,10 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
       }
       __syncwarp();
       if (lane < 2) tma_load_2d(st + lane * G::A_HALF_BYTES, &tmap_a, (int)(kb * kTileK + lane * 64), 0, &full[s], pol_a);
-      if (++s == nstages) { s = 0; ph ^= 1u; }
-      wsrc += (size_t)cs * kChunkBytes;
-      if (++kb == KB) {
-        kb = 0;
-        ++col;
-        nb = col * NW;
-        sc = nb >> 2;
-        cs = min(4u, nb64 - 4u * sc);
-        wsrc = p.wq + ((size_t)sc * 4u * KB + (nb & 3u)) * kChunkBytes;
-      }
+      s += kProducerWarps;
+      if (s >= nstages) { s -= nstages; ph ^= 1u; }
     }
+    if (pw == 0) MARLIN_STAMP(3);
     if (*abort_flag) {
       // give copies that may still be in flight time to land before the CTA's shared memory goes away
       for (int x = 0; x < 1000; ++x) __nanosleep(1000);
@@ -273,6 +328,11 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
   }
 
   // --------------------------------- consumers ----------------------------------------------
+  setmaxnreg_inc<kConsumerRegs>();
+  // From here on this kernel writes C and the workspace, which the previous kernel of the stream
+  // may still be using: wait until it has finished and its memory is visible.
+  pdl_wait_prior_grids();
+  if (warp == 0) MARLIN_STAMP(11);
   const int grp = warp / NW;
   const int wn = warp % NW;
   const int g = lane >> 2, c = lane & 3;
@@ -327,7 +387,7 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
     for (uint32_t x = off; x < len; x += SK) {
       const uint32_t kb = kb0 + x;
       if (p.grouped) {
-        const int gi = (int)(kb / (uint32_t)p.kb_per_group);
+        const int gi = p.group_shift >= 0 ? (int)(kb >> p.group_shift) : (int)(kb / (uint32_t)p.kb_per_group);
         if (gi != cur_group) {
           if (cur_group >= 0) close_group();
           cur_raw = __ldg(reinterpret_cast<const uint4*>(srow + (size_t)gi * p.N));  // used when the group closes
@@ -335,6 +395,7 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
         }
       }
       mbar_wait(&full[s], ph, abort_flag, p.status);
+      if (warp == 0 && x == off && it0 == 0) MARLIN_STAMP(4);
       const uint8_t* st = stage0 + (size_t)s * G::STAGE_BYTES;
       const uint4* wp = reinterpret_cast<const uint4*>(st + G::A_BYTES + wn * kChunkBytes) + lane;
 #pragma unroll
@@ -348,14 +409,20 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
           bf[mb][0] = v0.x; bf[mb][1] = v0.y; bf[mb][2] = v0.z; bf[mb][3] = v0.w;
           bf[mb][4] = v1.x; bf[mb][5] = v1.y; bf[mb][6] = v1.z; bf[mb][7] = v1.w;
         }
+        // all four 16-column blocks of this half first, then step by step over k: consecutive MMAs
+        // go to different accumulators, so none waits for the one before it
+        uint32_t ww[4][4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const uint4 wv = wp[(h * 4 + j) * 32];
-          const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
+          ww[j][0] = wv.x; ww[j][1] = wv.y; ww[j][2] = wv.z; ww[j][3] = wv.w;
+        }
 #pragma unroll
-          for (int t = 0; t < 4; ++t) {
+        for (int t = 0; t < 4; ++t) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
             uint32_t a[4];
-            dequant8(ww[t], a);
+            dequant8(ww[j][t], a);
 #pragma unroll
             for (int mb = 0; mb < MB; ++mb) mma_16816(tmp[j * MB + mb], a, bf[mb][2 * t], bf[mb][2 * t + 1]);
           }
@@ -367,6 +434,8 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
       if (s >= nstages) { s -= nstages; ph ^= 1u; }
     }
     if (cur_group >= 0) close_group();
+    if (warp == 0) MARLIN_STAMP(5);
+    if (warp == kConsumerWarps - 1) MARLIN_STAMP(6);
 
     // ---- reduce the SK groups of this CTA (the last step of Algorithm 1, as a tree) ----
 #pragma unroll
@@ -388,6 +457,7 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
       named_bar_sync(1, kConsumerThreads);
     }
 
+    if (warp == 0) MARLIN_STAMP(7);
     // ---- stripe fix-up across CTAs and output ----
     const int first_w = (int)stripe_owner32(col * KB, U, P);
     const int last_w = (int)stripe_owner32((col + 1) * KB - 1, U, P);
@@ -414,7 +484,7 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
         // order of the fp32 sum never depends on who came last.  All consumer threads take part and
         // the loads of several contributors are in flight together.
         constexpr int PER = (G::TILE_F4 + kConsumerThreads - 1) / kConsumerThreads;
-        constexpr int BATCH = PER >= 8 ? 1 : (PER >= 4 ? 2 : 4);  // contributors whose loads are in flight together
+        constexpr int BATCH = PER >= 8 ? 1 : (PER >= 4 ? 2 : (PER >= 2 ? 4 : 8));  // contributors whose loads are in flight together
         float4 sum[PER];
         for (int w = first_w; w <= last_w; w += BATCH) {
           float4 v[BATCH][PER];
@@ -491,7 +561,9 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
 
     u += len;
     it0 += len;
+    if (warp == 0) MARLIN_STAMP(8);
   }
+  if (warp == 0) MARLIN_STAMP(9);
 }
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point (no link against libcuda).
@@ -525,7 +597,8 @@ bool make_a_tensor_map(CUtensorMap* map, const void* A, int M, int K, int mpad) 
 
 template <int MB, int NW>
 cudaError_t launch_one(const DensePlan& plan, const GemmParams& p, cudaStream_t stream) {
-  auto kernel = gemm_dense_kernel<MB, NW>;
+  constexpr int CW = consumer_warps_for(MB);
+  auto kernel = gemm_dense_kernel<MB, NW, CW>;
   static bool attr_set[64] = {};  // per device
   int dev = 0;
   cudaError_t err = cudaGetDevice(&dev);
@@ -537,13 +610,22 @@ cudaError_t launch_one(const DensePlan& plan, const GemmParams& p, cudaStream_t 
   }
   alignas(64) CUtensorMap tmap;
   if (!make_a_tensor_map(&tmap, p.A, p.M, p.K, MB * 8)) return cudaErrorInvalidValue;
-  kernel<<<plan.workers, kGemmThreads, plan.smem_bytes, stream>>>(p, tmap);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(plan.workers);
+  cfg.blockDim = dim3((CW + 4) * 32);
+  cfg.dynamicSmemBytes = plan.smem_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, p, tmap);
 }
 
 template <int MB, int NW>
 void fill_geometry(DensePlan* plan) {
-  using G = Geometry<MB, NW>;
+  using G = Geometry<MB, NW, consumer_warps_for(MB)>;
   plan->stage_bytes = G::STAGE_BYTES;
   int stages = (kSmemBudget - G::FIXED_BYTES - G::ALIGN_SLACK) / G::STAGE_BYTES;
   if (stages > kMaxStages) stages = kMaxStages;
@@ -553,6 +635,12 @@ void fill_geometry(DensePlan* plan) {
 }
 
 }  // namespace
+
+#ifdef MARLIN_TIMING
+extern "C" __attribute__((visibility("default"))) int marlin_timing_read(void* host) {
+  return (int)cudaMemcpyFromSymbol(host, g_timing, sizeof(g_timing));
+}
+#endif
 
 #define MARLIN_DISPATCH(MBV, NWV, STMT)         \
   if (plan_mb == MBV && plan_nw == NWV) { STMT; }
@@ -583,7 +671,7 @@ bool make_dense_plan(int m_slab, int K, int N, int sm_count, DensePlan* plan) {
   MARLIN_DISPATCH(4, 1, (fill_geometry<4, 1>(plan)))
   MARLIN_DISPATCH(4, 2, (fill_geometry<4, 2>(plan)))
   MARLIN_DISPATCH(4, 4, (fill_geometry<4, 4>(plan)))
-  return plan->stages >= kConsumerWarps / nw && plan->stages >= 2;
+  return plan->stages >= consumer_warps_for(mb) / nw && plan->stages >= kProducerWarps;
 }
 
 cudaError_t launch_gemm_dense(const DensePlan& plan, const GemmParams& p, cudaStream_t stream) {

@@ -17,8 +17,10 @@ namespace marlin_b200 {
 constexpr int kTileK = 128;           // rows of W per k-block
 constexpr int kChunkN = 64;           // columns of W per chunk
 constexpr int kChunkBytes = 4096;     // dense chunk
-constexpr int kConsumerWarps = 8;
-constexpr int kGemmThreads = (kConsumerWarps + 1) * 32;  // + one producer warp
+constexpr int kProducerWarps = 4;     // the warps of the third warpgroup that issue copies
+// The last warpgroup of a CTA issues the copies; it shrinks to kProducerRegs registers per thread
+// (setmaxnreg) and the consumer warpgroups share what that frees.
+constexpr int kProducerRegs = 40;
 constexpr int kMaxStages = 32;
 constexpr int kMaxWorkers = 160;      // grid size cap (a B200 has 148 SMs)
 constexpr int kMaxSlabM = 32;         // rows of A handled by one launch of the mma.sync kernel
@@ -55,6 +57,7 @@ struct GemmParams {
   int M, K, N;
   uint32_t kb;       // K / 128
   int kb_per_group;  // group_size / 128
+  int group_shift;   // log2(kb_per_group) if it is a power of two, else -1
   int grouped;       // 0: one scale per column (group_size == K)
   int ncols;
   uint32_t units;
