@@ -103,6 +103,26 @@ MARLIN_API int marlin_gemm(const void* A, const void* w_packed, const void* s_pa
                 int M, int K, int N, int group_size,
                 void* workspace, size_t workspace_bytes, marlin_stream stream);
 
+/* The same layer for callers that cannot allocate device memory or carry a workspace pointer
+ * around: for example a plug-in that runs inside another framework's pre-captured execution plan,
+ * or a constrained runtime where cudaMalloc is forbidden after start-up.  (The paper has no
+ * counterpart; this is a convenience of this library.)
+ *
+ * Works like marlin_gemm, but the fix-up workspace is a fixed array inside the library's device
+ * image (about 5 MB, held by every GPU that loads the library until the process exits), so only
+ * M <= MARLIN_STATIC_WS_MAX_M is accepted; larger M returns MARLIN_ERR_SHAPE.  The call allocates
+ * nothing: no cudaMalloc, no cudaFree, no library routine that allocates.
+ *
+ * The first call on each device looks up the device address of that array (with that device
+ * current) and remembers it; make this first call outside any stream capture.  Every call clears
+ * the status word and the arrival counters of the array on `stream` before the kernels run, and
+ * all calls on one device share the one array: two such calls that can overlap on the GPU (two
+ * streams, or two host threads) race with each other and must be serialised by the caller.
+ * Errors: as marlin_gemm; MARLIN_ERR_CUDA if the address lookup or the clearing fails. */
+#define MARLIN_STATIC_WS_MAX_M 16
+MARLIN_API int marlin_gemm_static_ws(const void* A, const void* w_packed, const void* s_packed, void* C,
+                                     int M, int K, int N, int group_size, marlin_stream stream);
+
 /* ---- 2:4 structured-sparse variant (Section 4: values structure + metadata indices) ------------ */
 
 /* Pack the compressed form.

@@ -8,6 +8,7 @@ from .binding import (  # noqa: F401
     MarlinError,
     gemm,
     gemm_sparse24,
+    gemm_static_ws,
     lib,
     library_path,
     new_workspace,

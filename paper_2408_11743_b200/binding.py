@@ -17,7 +17,9 @@ EXPORTS = [
     "marlin_status_string", "marlin_packed_weight_bytes", "marlin_packed_scale_bytes", "marlin_packed_meta_bytes",
     "marlin_workspace_bytes", "marlin_pack", "marlin_unpack", "marlin_gemm", "marlin_pack_sparse24",
     "marlin_unpack_sparse24", "marlin_gemm_sparse24", "marlin_read_status", "marlin_plan_stripes",
+    "marlin_gemm_static_ws",
 ]
+STATIC_WS_MAX_M = 16  # MARLIN_STATIC_WS_MAX_M of the header
 
 
 class MarlinError(RuntimeError):
@@ -56,12 +58,13 @@ def lib():
     L.marlin_pack.argtypes = [vp, vp, vp, vp, i, i, i, vp]
     L.marlin_unpack.argtypes = [vp, vp, vp, vp, i, i, i, vp]
     L.marlin_gemm.argtypes = [vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
+    L.marlin_gemm_static_ws.argtypes = [vp, vp, vp, vp, i, i, i, i, vp]
     L.marlin_pack_sparse24.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, vp]
     L.marlin_unpack_sparse24.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, vp]
     L.marlin_gemm_sparse24.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
     L.marlin_read_status.argtypes = [vp, vp]
     L.marlin_plan_stripes.argtypes = [i, i, i, i, vp, vp, vp, i]
-    for name in ("marlin_pack", "marlin_unpack", "marlin_gemm", "marlin_pack_sparse24", "marlin_unpack_sparse24",
+    for name in ("marlin_gemm_static_ws", "marlin_pack", "marlin_unpack", "marlin_gemm", "marlin_pack_sparse24", "marlin_unpack_sparse24",
                  "marlin_gemm_sparse24", "marlin_read_status", "marlin_plan_stripes"):
         getattr(L, name).restype = i
     _lib = L
@@ -166,6 +169,34 @@ def gemm(A, w_packed, s_packed, K: int, N: int, group_size: int, workspace, out=
             raise ValueError("out must be [M, N]")
     _check(L.marlin_gemm(A.data_ptr(), w.data_ptr(), s.data_ptr(), out.data_ptr(), M, K, N, group_size,
                          ws.data_ptr(), ws.numel(), _stream_ptr(stream)), "marlin_gemm")
+    return out
+
+
+def gemm_static_ws(A, w_packed, s_packed, K: int, N: int, group_size: int, out=None, stream=None):
+    """marlin_gemm_static_ws: the layer for callers that cannot allocate or pass a workspace.
+
+    Same result as `gemm`, M <= STATIC_WS_MAX_M only.  The scratch memory is a fixed array inside the
+    library; calls on one device share it, so do not let two of them overlap on the GPU.  `out` should
+    be supplied by callers that must not allocate (without it this binding asks torch for the output).
+    """
+    torch = _torch()
+    A = _dev(A, torch.float16, "A")
+    if A.dim() != 2 or A.shape[1] != K:
+        raise ValueError("A must be [M, K]")
+    M = A.shape[0]
+    w = _dev(w_packed, torch.uint8, "w_packed")
+    s = _dev(s_packed, torch.uint8, "s_packed")
+    L = lib()
+    if w.numel() != L.marlin_packed_weight_bytes(K, N, 0) or s.numel() != L.marlin_packed_scale_bytes(K, N, group_size):
+        raise ValueError("packed buffer sizes do not match K, N, group_size")
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float16, device=A.device)
+    else:
+        _dev(out, torch.float16, "out")
+        if tuple(out.shape) != (M, N):
+            raise ValueError("out must be [M, N]")
+    _check(L.marlin_gemm_static_ws(A.data_ptr(), w.data_ptr(), s.data_ptr(), out.data_ptr(), M, K, N, group_size,
+                                   _stream_ptr(stream)), "marlin_gemm_static_ws")
     return out
 
 

@@ -171,6 +171,34 @@ int marlin_gemm(const void* A, const void* w_packed, const void* s_packed, void*
   return MARLIN_OK;
 }
 
+// ---- the variant with a built-in workspace ------------------------------------------------------
+// Scratch for marlin_gemm_static_ws: the workspace of one layer call with M <= MARLIN_STATIC_WS_MAX_M,
+// as a file-scope device array.  In host code the name `g_static_workspace` is only a handle for
+// cudaGetSymbolAddress; the kernels get the device address that call returns.
+constexpr size_t kStaticWsBytes =
+    kWsPartialOff + (size_t)2 * kMaxWorkers * kWsSlotCols * MARLIN_STATIC_WS_MAX_M * sizeof(float);
+static __device__ __align__(256) unsigned char g_static_workspace[kStaticWsBytes];
+
+int marlin_gemm_static_ws(const void* A, const void* w_packed, const void* s_packed, void* C, int M, int K, int N,
+                          int group_size, marlin_stream stream) {
+  if (M < 1 || M > MARLIN_STATIC_WS_MAX_M) return MARLIN_ERR_SHAPE;
+  if (marlin_workspace_bytes(M, K, N) == 0) return MARLIN_ERR_SHAPE;
+  if (marlin_workspace_bytes(M, K, N) > kStaticWsBytes) return MARLIN_ERR_WORKSPACE;
+  static void* device_address[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MARLIN_ERR_CUDA;
+  if (!device_address[dev]) {
+    // once per device, with that device current: where the array lives on this GPU
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_workspace) != cudaSuccess || !ptr) return MARLIN_ERR_CUDA;
+    device_address[dev] = ptr;
+  }
+  void* ws = device_address[dev];
+  // the array keeps whatever the last call left: start from a clean status word and clean counters
+  if (cudaMemsetAsync(ws, 0, kWsPartialOff, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MARLIN_ERR_CUDA;
+  return marlin_gemm(A, w_packed, s_packed, C, M, K, N, group_size, ws, kStaticWsBytes, stream);
+}
+
 int marlin_pack_sparse24(const uint32_t*, const uint8_t*, const void*, void*, void*, void*, int, int, int,
                          marlin_stream) {
   return MARLIN_ERR_SHAPE;  // filled in by gemm_sparse24.cu once that kernel exists
