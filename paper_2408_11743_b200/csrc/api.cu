@@ -50,8 +50,20 @@ int device_info(DeviceInfo* out) {
   return MARLIN_OK;
 }
 
+// rows of the widest launch a call with this M can make, padded the way that launch pads them
 int slab_mpad(int max_M) {
-  return max_M <= 8 ? 8 : (max_M <= 16 ? 16 : 32);  // rows of one launch, padded to its 8-row blocks
+  return max_M <= 8 ? 8 : (max_M <= 16 ? 16 : (max_M <= 32 ? 32 : (max_M <= 64 ? 64 : 128)));
+}
+
+// Batch size from which the tcgen05 kernel takes over from the warp-level MMA kernel.
+int tc_min_m() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("MARLIN_B200_TC_MIN_M");  // tuning knob; default below
+    v = e ? atoi(e) : 17;
+    if (v < 1) v = 1;
+  }
+  return v;
 }
 
 }  // namespace
@@ -139,10 +151,11 @@ int marlin_gemm(const void* A, const void* w_packed, const void* s_packed, void*
   if (info.cc_major != 10) return MARLIN_ERR_ARCH;
 
   uint8_t* ws = static_cast<uint8_t*>(workspace);
-  for (int m0 = 0; m0 < M; m0 += kMaxSlabM) {
-    const int m_slab = (M - m0) < kMaxSlabM ? (M - m0) : kMaxSlabM;
-    DensePlan plan;
-    if (!make_dense_plan(m_slab, K, N, info.sm_count, &plan)) return MARLIN_ERR_SHAPE;
+  int m0 = 0;
+  while (m0 < M) {
+    const int rem = M - m0;
+    const bool use_tc = rem >= tc_min_m() && tc_path_supported(rem < kTcMaxSlabM ? rem : kTcMaxSlabM, K, N);
+    const int m_slab = use_tc ? (rem < kTcMaxSlabM ? rem : kTcMaxSlabM) : (rem < kMaxSlabM ? rem : kMaxSlabM);
     GemmParams p;
     p.A = static_cast<const uint16_t*>(A) + (size_t)m0 * K;
     p.wq = static_cast<const uint8_t*>(w_packed);
@@ -151,22 +164,30 @@ int marlin_gemm(const void* A, const void* w_packed, const void* s_packed, void*
     p.M = m_slab;
     p.K = K;
     p.N = N;
-    p.kb = (uint32_t)plan.kb;
+    p.kb = (uint32_t)(K / kTileK);
     p.kb_per_group = G / kTileK;
     p.group_shift = -1;
     for (int sh = 0; sh < 31; ++sh)
       if ((1 << sh) == p.kb_per_group) p.group_shift = sh;
     p.grouped = (G != K) ? 1 : 0;
-    p.ncols = plan.ncols;
-    p.units = (uint32_t)plan.units;
-    p.workers = (uint32_t)plan.workers;
-    p.stages = plan.stages;
-    p.stage_bytes = plan.stage_bytes;
     p.status = reinterpret_cast<int*>(ws + kWsStatusOff);
     p.counters = reinterpret_cast<int*>(ws + kWsCounterOff);
     p.partials = reinterpret_cast<float*>(ws + kWsPartialOff);
     p.slot_floats = kWsSlotCols * slab_mpad(M);
-    if (launch_gemm_dense(plan, p, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MARLIN_ERR_CUDA;
+    if (use_tc) {
+      if (launch_gemm_dense_tc(p, info.sm_count, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return MARLIN_ERR_CUDA;
+    } else {
+      DensePlan plan;
+      if (!make_dense_plan(m_slab, K, N, info.sm_count, &plan)) return MARLIN_ERR_SHAPE;
+      p.ncols = plan.ncols;
+      p.units = (uint32_t)plan.units;
+      p.workers = (uint32_t)plan.workers;
+      p.stages = plan.stages;
+      p.stage_bytes = plan.stage_bytes;
+      if (launch_gemm_dense(plan, p, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MARLIN_ERR_CUDA;
+    }
+    m0 += m_slab;
   }
   return MARLIN_OK;
 }

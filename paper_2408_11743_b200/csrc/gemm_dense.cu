@@ -32,154 +32,11 @@
 #include <cuda.h>
 #include <stdlib.h>
 
+#include "device_utils.cuh"
 #include "marlin_internal.cuh"
 
 namespace marlin_b200 {
 namespace {
-
-// ---------------------------------------------------------------------------------------------
-// PTX wrappers
-// ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n"
-      ".reg .pred p;\n"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      "selp.u32 %0, 1, 0, p;\n"
-      "}\n"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ uint64_t global_timer_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-
-// Bounded wait.  After kWaitLimitNs without completion the CTA-wide abort flag and the status word
-// are set; from then on every wait of the CTA returns at once, so all warps run to the end of the
-// kernel through their normal control flow (no barrier is left unattended) and the host sees
-// MARLIN_ERR_DEVICE_TIMEOUT instead of a hang.
-constexpr uint64_t kWaitLimitNs = 2000000000ull;
-__device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
-  if (mbar_try_wait(bar, parity)) return;
-  uint32_t spins = 0;
-  uint64_t t0 = 0;
-  while (!mbar_try_wait(bar, parity)) {
-    if ((++spins & 255u) == 0) {
-      if (*abort_flag) return;
-      uint64_t now = global_timer_ns();
-      if (t0 == 0) t0 = now;
-      if (now - t0 > kWaitLimitNs) {
-        *abort_flag = 1;
-        atomicExch(status, (int)MARLIN_ERR_DEVICE_TIMEOUT);
-        return;
-      }
-    }
-  }
-}
-
-__device__ __forceinline__ uint64_t policy_evict_first() {
-  uint64_t pol;
-  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-  return pol;
-}
-__device__ __forceinline__ uint64_t policy_evict_last() {
-  uint64_t pol;
-  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
-  return pol;
-}
-// global -> shared bulk copy; dst, src 16-byte aligned, bytes a multiple of 16.
-__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar, uint64_t pol) {
-  asm volatile(
-      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
-      ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(pol)
-      : "memory");
-}
-// One box of a 2-D tensor map -> shared memory (no multicast: every CTA fetches its own copy).
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar,
-                                            uint64_t pol) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
-      " [%0], [%1, {%2, %3}], [%4], %5;"
-      ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(pol)
-      : "memory");
-}
-__device__ __forceinline__ int atom_add_acq_rel_gpu(int* addr, int v) {
-  int old;
-  asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(addr), "r"(v) : "memory");
-  return old;
-}
-__device__ __forceinline__ void named_bar_sync(int id, int threads) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
-}
-
-template <int LUT>
-__device__ __forceinline__ uint32_t lop3(uint32_t a, uint32_t b, uint32_t c) {
-  uint32_t r;
-  asm("lop3.b32 %0, %1, %2, %3, %4;" : "=r"(r) : "r"(a), "r"(b), "r"(c), "n"(LUT));
-  return r;
-}
-__device__ __forceinline__ uint32_t hsub2_u32(uint32_t a, uint32_t b) {
-  uint32_t r;
-  asm("sub.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
-  return r;
-}
-__device__ __forceinline__ uint32_t hfma2_u32(uint32_t a, uint32_t b, uint32_t c) {
-  uint32_t r;
-  asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
-  return r;
-}
-
-// Eight 4-bit codes of one word -> four registers of two fp16 values (q - 8), in the order of the
-// m16n8k16 A fragment.  A code OR'ed under 0x6400 is the fp16 number 1024 + q (1024 + 16 q for the
-// upper nibble of a byte); subtracting 1032, or multiplying by 1/16 and subtracting 72, leaves q - 8
-// exactly (Section 3.4, "Dequantization and Tensor Cores").
-__device__ __forceinline__ void dequant8(uint32_t w, uint32_t (&a)[4]) {
-  constexpr uint32_t LO = 0x000f000fu, HI = 0x00f000f0u, EX = 0x64006400u;
-  constexpr uint32_t SUB = 0x64086408u;  // {1032, 1032}
-  constexpr uint32_t MUL = 0x2c002c00u;  // {1/16, 1/16}
-  constexpr uint32_t ADD = 0xd480d480u;  // {-72, -72}
-  uint32_t w2 = w >> 8;
-  a[0] = hsub2_u32(lop3<0xea>(w, LO, EX), SUB);
-  a[1] = hfma2_u32(lop3<0xea>(w, HI, EX), MUL, ADD);
-  a[2] = hsub2_u32(lop3<0xea>(w2, LO, EX), SUB);
-  a[3] = hfma2_u32(lop3<0xea>(w2, HI, EX), MUL, ADD);
-}
-
-__device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm(
-      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
-// Register re-allocation between warpgroups (all four warps of a warpgroup execute it together).
-template <int N>
-__device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
-template <int N>
-__device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
-
-// Programmatic dependent launch: let the next kernel of the stream start its prologue while this
-// one drains, and wait for the previous kernel's memory before touching anything it may have written.
-__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void pdl_wait_prior_grids() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-
-__device__ __forceinline__ float4 ld_cg_f4(const float4* p) { return __ldcg(p); }
 
 // Optional per-CTA cycle stamps for tuning (built only with -DMARLIN_TIMING; not part of the library).
 #ifdef MARLIN_TIMING
@@ -398,6 +255,15 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
       if (warp == 0 && x == off && it0 == 0) MARLIN_STAMP(4);
       const uint8_t* st = stage0 + (size_t)s * G::STAGE_BYTES;
       const uint4* wp = reinterpret_cast<const uint4*>(st + G::A_BYTES + wn * kChunkBytes) + lane;
+      // codes of this lane: columns g (X) and g + 8 (Y) of each 16-column block j, its 32 rows of the k-block
+      uint32_t X[4][4], Y[4][4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint4 xv = wp[(2 * j) * 32];
+        const uint4 yv = wp[(2 * j + 1) * 32];
+        X[j][0] = xv.x; X[j][1] = xv.y; X[j][2] = xv.z; X[j][3] = xv.w;
+        Y[j][0] = yv.x; Y[j][1] = yv.y; Y[j][2] = yv.z; Y[j][3] = yv.w;
+      }
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         uint32_t bf[MB][8];
@@ -409,22 +275,21 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
           bf[mb][0] = v0.x; bf[mb][1] = v0.y; bf[mb][2] = v0.z; bf[mb][3] = v0.w;
           bf[mb][4] = v1.x; bf[mb][5] = v1.y; bf[mb][6] = v1.z; bf[mb][7] = v1.w;
         }
-        // all four 16-column blocks of this half first, then step by step over k: consecutive MMAs
-        // go to different accumulators, so none waits for the one before it
-        uint32_t ww[4][4];
+        // one word of X and one of Y feed two MMA steps; consecutive MMAs go to different accumulators
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const uint4 wv = wp[(h * 4 + j) * 32];
-          ww[j][0] = wv.x; ww[j][1] = wv.y; ww[j][2] = wv.z; ww[j][3] = wv.w;
-        }
-#pragma unroll
-        for (int t = 0; t < 4; ++t) {
+        for (int u = 0; u < 2; ++u) {
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
-            uint32_t a[4];
-            dequant8(ww[j][t], a);
+            uint32_t x[4], y[4];
+            dequant8(X[j][2 * h + u], x);
+            dequant8(Y[j][2 * h + u], y);
+            const uint32_t a0[4] = {x[0], y[0], x[1], y[1]};
+            const uint32_t a1[4] = {x[2], y[2], x[3], y[3]};
 #pragma unroll
-            for (int mb = 0; mb < MB; ++mb) mma_16816(tmp[j * MB + mb], a, bf[mb][2 * t], bf[mb][2 * t + 1]);
+            for (int mb = 0; mb < MB; ++mb) {
+              mma_16816(tmp[j * MB + mb], a0, bf[mb][4 * u], bf[mb][4 * u + 1]);
+              mma_16816(tmp[j * MB + mb], a1, bf[mb][4 * u + 2], bf[mb][4 * u + 3]);
+            }
           }
         }
       }
@@ -583,6 +448,8 @@ EncodeTiledFn encode_tiled_fn() {
 }
 
 // A[M][K] fp16 row-major as a 2-D tensor (inner K); box = 64 columns x mpad rows, 128-byte swizzle.
+}  // namespace
+
 bool make_a_tensor_map(CUtensorMap* map, const void* A, int M, int K, int mpad) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
@@ -594,6 +461,8 @@ bool make_a_tensor_map(CUtensorMap* map, const void* A, int M, int K, int mpad) 
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
+
+namespace {
 
 template <int MB, int NW>
 cudaError_t launch_one(const DensePlan& plan, const GemmParams& p, cudaStream_t stream) {

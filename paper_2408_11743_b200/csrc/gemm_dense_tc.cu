@@ -1,0 +1,481 @@
+// Dense W4A16 layer for sm_100a, batch sizes 17..128 per launch: tcgen05 tensor cores with the WEIGHTS
+// as the A operand in tensor memory.
+//
+// The warp-level MMA (mma.sync) of the small-batch kernel runs at about a quarter of the tcgen05 rate on
+// this architecture and is out of steam above batch 16.  Here the product is computed transposed, as the
+// paper does for its sparse kernel (Section 4: C = (B^T A^T)^T): per 256-column tile of W and 128-row
+// k-block
+//     D_t[128 channels x MPAD batch rows] += W_t^T[128 x 128] . A^T[128 x MPAD],   t = 0, 1
+// with UMMA shape M = 128 (output channels on the TMEM lanes), N = MPAD (batch), K = 16.
+//
+// One CTA per SM, 384 threads:
+//   warps 0..7   dequantisers: thread = one output channel of the tile.  It reads its 128 codes of the
+//                k-block (four 16-byte shared loads), converts them to fp16 (q - 8) with the
+//                exponent-bias trick (Section 3.4 "Dequantization and Tensor Cores"), multiplies by the
+//                group scale (Section 3.4 "Groups and Instruction Ordering": applied in the main loop)
+//                and writes the 128 values into its TMEM lane with tcgen05.st (64 columns, two k per
+//                column).  Two A-operand slots let conversion of k-block i+1 overlap the MMAs of i.
+//                At the end of a column segment the same warps read the accumulator back (tcgen05.ld),
+//                run the stripe fix-up and store C.
+//   warps 8, 9   producers: per k-block one 16 KB bulk copy of packed weights (evict-first) and one TMA
+//                tensor tile per 64-wide half of the activations (128-byte swizzle = the canonical
+//                K-major UMMA layout, rows >= M zero-filled), into a ring of shared-memory stages.
+//   warp 10      MMA issuer: one thread issues 2 x 8 tcgen05.mma per k-block (A from TMEM, B = the
+//                activation tile through a shared-memory descriptor), then tcgen05.commit to the
+//                barriers that free the A slot and the stage.  It also owns the TMEM allocation.
+//   warp 11      idle (completes the producer warpgroup for setmaxnreg).
+//
+// Stripe partition, fix-up protocol, bounded waits and programmatic dependent launch are those of the
+// small-batch kernel (gemm_dense.cu).
+#include <stdlib.h>
+
+#include "device_utils.cuh"
+#include "marlin_internal.cuh"
+
+namespace marlin_b200 {
+namespace {
+
+// ---------------------------------------------------------------------------------------------
+// tcgen05 wrappers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void tmem_alloc(uint32_t* smem_dst, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_dst)), "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// the mbarrier gets one arrival when all tcgen05 operations issued so far by this thread have completed
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+// D[tmem] (+)= A[tmem] . B[smem descriptor]; fp16 inputs, fp32 accumulation
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
+      "}\n" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// eight consecutive 32-bit columns of this thread's TMEM lane
+__device__ __forceinline__ void tc_st_x8(uint32_t taddr, const uint32_t (&r)[8]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr), "r"(r[0]),
+               "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+               : "memory");
+}
+__device__ __forceinline__ void tc_ld_x32(uint32_t taddr, float (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=f"(r[0]), "=f"(r[1]), "=f"(r[2]), "=f"(r[3]), "=f"(r[4]), "=f"(r[5]), "=f"(r[6]), "=f"(r[7]), "=f"(r[8]),
+        "=f"(r[9]), "=f"(r[10]), "=f"(r[11]), "=f"(r[12]), "=f"(r[13]), "=f"(r[14]), "=f"(r[15]), "=f"(r[16]),
+        "=f"(r[17]), "=f"(r[18]), "=f"(r[19]), "=f"(r[20]), "=f"(r[21]), "=f"(r[22]), "=f"(r[23]), "=f"(r[24]),
+        "=f"(r[25]), "=f"(r[26]), "=f"(r[27]), "=f"(r[28]), "=f"(r[29]), "=f"(r[30]), "=f"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ uint32_t hmul2_u32(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
+
+// K-major operand tile in shared memory, 128-byte swizzle: rows of 64 fp16 (128 bytes), groups of eight
+// rows 1024 bytes apart.  Fields: start address >> 4 (bits 0-13), leading byte offset >> 4 (bits 16-29,
+// one 16-byte unit: the two halves of a K = 16 step are adjacent), stride byte offset >> 4 (bits 32-45:
+// 1024 bytes between 8-row groups), descriptor version 1 (bits 46-47), swizzle mode 128B = 2 (bits 61-63).
+__device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t smem_addr) {
+  return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// kind::f16 instruction descriptor: D fp32 (bits 4-5 = 1), A and B fp16 (0), both K-major (bits 15, 16 = 0),
+// N >> 3 in bits 17-22, M >> 4 in bits 24-28.
+__host__ __device__ constexpr uint32_t instr_desc_f16(int m, int n) {
+  return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+// ---------------------------------------------------------------------------------------------
+// geometry
+// ---------------------------------------------------------------------------------------------
+constexpr int kTcThreads = 384;
+constexpr int kDequantWarps = 8;
+constexpr int kDequantThreads = kDequantWarps * 32;
+constexpr int kTcProducerWarps = 2;
+constexpr int kMmaWarp = 10;
+constexpr int kTcMaxStages = 8;
+constexpr int kTileN = 256;          // columns of W per CTA tile: two UMMA tiles of 128 channels
+constexpr int kASlots = 2;
+constexpr int kTmemCols = 512;
+constexpr int kASlotCol0 = 256;      // A-operand slots live in columns 256..511, accumulators in 0..255
+
+template <int MPAD>
+struct TcGeometry {
+  static constexpr int A_HALF_BYTES = MPAD * 128;
+  static constexpr int A_BYTES = 2 * A_HALF_BYTES;
+  static constexpr int W_BYTES = 4 * kChunkBytes;
+  static constexpr int STAGE_BYTES = A_BYTES + W_BYTES;
+  static constexpr int FIXED_BYTES = 1024;
+  static constexpr int ALIGN_SLACK = 1024;
+  static constexpr int STAGES =
+      (kSmemBudget - FIXED_BYTES - ALIGN_SLACK) / STAGE_BYTES > kTcMaxStages
+          ? kTcMaxStages
+          : (kSmemBudget - FIXED_BYTES - ALIGN_SLACK) / STAGE_BYTES;
+  static constexpr int SMEM_BYTES = FIXED_BYTES + ALIGN_SLACK + STAGES * STAGE_BYTES;
+};
+
+// ---------------------------------------------------------------------------------------------
+// the kernel
+// ---------------------------------------------------------------------------------------------
+template <int MPAD>
+__global__ void __launch_bounds__(kTcThreads, 1)
+gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a) {
+  using G = TcGeometry<MPAD>;
+  constexpr int NSTAGES = G::STAGES;
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem);          // [8]  TMA data of a stage has landed
+  uint64_t* empty = reinterpret_cast<uint64_t*>(smem + 64);    // [8]  stage may be refilled
+  uint64_t* afull = reinterpret_cast<uint64_t*>(smem + 128);   // [2]  A-operand slot written
+  uint64_t* aempty = reinterpret_cast<uint64_t*>(smem + 144);  // [2]  A-operand slot consumed by the MMAs
+  uint64_t* dfull = reinterpret_cast<uint64_t*>(smem + 160);   //      accumulators of a segment complete
+  uint64_t* dempty = reinterpret_cast<uint64_t*>(smem + 168);  //      accumulators read out
+  uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(smem + 176);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + 180);
+  volatile int* last_flag = reinterpret_cast<volatile int*>(smem + 184);
+  uint8_t* stage0 = smem + G::FIXED_BYTES;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t worker = blockIdx.x;
+  const uint32_t U = p.units, P = p.workers, KB = p.kb;
+  const uint32_t u0 = stripe_begin32(worker, U, P), u1 = stripe_begin32(worker + 1, U, P);
+
+  pdl_launch_dependents();
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < NSTAGES; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&empty[s], kDequantWarps + 1);
+    }
+    for (int a = 0; a < kASlots; ++a) {
+      mbar_init(&afull[a], kDequantWarps);
+      mbar_init(&aempty[a], 1);
+    }
+    mbar_init(dfull, 1);
+    mbar_init(dempty, kDequantWarps);
+    *abort_flag = 0;
+    *last_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == kMmaWarp) {
+    tmem_alloc(tmem_base_slot, kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_base_slot;
+
+  if (warp >= kDequantWarps) {
+    setmaxnreg_dec<56>();
+    if (warp < kDequantWarps + kTcProducerWarps) {
+      // ------------------------------- producers --------------------------------------------
+      const int pw = warp - kDequantWarps;
+      if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
+      const uint64_t pol_w = policy_evict_first();
+      const uint64_t pol_a = policy_evict_last();
+      constexpr uint32_t tx_bytes = G::W_BYTES + G::A_BYTES;
+      // weights of (kb, col): the four chunks of a 256-column tile are adjacent, k-blocks follow one another
+      auto weight_src = [&](uint32_t col, uint32_t kb) -> const uint8_t* {
+        return p.wq + ((size_t)col * KB + kb) * (size_t)G::W_BYTES;
+      };
+      // first pass over the ring: weights before the dependency wait, activations after it
+      uint32_t u = u0 + pw;
+      int s = pw;
+      if (lane == 0) {
+        for (; u < u1 && s < NSTAGES; u += kTcProducerWarps, s += kTcProducerWarps) {
+          const uint32_t col = u / KB, kb = u - col * KB;
+          mbar_expect_tx(&full[s], tx_bytes);
+          bulk_g2s(stage0 + (size_t)s * G::STAGE_BYTES + G::A_BYTES, weight_src(col, kb), G::W_BYTES, &full[s], pol_w);
+        }
+      }
+      __syncwarp();
+      pdl_wait_prior_grids();
+      u = u0 + pw;
+      s = pw;
+      for (; u < u1 && s < NSTAGES; u += kTcProducerWarps, s += kTcProducerWarps) {
+        const uint32_t col = u / KB, kb = u - col * KB;
+        if (lane < 2)
+          tma_load_2d(stage0 + (size_t)s * G::STAGE_BYTES + lane * G::A_HALF_BYTES, &tmap_a,
+                      (int)(kb * kTileK + lane * 64), 0, &full[s], pol_a);
+      }
+      uint32_t ph = 1;
+      s -= NSTAGES;
+      for (; u < u1; u += kTcProducerWarps) {
+        const uint32_t col = u / KB, kb = u - col * KB;
+        mbar_wait(&empty[s], ph ^ 1u, abort_flag, p.status);
+        uint8_t* st = stage0 + (size_t)s * G::STAGE_BYTES;
+        if (lane == 0) {
+          mbar_expect_tx(&full[s], tx_bytes);
+          bulk_g2s(st + G::A_BYTES, weight_src(col, kb), G::W_BYTES, &full[s], pol_w);
+        }
+        __syncwarp();
+        if (lane < 2)
+          tma_load_2d(st + lane * G::A_HALF_BYTES, &tmap_a, (int)(kb * kTileK + lane * 64), 0, &full[s], pol_a);
+        s += kTcProducerWarps;
+        if (s >= NSTAGES) { s -= NSTAGES; ph ^= 1u; }
+      }
+      if (*abort_flag) {
+        for (int x = 0; x < 1000; ++x) __nanosleep(1000);
+      }
+      return;
+    }
+    if (warp == kMmaWarp) {
+      // ------------------------------- MMA issuer ---------------------------------------------
+      constexpr uint32_t idesc = instr_desc_f16(128, MPAD);
+      uint32_t it = 0;   // stage counter of this CTA
+      uint32_t seg = 0;  // segment counter
+      uint32_t u = u0;
+      while (u < u1) {
+        const uint32_t kb0 = u % KB;
+        const uint32_t len = min(KB - kb0, u1 - u);
+        // the accumulators are overwritten by the first MMA of the segment: the previous one must be read out
+        mbar_wait(dempty, (seg & 1u) ^ 1u, abort_flag, p.status);
+        for (uint32_t x = 0; x < len; ++x, ++it) {
+          const int s = (int)(it % NSTAGES);
+          const int slot = (int)(it & 1u);
+          mbar_wait(&full[s], (it / NSTAGES) & 1u, abort_flag, p.status);
+          mbar_wait(&afull[slot], (it >> 1) & 1u, abort_flag, p.status);
+          tc_fence_after_sync();
+          if (lane == 0) {
+            const uint32_t a_smem = smem_u32(stage0 + (size_t)s * G::STAGE_BYTES);
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+              const uint32_t d_tmem = tmem_base + (uint32_t)(t * MPAD);
+              const uint32_t a_tmem = tmem_base + (uint32_t)(kASlotCol0 + (slot * 2 + t) * 64);
+#pragma unroll
+              for (int ks = 0; ks < 8; ++ks) {
+                const uint64_t bdesc = smem_desc_k_sw128(a_smem + (ks >> 2) * G::A_HALF_BYTES + (ks & 3) * 32);
+                tc_mma_ts(d_tmem, a_tmem + ks * 8, bdesc, idesc, (x == 0 && ks == 0) ? 0u : 1u);
+              }
+            }
+            tc_commit(&aempty[slot]);  // the A slot may be rewritten
+            tc_commit(&empty[s]);      // the activation tile of the stage may be refilled
+            if (x + 1 == len) tc_commit(dfull);
+          }
+          __syncwarp();
+        }
+        u += len;
+        ++seg;
+      }
+    }
+    // ---- the TMEM owner waits for everybody who touches tensor memory, then frees it ----
+    if (warp == kMmaWarp) {
+      named_bar_sync(2, kDequantThreads + 32);
+      tc_fence_after_sync();
+      tmem_dealloc(tmem_base, kTmemCols);
+    }
+    return;
+  }
+
+  // --------------------------------- dequantisers / epilogue ----------------------------------
+  setmaxnreg_inc<224>();
+  const int tile = warp >> 2;                 // which 128 channels of the 256-column tile
+  const uint32_t lane_win = (uint32_t)(warp & 3) * 32u;  // this warp's TMEM lanes
+  const int n256 = tile * 128 + (int)lane_win + lane;    // column of the thread inside the CTA tile
+  const int q = n256 >> 6, n64 = n256 & 63;
+  const int j = n64 >> 4, b = (n64 >> 3) & 1, g = n64 & 7;
+  const uint32_t vec_off = (uint32_t)q * kChunkBytes + (uint32_t)(((2 * j + b) * 32 + 4 * g) * 16);
+  const int spos = q * 64 + 8 * g + 2 * j + b;  // position of this column's scale inside the tile's 256 scales
+  const int ctid = threadIdx.x;
+  const uint32_t tmem_lane = tmem_base + (lane_win << 16);
+
+  uint32_t it = 0, seg = 0;
+  uint32_t u = u0;
+  bool waited_for_prior_grid = false;
+  while (u < u1) {
+    const uint32_t col = u / KB;
+    const uint32_t kb0 = u % KB;
+    const uint32_t len = min(KB - kb0, u1 - u);
+    const uint16_t* sptr = reinterpret_cast<const uint16_t*>(p.sq) + (size_t)col * kTileN + spos;
+
+    int cur_group = -1;
+    uint32_t s2 = 0;  // {scale, scale} of the open group
+    for (uint32_t x = 0; x < len; ++x, ++it) {
+      const uint32_t kb = kb0 + x;
+      const int gi = p.grouped ? (p.group_shift >= 0 ? (int)(kb >> p.group_shift) : (int)(kb / (uint32_t)p.kb_per_group)) : 0;
+      if (gi != cur_group) {
+        const uint32_t sv = __ldg(sptr + (size_t)gi * p.N);
+        s2 = sv | (sv << 16);
+        cur_group = gi;
+      }
+      const int s = (int)(it % NSTAGES);
+      const int slot = (int)(it & 1u);
+      mbar_wait(&full[s], (it / NSTAGES) & 1u, abort_flag, p.status);
+      const uint8_t* wbase = stage0 + (size_t)s * G::STAGE_BYTES + G::A_BYTES + vec_off;
+      uint4 v[4];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) v[c] = *reinterpret_cast<const uint4*>(wbase + c * 16);
+      // the codes are in registers: the weight part of the stage is free as far as this warp is concerned
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&empty[s]);
+
+      mbar_wait(&aempty[slot], ((it >> 1) & 1u) ^ 1u, abort_flag, p.status);
+      tc_fence_after_sync();
+      const uint32_t a_col = tmem_lane + (uint32_t)(kASlotCol0 + (slot * 2 + tile) * 64);
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          uint32_t lo[4], hi[4], r[8];
+          dequant8(w[2 * h], lo);      // rows 64h + 16c + 0..7
+          dequant8(w[2 * h + 1], hi);  // rows 64h + 16c + 8..15
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            r[e] = hmul2_u32(lo[e], s2);
+            r[4 + e] = hmul2_u32(hi[e], s2);
+          }
+          tc_st_x8(a_col + (uint32_t)(32 * h + 8 * c), r);  // column = row / 2
+        }
+      }
+      tc_wait_st();
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&afull[slot]);
+    }
+
+    // ---- segment end: read the accumulators, fix-up across CTAs, store C ----
+    mbar_wait(dfull, seg & 1u, abort_flag, p.status);
+    tc_fence_after_sync();
+    float acc[MPAD];
+#pragma unroll
+    for (int cc = 0; cc < MPAD / 32; ++cc) {
+      float part[32];
+      tc_ld_x32(tmem_lane + (uint32_t)(tile * MPAD + cc * 32), part);
+      tc_wait_ld();
+#pragma unroll
+      for (int e = 0; e < 32; ++e) acc[cc * 32 + e] = part[e];
+    }
+    tc_fence_before_sync();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(dempty);
+    ++seg;
+
+    if (!waited_for_prior_grid) {
+      // first write to C or the workspace: the previous kernel of the stream must be done with them
+      pdl_wait_prior_grids();
+      waited_for_prior_grid = true;
+    }
+    const int first_w = (int)stripe_owner32(col * KB, U, P);
+    const int last_w = (int)stripe_owner32((col + 1) * KB - 1, U, P);
+    bool store = true;
+    if (last_w > first_w) {
+      // partial tile layout in the workspace: float4 index = (m / 4) * 256 + column, i.e. coalesced over columns
+      const int my_slot = 2 * (int)worker + (col != u0 / KB ? 1 : 0);
+      float4* mine = reinterpret_cast<float4*>(p.partials + (size_t)my_slot * p.slot_floats) + n256;
+#pragma unroll
+      for (int m4 = 0; m4 < MPAD / 4; ++m4)
+        mine[m4 * kTileN] = make_float4(acc[4 * m4], acc[4 * m4 + 1], acc[4 * m4 + 2], acc[4 * m4 + 3]);
+      named_bar_sync(1, kDequantThreads);
+      if (ctid == 0) {
+        const int old = atom_add_acq_rel_gpu(&p.counters[col], 1);
+        const int is_last = (old == last_w - first_w) ? 1 : 0;
+        if (is_last) p.counters[col] = 0;
+        *last_flag = is_last;
+      }
+      named_bar_sync(1, kDequantThreads);
+      store = (*last_flag != 0);
+      if (store) {
+        // the last arriver adds all partials, its own included, in stripe order (deterministic)
+        for (int w = first_w; w <= last_w; ++w) {
+          const int slot = 2 * w + (col != stripe_begin32(w, U, P) / KB ? 1 : 0);
+          const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)slot * p.slot_floats) + n256;
+#pragma unroll
+          for (int m4 = 0; m4 < MPAD / 4; ++m4) {
+            const float4 t4 = ld_cg_f4(src + m4 * kTileN);
+            if (w == first_w) {
+              acc[4 * m4] = t4.x; acc[4 * m4 + 1] = t4.y; acc[4 * m4 + 2] = t4.z; acc[4 * m4 + 3] = t4.w;
+            } else {
+              acc[4 * m4] += t4.x; acc[4 * m4 + 1] += t4.y; acc[4 * m4 + 2] += t4.z; acc[4 * m4 + 3] += t4.w;
+            }
+          }
+        }
+      }
+      named_bar_sync(1, kDequantThreads);  // last_flag may be rewritten by the next segment
+    }
+    if (store) {
+      uint16_t* cptr = p.C + (size_t)col * kTileN + n256;
+#pragma unroll
+      for (int m = 0; m < MPAD; ++m)
+        if (m < p.M) cptr[(size_t)m * p.N] = __half_as_ushort(__float2half_rn(acc[m]));
+    }
+    u += len;
+  }
+  // everybody is done with tensor memory
+  tc_fence_before_sync();
+  named_bar_sync(2, kDequantThreads + 32);
+}
+
+template <int MPAD>
+cudaError_t launch_tc(const GemmParams& p, int workers, cudaStream_t stream) {
+  using G = TcGeometry<MPAD>;
+  auto kernel = gemm_dense_tc_kernel<MPAD>;
+  static bool attr_set[64] = {};
+  int dev = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM_BYTES);
+    if (err != cudaSuccess) return err;
+    if (dev >= 0 && dev < 64) attr_set[dev] = true;
+  }
+  alignas(64) CUtensorMap tmap;
+  if (!make_a_tensor_map(&tmap, p.A, p.M, p.K, MPAD)) return cudaErrorInvalidValue;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(workers);
+  cfg.blockDim = dim3(kTcThreads);
+  cfg.dynamicSmemBytes = G::SMEM_BYTES;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, p, tmap);
+}
+
+}  // namespace
+
+bool tc_path_supported(int m_slab, int K, int N) {
+  return m_slab >= 1 && m_slab <= kTcMaxSlabM && N % kTileN == 0 && K % kTileK == 0;
+}
+
+int tc_mpad(int m_slab) { return m_slab <= 32 ? 32 : (m_slab <= 64 ? 64 : 128); }
+
+cudaError_t launch_gemm_dense_tc(GemmParams p, int sm_count, cudaStream_t stream) {
+  // stripe plan for 256-column tiles
+  const long long units = (long long)(p.N / kTileN) * (p.K / kTileK);
+  long long workers = sm_count < kMaxWorkers ? sm_count : kMaxWorkers;
+  if (workers > units) workers = units;
+  p.ncols = p.N / kTileN;
+  p.units = (uint32_t)units;
+  p.workers = (uint32_t)workers;
+  const int mpad = tc_mpad(p.M);
+  if (mpad == 32) return launch_tc<32>(p, (int)workers, stream);
+  if (mpad == 64) return launch_tc<64>(p, (int)workers, stream);
+  return launch_tc<128>(p, (int)workers, stream);
+}
+
+}  // namespace marlin_b200

@@ -12,18 +12,17 @@
 //     chunk index = sc * 4 * (K/128) + kb * cs + (nb % 4)
 //   so the weights a CTA streams for a 256-column tile are one contiguous run of memory, k-block after
 //   k-block, and one k-block of a tile is a single 16 KB bulk copy.
-//   word index = ((chunk index * 8 + i) * 32 + lane) * 4 + t
-//     i    = 4*h + j                         h: which 64-row half of the k-block, j: which 16 columns
-//     lane = 4*g + c                         the consuming thread; g = lane / 4, c = lane % 4
-//     t    = 0..3                            which 16-row MMA step inside the half
-//   nibble p of the word (bits 4p..4p+3): with r = p % 4,
-//     column n = 64*nb + 16*j + g + 8*(r & 1)
-//     row    k = 128*kb + 64*h + 16*c + 4*t + 2*(r >> 1) + (p >> 2)
-//   so the nibble pairs (0,4) (1,5) (2,6) (3,7) are the four 2 x fp16 registers of the m16n8k16
-//   A-operand fragment with the weights transposed onto the 16-wide side, and thread c owns 16
-//   consecutive rows of k inside each 64-row half (the order of k inside an MMA step is free as long
-//   as both operands agree).
-//
+//   Inside a chunk, 16-byte vector number v = (2*j + b) * 32 + lane holds 32 codes of ONE column:
+//     column n = 64*nb + 16*j + 8*b + g        (lane = 4*g + c, g = lane / 4, c = lane % 4)
+//     rows   k = 128*kb + {16*c .. 16*c + 15} and 128*kb + 64 + {16*c .. 16*c + 15}
+//   word w of the vector (w = 2*h + u) holds rows 128*kb + 64*h + 16*c + 8*u + o, o = 0..7, with
+//   row offset o in nibble (o >> 1) + 4*(o & 1): one AND+OR pulls out the two codes of rows (2i, 2i+1).
+//   Two readers use this order:
+//     - the warp-level MMA kernel: lane (g, c) reads the vectors of columns g and g + 8 of a 16-column
+//       block; one word of each gives the A-operand registers of two m16n8k16 steps (weights on the
+//       16-wide side), and the lane's activations for its rows are 16 contiguous fp16 per 64-row half;
+//     - the tcgen05 kernel: a thread owns one column and reads its four vectors (c = 0..3), i.e. all
+//       128 rows of the k-block, dequantises and stores them to tensor memory in row order.
 //   scales: inside every run of 64 columns, position 8*g + 2*j + b holds column 16*j + 8*b + g,
 //   so that the 8 scales a thread needs are one 16-byte load.
 #include "marlin_internal.cuh"
@@ -31,11 +30,13 @@
 namespace marlin_b200 {
 namespace {
 
-__device__ __forceinline__ void decode_position(int p, int g, int c, int t, int h, int j, int kb, int nb, int* k,
-                                                int* n) {
-  int r = p & 3;
-  *n = 64 * nb + 16 * j + g + 8 * (r & 1);
-  *k = 128 * kb + 64 * h + 16 * c + 4 * t + 2 * (r >> 1) + (p >> 2);
+// word `wi` (0..1023) of chunk (kb, nb), nibble p -> matrix position
+__device__ __forceinline__ void decode_position(int wi, int p, int kb, int nb, int* k, int* n) {
+  int w = wi & 3, lane = (wi >> 2) & 31, i = wi >> 7;
+  int g = lane >> 2, c = lane & 3, j = i >> 1, b = i & 1;
+  int o = 2 * (p & 3) + (p >> 2);
+  *n = 64 * nb + 16 * j + 8 * b + g;
+  *k = 128 * kb + 64 * (w >> 1) + 16 * c + 8 * (w & 1) + o;
 }
 
 // chunk index <-> (kb, nb)
@@ -63,18 +64,14 @@ __global__ void pack_weights_kernel(const uint32_t* __restrict__ q, uint32_t* __
   long long total = (long long)K * N / 8;
   for (long long wi = blockIdx.x * (long long)blockDim.x + threadIdx.x; wi < total;
        wi += (long long)gridDim.x * blockDim.x) {
-    int t = (int)(wi & 3);
-    int lane = (int)((wi >> 2) & 31);
-    int i = (int)((wi >> 7) & 7);
     int nb64 = N / 64;
     int kb, nb;
     chunk_coords(wi >> 10, K / 128, nb64, &kb, &nb);
-    int g = lane >> 2, c = lane & 3, h = i >> 2, j = i & 3;
     uint32_t out = 0;
 #pragma unroll
     for (int p = 0; p < 8; ++p) {
       int k, n;
-      decode_position(p, g, c, t, h, j, kb, nb, &k, &n);
+      decode_position((int)(wi & 1023), p, kb, nb, &k, &n);
       uint32_t code = (q[(size_t)(k >> 3) * N + n] >> (4 * (k & 7))) & 15u;
       out |= code << (4 * p);
     }
@@ -89,16 +86,15 @@ __global__ void unpack_weights_kernel(const uint32_t* __restrict__ wq, uint32_t*
        qi += (long long)gridDim.x * blockDim.x) {
     int n = (int)(qi % N);
     int k8 = (int)(qi / N);
-    int nb = n >> 6, j = (n >> 4) & 3, row = n & 15;
-    int g = row & 7, rbit0 = row >> 3;
+    int nb = n >> 6, j = (n >> 4) & 3, b = (n >> 3) & 1, g = n & 7;
     uint32_t out = 0;
 #pragma unroll
     for (int jn = 0; jn < 8; ++jn) {
       int k = 8 * k8 + jn;
-      int kb = k >> 7, h = (k >> 6) & 1, c = (k >> 4) & 3, t = (k >> 2) & 3, e = k & 3;
-      int p = (rbit0 | ((e >> 1) << 1)) + 4 * (e & 1);
-      int lane = 4 * g + c, i = 4 * h + j;
-      long long wi = ((chunk_index(kb, nb, K / 128, nb64) * 8 + i) * 32 + lane) * 4 + t;
+      int kb = k >> 7, h = (k >> 6) & 1, c = (k >> 4) & 3, u = (k >> 3) & 1, o = k & 7;
+      int p = (o >> 1) + 4 * (o & 1);
+      int lane = 4 * g + c, i = 2 * j + b, w = 2 * h + u;
+      long long wi = ((chunk_index(kb, nb, K / 128, nb64) * 8 + i) * 32 + lane) * 4 + w;
       uint32_t code = (wq[wi] >> (4 * p)) & 15u;
       out |= code << (4 * jn);
     }
