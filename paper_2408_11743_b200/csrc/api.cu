@@ -60,7 +60,7 @@ int tc_min_m() {
   static int v = -1;
   if (v < 0) {
     const char* e = getenv("MARLIN_B200_TC_MIN_M");  // tuning knob; default below
-    v = e ? atoi(e) : 17;
+    v = e ? atoi(e) : 33;
     if (v < 1) v = 1;
   }
   return v;
@@ -101,9 +101,21 @@ size_t marlin_packed_meta_bytes(int K, int N) {
   return (size_t)K * N / 8;
 }
 
+// Workspace map: [status word, counters: 8192 bytes][partial-tile slots of the warp-MMA kernel]
+// ... [fp32 accumulation tiles of the tcgen05 kernel, placed at the END of the buffer].  Everything is
+// zero at rest; both kernels leave it that way.
+static size_t mma_slot_bytes(int max_M) {
+  const int rows = slab_mpad(max_M) < kMaxSlabM ? slab_mpad(max_M) : kMaxSlabM;
+  return (size_t)2 * kMaxWorkers * kWsSlotCols * rows * sizeof(float);
+}
+static size_t tc_tile_bytes(int max_M, int N) {
+  if (max_M < tc_min_m() || N % 256) return 0;
+  return (size_t)N * (size_t)tc_mpad(max_M < kTcMaxSlabM ? max_M : kTcMaxSlabM) * sizeof(float);
+}
+
 size_t marlin_workspace_bytes(int max_M, int K, int N) {
   if (max_M < 1 || !shape_ok(K, N)) return 0;
-  return kWsPartialOff + (size_t)2 * kMaxWorkers * kWsSlotCols * slab_mpad(max_M) * sizeof(float);
+  return kWsPartialOff + mma_slot_bytes(max_M) + tc_tile_bytes(max_M, N);
 }
 
 int marlin_pack(const uint32_t* q_kpacked, const void* scales, void* w_packed, void* s_packed, int K, int N,
@@ -173,7 +185,9 @@ int marlin_gemm(const void* A, const void* w_packed, const void* s_packed, void*
     p.status = reinterpret_cast<int*>(ws + kWsStatusOff);
     p.counters = reinterpret_cast<int*>(ws + kWsCounterOff);
     p.partials = reinterpret_cast<float*>(ws + kWsPartialOff);
-    p.slot_floats = kWsSlotCols * slab_mpad(M);
+    p.tc_tiles = use_tc ? reinterpret_cast<float*>(ws + ((workspace_bytes & ~(size_t)255) - tc_tile_bytes(m_slab, N)))
+                        : nullptr;
+    p.slot_floats = kWsSlotCols * (slab_mpad(m_slab) < kMaxSlabM ? slab_mpad(m_slab) : kMaxSlabM);
     if (use_tc) {
       if (launch_gemm_dense_tc(p, info.sm_count, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return MARLIN_ERR_CUDA;

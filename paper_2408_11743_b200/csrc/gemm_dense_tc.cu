@@ -25,8 +25,8 @@
 //                barriers that free the A slot and the stage.  It also owns the TMEM allocation.
 //   warp 11      idle (completes the producer warpgroup for setmaxnreg).
 //
-// Stripe partition, fix-up protocol, bounded waits and programmatic dependent launch are those of the
-// small-batch kernel (gemm_dense.cu).
+// Stripe partition, bounded waits and programmatic dependent launch are those of the small-batch kernel
+// (gemm_dense.cu); the stripe fix-up adds the partial tiles with L2 reductions instead of gathering them.
 #include <stdlib.h>
 
 #include "device_utils.cuh"
@@ -86,6 +86,10 @@ __device__ __forceinline__ void tc_ld_x32(uint32_t taddr, float (&r)[32]) {
       : "r"(taddr)
       : "memory");
 }
+// fire-and-forget fp32 vector reduction at the L2
+__device__ __forceinline__ void red_add_f32x4(float4* addr, float a, float b, float c, float d) {
+  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
 __device__ __forceinline__ uint32_t hmul2_u32(uint32_t a, uint32_t b) {
   uint32_t r;
   asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
@@ -106,6 +110,13 @@ __host__ __device__ constexpr uint32_t instr_desc_f16(int m, int n) {
   return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
+#ifdef MARLIN_TIMING
+__device__ long long g_timing_tc[kMaxWorkers][16];
+#define MARLIN_STAMP(slot) do { if (lane == 0) g_timing_tc[blockIdx.x][slot] = (long long)global_timer_ns(); } while (0)
+#else
+#define MARLIN_STAMP(slot) do { } while (0)
+#endif
+
 // ---------------------------------------------------------------------------------------------
 // geometry
 // ---------------------------------------------------------------------------------------------
@@ -116,9 +127,7 @@ constexpr int kTcProducerWarps = 2;
 constexpr int kMmaWarp = 10;
 constexpr int kTcMaxStages = 8;
 constexpr int kTileN = 256;          // columns of W per CTA tile: two UMMA tiles of 128 channels
-constexpr int kASlots = 2;
 constexpr int kTmemCols = 512;
-constexpr int kASlotCol0 = 256;      // A-operand slots live in columns 256..511, accumulators in 0..255
 
 template <int MPAD>
 struct TcGeometry {
@@ -133,6 +142,10 @@ struct TcGeometry {
           ? kTcMaxStages
           : (kSmemBudget - FIXED_BYTES - ALIGN_SLACK) / STAGE_BYTES;
   static constexpr int SMEM_BYTES = FIXED_BYTES + ALIGN_SLACK + STAGES * STAGE_BYTES;
+  // tensor memory: accumulators of the two 128-channel tiles in columns [0, 2*MPAD), then as many
+  // A-operand slots (2 tiles x 64 columns each) as fit in the 512 columns
+  static constexpr int A_SLOTS = (kTmemCols - 2 * MPAD) / 128 > 4 ? 4 : (kTmemCols - 2 * MPAD) / 128;
+  static constexpr int A_COL0 = kTmemCols - A_SLOTS * 128;
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -143,17 +156,18 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a) {
   using G = TcGeometry<MPAD>;
   constexpr int NSTAGES = G::STAGES;
+  constexpr int NSLOTS = G::A_SLOTS;
   extern __shared__ __align__(128) uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   uint64_t* full = reinterpret_cast<uint64_t*>(smem);          // [8]  TMA data of a stage has landed
   uint64_t* empty = reinterpret_cast<uint64_t*>(smem + 64);    // [8]  stage may be refilled
-  uint64_t* afull = reinterpret_cast<uint64_t*>(smem + 128);   // [2]  A-operand slot written
-  uint64_t* aempty = reinterpret_cast<uint64_t*>(smem + 144);  // [2]  A-operand slot consumed by the MMAs
-  uint64_t* dfull = reinterpret_cast<uint64_t*>(smem + 160);   //      accumulators of a segment complete
-  uint64_t* dempty = reinterpret_cast<uint64_t*>(smem + 168);  //      accumulators read out
-  uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(smem + 176);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + 180);
-  volatile int* last_flag = reinterpret_cast<volatile int*>(smem + 184);
+  uint64_t* afull = reinterpret_cast<uint64_t*>(smem + 128);   // [4]  A-operand slot written
+  uint64_t* aempty = reinterpret_cast<uint64_t*>(smem + 160);  // [4]  A-operand slot consumed by the MMAs
+  uint64_t* dfull = reinterpret_cast<uint64_t*>(smem + 192);   //      accumulators of a segment complete
+  uint64_t* dempty = reinterpret_cast<uint64_t*>(smem + 200);  //      accumulators read out
+  uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(smem + 208);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + 212);
+  volatile int* last_flag = reinterpret_cast<volatile int*>(smem + 216);
   uint8_t* stage0 = smem + G::FIXED_BYTES;
 
   const int warp = threadIdx.x >> 5;
@@ -163,12 +177,13 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
   const uint32_t u0 = stripe_begin32(worker, U, P), u1 = stripe_begin32(worker + 1, U, P);
 
   pdl_launch_dependents();
+  if (warp == 0) MARLIN_STAMP(10);
   if (threadIdx.x == 0) {
     for (int s = 0; s < NSTAGES; ++s) {
       mbar_init(&full[s], 1);
       mbar_init(&empty[s], kDequantWarps + 1);
     }
-    for (int a = 0; a < kASlots; ++a) {
+    for (int a = 0; a < NSLOTS; ++a) {
       mbar_init(&afull[a], kDequantWarps);
       mbar_init(&aempty[a], 1);
     }
@@ -186,6 +201,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_base_slot;
+  if (warp == 0) MARLIN_STAMP(0);
 
   if (warp >= kDequantWarps) {
     setmaxnreg_dec<56>();
@@ -211,7 +227,9 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         }
       }
       __syncwarp();
+      if (pw == 0) MARLIN_STAMP(1);
       pdl_wait_prior_grids();
+      if (pw == 0) MARLIN_STAMP(11);
       u = u0 + pw;
       s = pw;
       for (; u < u1 && s < NSTAGES; u += kTcProducerWarps, s += kTcProducerWarps) {
@@ -236,6 +254,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         s += kTcProducerWarps;
         if (s >= NSTAGES) { s -= NSTAGES; ph ^= 1u; }
       }
+      if (pw == 0) MARLIN_STAMP(3);
       if (*abort_flag) {
         for (int x = 0; x < 1000; ++x) __nanosleep(1000);
       }
@@ -254,19 +273,21 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         mbar_wait(dempty, (seg & 1u) ^ 1u, abort_flag, p.status);
         for (uint32_t x = 0; x < len; ++x, ++it) {
           const int s = (int)(it % NSTAGES);
-          const int slot = (int)(it & 1u);
+          const int slot = (int)(it % NSLOTS);
           mbar_wait(&full[s], (it / NSTAGES) & 1u, abort_flag, p.status);
-          mbar_wait(&afull[slot], (it >> 1) & 1u, abort_flag, p.status);
+          mbar_wait(&afull[slot], (it / NSLOTS) & 1u, abort_flag, p.status);
+          if (it == 0) MARLIN_STAMP(4);
           tc_fence_after_sync();
           if (lane == 0) {
-            const uint32_t a_smem = smem_u32(stage0 + (size_t)s * G::STAGE_BYTES);
+            // descriptor of the first K = 16 step of the stage; the others differ in the address field only
+            const uint64_t desc0 = smem_desc_k_sw128(smem_u32(stage0 + (size_t)s * G::STAGE_BYTES));
 #pragma unroll
             for (int t = 0; t < 2; ++t) {
               const uint32_t d_tmem = tmem_base + (uint32_t)(t * MPAD);
-              const uint32_t a_tmem = tmem_base + (uint32_t)(kASlotCol0 + (slot * 2 + t) * 64);
+              const uint32_t a_tmem = tmem_base + (uint32_t)(G::A_COL0 + (slot * 2 + t) * 64);
 #pragma unroll
               for (int ks = 0; ks < 8; ++ks) {
-                const uint64_t bdesc = smem_desc_k_sw128(a_smem + (ks >> 2) * G::A_HALF_BYTES + (ks & 3) * 32);
+                const uint64_t bdesc = desc0 + (uint64_t)(((ks >> 2) * G::A_HALF_BYTES + (ks & 3) * 32) >> 4);
                 tc_mma_ts(d_tmem, a_tmem + ks * 8, bdesc, idesc, (x == 0 && ks == 0) ? 0u : 1u);
               }
             }
@@ -279,6 +300,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         u += len;
         ++seg;
       }
+      MARLIN_STAMP(5);
     }
     // ---- the TMEM owner waits for everybody who touches tensor memory, then frees it ----
     if (warp == kMmaWarp) {
@@ -321,8 +343,11 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         cur_group = gi;
       }
       const int s = (int)(it % NSTAGES);
-      const int slot = (int)(it & 1u);
+      const int slot = (int)(it % NSLOTS);
+      const bool tr = (warp == 0 && it == 6);
+      if (tr) MARLIN_STAMP(12);
       mbar_wait(&full[s], (it / NSTAGES) & 1u, abort_flag, p.status);
+      if (tr) MARLIN_STAMP(13);
       const uint8_t* wbase = stage0 + (size_t)s * G::STAGE_BYTES + G::A_BYTES + vec_off;
       uint4 v[4];
 #pragma unroll
@@ -331,9 +356,10 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty[s]);
 
-      mbar_wait(&aempty[slot], ((it >> 1) & 1u) ^ 1u, abort_flag, p.status);
+      mbar_wait(&aempty[slot], ((it / NSLOTS) & 1u) ^ 1u, abort_flag, p.status);
+      if (tr) MARLIN_STAMP(14);
       tc_fence_after_sync();
-      const uint32_t a_col = tmem_lane + (uint32_t)(kASlotCol0 + (slot * 2 + tile) * 64);
+      const uint32_t a_col = tmem_lane + (uint32_t)(G::A_COL0 + (slot * 2 + tile) * 64);
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         const uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
@@ -350,14 +376,18 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
           tc_st_x8(a_col + (uint32_t)(32 * h + 8 * c), r);  // column = row / 2
         }
       }
+      if (tr) MARLIN_STAMP(15);
       tc_wait_st();
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(&afull[slot]);
+      if (tr) MARLIN_STAMP(2);
     }
 
     // ---- segment end: read the accumulators, fix-up across CTAs, store C ----
+    if (warp == 0) MARLIN_STAMP(6);
     mbar_wait(dfull, seg & 1u, abort_flag, p.status);
+    if (warp == 0) MARLIN_STAMP(7);
     tc_fence_after_sync();
     float acc[MPAD];
 #pragma unroll
@@ -382,12 +412,17 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
     const int last_w = (int)stripe_owner32((col + 1) * KB - 1, U, P);
     bool store = true;
     if (last_w > first_w) {
-      // partial tile layout in the workspace: float4 index = (m / 4) * 256 + column, i.e. coalesced over columns
-      const int my_slot = 2 * (int)worker + (col != u0 / KB ? 1 : 0);
-      float4* mine = reinterpret_cast<float4*>(p.partials + (size_t)my_slot * p.slot_floats) + n256;
+      // The column tile is shared by several CTAs.  With up to 128 rows a partial tile is large and
+      // a small layer splits every column many ways, so the sum is left to the L2: every contributor
+      // adds its partial into the tile's fp32 accumulation buffer with fire-and-forget reductions
+      // (float4 index = (m / 4) * 256 + column: coalesced over columns), the last arriver reads the
+      // total, clears the buffer for the next call and stores C.  (The order of these fp32 additions
+      // is not fixed, so the last bits of a shared tile can differ from run to run.)
+      float* tile_acc = p.tc_tiles + (size_t)col * (kTileN * MPAD);
+      float4* mine = reinterpret_cast<float4*>(tile_acc) + n256;
 #pragma unroll
       for (int m4 = 0; m4 < MPAD / 4; ++m4)
-        mine[m4 * kTileN] = make_float4(acc[4 * m4], acc[4 * m4 + 1], acc[4 * m4 + 2], acc[4 * m4 + 3]);
+        red_add_f32x4(mine + m4 * kTileN, acc[4 * m4], acc[4 * m4 + 1], acc[4 * m4 + 2], acc[4 * m4 + 3]);
       named_bar_sync(1, kDequantThreads);
       if (ctid == 0) {
         const int old = atom_add_acq_rel_gpu(&p.counters[col], 1);
@@ -398,20 +433,13 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       named_bar_sync(1, kDequantThreads);
       store = (*last_flag != 0);
       if (store) {
-        // the last arriver adds all partials, its own included, in stripe order (deterministic)
-        for (int w = first_w; w <= last_w; ++w) {
-          const int slot = 2 * w + (col != stripe_begin32(w, U, P) / KB ? 1 : 0);
-          const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)slot * p.slot_floats) + n256;
 #pragma unroll
-          for (int m4 = 0; m4 < MPAD / 4; ++m4) {
-            const float4 t4 = ld_cg_f4(src + m4 * kTileN);
-            if (w == first_w) {
-              acc[4 * m4] = t4.x; acc[4 * m4 + 1] = t4.y; acc[4 * m4 + 2] = t4.z; acc[4 * m4 + 3] = t4.w;
-            } else {
-              acc[4 * m4] += t4.x; acc[4 * m4 + 1] += t4.y; acc[4 * m4 + 2] += t4.z; acc[4 * m4 + 3] += t4.w;
-            }
-          }
+        for (int m4 = 0; m4 < MPAD / 4; ++m4) {
+          const float4 t4 = ld_cg_f4(mine + m4 * kTileN);
+          acc[4 * m4] = t4.x; acc[4 * m4 + 1] = t4.y; acc[4 * m4 + 2] = t4.z; acc[4 * m4 + 3] = t4.w;
         }
+#pragma unroll
+        for (int m4 = 0; m4 < MPAD / 4; ++m4) mine[m4 * kTileN] = make_float4(0.f, 0.f, 0.f, 0.f);
       }
       named_bar_sync(1, kDequantThreads);  // last_flag may be rewritten by the next segment
     }
@@ -422,7 +450,9 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         if (m < p.M) cptr[(size_t)m * p.N] = __half_as_ushort(__float2half_rn(acc[m]));
     }
     u += len;
+    if (warp == 0) MARLIN_STAMP(8);
   }
+  if (warp == 0) MARLIN_STAMP(9);
   // everybody is done with tensor memory
   tc_fence_before_sync();
   named_bar_sync(2, kDequantThreads + 32);
@@ -457,6 +487,12 @@ cudaError_t launch_tc(const GemmParams& p, int workers, cudaStream_t stream) {
 }
 
 }  // namespace
+
+#ifdef MARLIN_TIMING
+extern "C" __attribute__((visibility("default"))) int marlin_timing_read_tc(void* host) {
+  return (int)cudaMemcpyFromSymbol(host, g_timing_tc, sizeof(g_timing_tc));
+}
+#endif
 
 bool tc_path_supported(int m_slab, int K, int N) {
   return m_slab >= 1 && m_slab <= kTcMaxSlabM && N % kTileN == 0 && K % kTileK == 0;

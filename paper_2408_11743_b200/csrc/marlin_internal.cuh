@@ -67,7 +67,8 @@ struct GemmParams {
   int stage_bytes;
   int* status;
   int* counters;
-  float* partials;
+  float* partials;   // warp-MMA kernel: partial-tile slots
+  float* tc_tiles;   // tcgen05 kernel: one fp32 accumulation tile per 256-column tile
   int slot_floats;   // floats per partial-tile slot
 };
 

@@ -67,7 +67,14 @@ def test_same_layer_many_batch_sizes_and_repeatability(marlin, oracle_lib):
         # but the bound's rms is over the compared block
         _assert_close(oracle_lib, C, np.ascontiguousarray(C_ref[:M]))
         C2 = layer(case.A[:M])
-        assert np.array_equal(C.view(np.uint16), C2.view(np.uint16))  # deterministic fix-up
+        if M <= 32:
+            # warp-MMA kernel: partial tiles are summed in stripe order, the result is reproducible bit for bit
+            assert np.array_equal(C.view(np.uint16), C2.view(np.uint16))
+        else:
+            # tcgen05 kernel: shared tiles are summed by L2 reductions in arrival order (fp32): equal up to
+            # the last bit of the fp16 result (one fp16 ulp is up to ~0.1 of the allowance here)
+            bad, worst, _ = oracle_lib.check_tolerance(C2, C)
+            assert bad == 0 and worst < 0.25
 
 
 def test_zero_codes_give_zero(marlin):
@@ -157,3 +164,17 @@ def test_errors_and_status(marlin):
     layer(case.A)
     counters = to_host(layer.ws[256:256 + 4096]).view(np.int32)
     assert np.all(counters == 0)
+
+
+def test_workspace_is_clean_after_large_batch_calls(marlin, oracle_lib):
+    # the tcgen05 kernel accumulates shared tiles in the workspace and must leave them zero for the next call
+    K, N, G = 1024, 512, 128
+    case = inputs.make_dense(128, K, N, G, seed=12)
+    layer = DenseLayer(marlin, case.q_kpacked, case.S, G, max_M=128)
+    C_ref = oracle_lib.gemm(case.A, case.q_kpacked, case.S, G)
+    for M in (128, 40, 128, 64):
+        C = layer(case.A[:M])
+        _assert_close(oracle_lib, C, np.ascontiguousarray(C_ref[:M]))
+        ws = to_host(layer.ws)
+        assert np.all(ws[256:8192] == 0)                    # counters
+        assert np.all(ws[-N * 128 * 4:] == 0)               # accumulation tiles (placed at the end)
