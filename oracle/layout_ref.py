@@ -51,3 +51,65 @@ def pack_scales(S: np.ndarray) -> np.ndarray:
     g, j, b = pos >> 3, (pos >> 1) & 3, pos & 1
     src = 16 * j + 8 * b + g
     return S.reshape(R, N // 64, 64)[:, :, src].reshape(R, N)
+
+
+# ---- 2:4 variant ---------------------------------------------------------------------------------------
+# Per chunk (128 rows of the original K = 64 kept rows, 64 columns; chunks ordered as in the dense layout):
+#   codes (512 words): word (j*32 + lane)*4 + t, lane = 4g + c; nibble p (r = p % 4, e = p // 4) = kept value e of
+#     column 64nb + 16j + g + 8(r & 1), MMA group gamma = c + 4(r >> 1) of step t, where MMA group gamma stands for
+#     the actual group Gamma = 4(gamma % 2) + gamma // 2 of the step's eight groups of four original rows;
+#     kept-value row T = 2*(32kb + 8t + Gamma) + e.
+#   metadata (256 words): word ((j // 2)*32 + lane)*4 + (j % 2)*2 + w is supplied by lane (g, c) for step
+#     t = c // 2 + 2w; nibble x = idx_first | idx_second << 2 for column 64nb + 16j + g + 8(x // 4), MMA group
+#     4(c % 2) + x % 4.
+
+def _chunk_order(KB, NB):
+    order = np.empty((KB, NB), dtype=np.int64)
+    for nb_ in range(NB):
+        sc = nb_ // 4
+        cs = min(4, NB - 4 * sc)
+        order[:, nb_] = sc * 4 * KB + np.arange(KB) * cs + nb_ % 4
+    return order
+
+
+def pack_sparse_codes(Qc: np.ndarray, K: int) -> np.ndarray:
+    """Kept codes Qc[K/2, N] (uint8) -> packed uint32 words (K*N/16)."""
+    N = Qc.shape[1]
+    KB, NB = K // 128, N // 64
+    kb, nb, j, g, c, t, p = np.meshgrid(np.arange(KB), np.arange(NB), np.arange(4), np.arange(8), np.arange(4),
+                                        np.arange(4), np.arange(8), indexing="ij")
+    r, e = p & 3, p >> 2
+    n = 64 * nb + 16 * j + g + 8 * (r & 1)
+    gamma = c + 4 * (r >> 1)
+    Gamma = 4 * (gamma % 2) + gamma // 2
+    T = 2 * (32 * kb + 8 * t + Gamma) + e
+    codes = Qc[T, n].astype(np.uint32)
+    words = np.zeros(codes.shape[:-1], dtype=np.uint32)
+    for pp in range(8):
+        words |= codes[..., pp] << np.uint32(4 * pp)
+    chunks = words.reshape(KB, NB, 512)
+    out = np.empty((KB * NB, 512), dtype=np.uint32)
+    out[_chunk_order(KB, NB).reshape(-1)] = chunks.reshape(KB * NB, 512)
+    return out.reshape(-1)
+
+
+def pack_sparse_meta(idx: np.ndarray, K: int) -> np.ndarray:
+    """Positions idx[K/2, N] (uint8, 0..3) -> packed uint32 metadata words (K*N/32)."""
+    N = idx.shape[1]
+    KB, NB = K // 128, N // 64
+    kb, nb, jh, g, c, jl, w, x = np.meshgrid(np.arange(KB), np.arange(NB), np.arange(2), np.arange(8), np.arange(4),
+                                             np.arange(2), np.arange(2), np.arange(8), indexing="ij")
+    j = 2 * jh + jl
+    t = c // 2 + 2 * w
+    n = 64 * nb + 16 * j + g + 8 * (x >> 2)
+    gamma = 4 * (c % 2) + (x & 3)
+    Gamma = 4 * (gamma % 2) + gamma // 2
+    G2 = 2 * (32 * kb + 8 * t + Gamma)
+    nib = idx[G2, n].astype(np.uint32) | (idx[G2 + 1, n].astype(np.uint32) << np.uint32(2))
+    words = np.zeros(nib.shape[:-1], dtype=np.uint32)
+    for xx in range(8):
+        words |= nib[..., xx] << np.uint32(4 * xx)
+    chunks = words.reshape(KB, NB, 256)  # order inside: [jh, g, c, jl, w] = ((jh*32 + lane)*4 + jl*2 + w)
+    out = np.empty((KB * NB, 256), dtype=np.uint32)
+    out[_chunk_order(KB, NB).reshape(-1)] = chunks.reshape(KB * NB, 256)
+    return out.reshape(-1)

@@ -148,13 +148,16 @@ int marlin_unpack(const void* w_packed, const void* s_packed, uint32_t* q_kpacke
   return err == cudaSuccess ? MARLIN_OK : MARLIN_ERR_CUDA;
 }
 
-int marlin_gemm(const void* A, const void* w_packed, const void* s_packed, void* C, int M, int K, int N,
-                int group_size, void* workspace, size_t workspace_bytes, marlin_stream stream) {
-  if (!A || !w_packed || !s_packed || !C || !workspace) return MARLIN_ERR_NULL;
+// Shared body of marlin_gemm and marlin_gemm_sparse24 (meta_packed == nullptr: dense).
+static int gemm_common(const void* A, const void* w_packed, const void* meta_packed, const void* s_packed, void* C, int M,
+                       int K, int N, int group_size, void* workspace, size_t workspace_bytes, marlin_stream stream,
+                       bool sparse24) {
+  if (!A || !w_packed || !s_packed || !C || !workspace || (sparse24 && !meta_packed)) return MARLIN_ERR_NULL;
   if (M < 1 || !shape_ok(K, N)) return MARLIN_ERR_SHAPE;
   int G = normalise_group(K, group_size);
   if (!G) return MARLIN_ERR_GROUP;
-  if (!aligned16(A) || !aligned16(w_packed) || !aligned16(s_packed) || !aligned16(C) || !aligned16(workspace))
+  if (!aligned16(A) || !aligned16(w_packed) || !aligned16(s_packed) || !aligned16(C) || !aligned16(workspace) ||
+      (sparse24 && !aligned16(meta_packed)))
     return MARLIN_ERR_ALIGN;
   if (workspace_bytes < marlin_workspace_bytes(M, K, N)) return MARLIN_ERR_WORKSPACE;
   DeviceInfo info;
@@ -166,12 +169,13 @@ int marlin_gemm(const void* A, const void* w_packed, const void* s_packed, void*
   int m0 = 0;
   while (m0 < M) {
     const int rem = M - m0;
-    const bool use_tc = rem >= tc_min_m() && tc_path_supported(rem < kTcMaxSlabM ? rem : kTcMaxSlabM, K, N);
+    const bool use_tc = !sparse24 && rem >= tc_min_m() && tc_path_supported(rem < kTcMaxSlabM ? rem : kTcMaxSlabM, K, N);
     const int m_slab = use_tc ? (rem < kTcMaxSlabM ? rem : kTcMaxSlabM) : (rem < kMaxSlabM ? rem : kMaxSlabM);
     GemmParams p;
     p.A = static_cast<const uint16_t*>(A) + (size_t)m0 * K;
     p.wq = static_cast<const uint8_t*>(w_packed);
     p.sq = static_cast<const uint8_t*>(s_packed);
+    p.meta = static_cast<const uint8_t*>(meta_packed);
     p.C = static_cast<uint16_t*>(C) + (size_t)m0 * N;
     p.M = m_slab;
     p.K = K;
@@ -193,17 +197,22 @@ int marlin_gemm(const void* A, const void* w_packed, const void* s_packed, void*
         return MARLIN_ERR_CUDA;
     } else {
       DensePlan plan;
-      if (!make_dense_plan(m_slab, K, N, info.sm_count, &plan)) return MARLIN_ERR_SHAPE;
+      if (!make_dense_plan(m_slab, K, N, info.sm_count, sparse24, &plan)) return MARLIN_ERR_SHAPE;
       p.ncols = plan.ncols;
       p.units = (uint32_t)plan.units;
       p.workers = (uint32_t)plan.workers;
       p.stages = plan.stages;
       p.stage_bytes = plan.stage_bytes;
-      if (launch_gemm_dense(plan, p, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MARLIN_ERR_CUDA;
+      if (launch_gemm_dense(plan, p, sparse24, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MARLIN_ERR_CUDA;
     }
     m0 += m_slab;
   }
   return MARLIN_OK;
+}
+
+int marlin_gemm(const void* A, const void* w_packed, const void* s_packed, void* C, int M, int K, int N,
+                int group_size, void* workspace, size_t workspace_bytes, marlin_stream stream) {
+  return gemm_common(A, w_packed, nullptr, s_packed, C, M, K, N, group_size, workspace, workspace_bytes, stream, false);
 }
 
 // ---- the variant with a built-in workspace ------------------------------------------------------
@@ -234,17 +243,43 @@ int marlin_gemm_static_ws(const void* A, const void* w_packed, const void* s_pac
   return marlin_gemm(A, w_packed, s_packed, C, M, K, N, group_size, ws, kStaticWsBytes, stream);
 }
 
-int marlin_pack_sparse24(const uint32_t*, const uint8_t*, const void*, void*, void*, void*, int, int, int,
-                         marlin_stream) {
-  return MARLIN_ERR_SHAPE;  // filled in by gemm_sparse24.cu once that kernel exists
+int marlin_pack_sparse24(const uint32_t* qc_kpacked, const uint8_t* idx, const void* scales, void* w_packed,
+                         void* meta_packed, void* s_packed, int K, int N, int group_size, marlin_stream stream) {
+  if (!qc_kpacked || !idx || !scales || !w_packed || !meta_packed || !s_packed) return MARLIN_ERR_NULL;
+  if (!shape_ok(K, N)) return MARLIN_ERR_SHAPE;
+  int G = normalise_group(K, group_size);
+  if (!G) return MARLIN_ERR_GROUP;
+  if (!aligned16(qc_kpacked) || !aligned16(idx) || !aligned16(scales) || !aligned16(w_packed) ||
+      !aligned16(meta_packed) || !aligned16(s_packed))
+    return MARLIN_ERR_ALIGN;
+  cudaError_t err = launch_pack_sparse24(
+      const_cast<uint32_t*>(qc_kpacked), const_cast<uint8_t*>(idx), static_cast<uint16_t*>(const_cast<void*>(scales)),
+      static_cast<uint32_t*>(w_packed), static_cast<uint32_t*>(meta_packed), static_cast<uint16_t*>(s_packed), K, N, G,
+      false, static_cast<cudaStream_t>(stream));
+  return err == cudaSuccess ? MARLIN_OK : MARLIN_ERR_CUDA;
 }
-int marlin_unpack_sparse24(const void*, const void*, const void*, uint32_t*, uint8_t*, void*, int, int, int,
-                           marlin_stream) {
-  return MARLIN_ERR_SHAPE;
+
+int marlin_unpack_sparse24(const void* w_packed, const void* meta_packed, const void* s_packed, uint32_t* qc_kpacked,
+                           uint8_t* idx, void* scales, int K, int N, int group_size, marlin_stream stream) {
+  if (!qc_kpacked || !idx || !scales || !w_packed || !meta_packed || !s_packed) return MARLIN_ERR_NULL;
+  if (!shape_ok(K, N)) return MARLIN_ERR_SHAPE;
+  int G = normalise_group(K, group_size);
+  if (!G) return MARLIN_ERR_GROUP;
+  if (!aligned16(qc_kpacked) || !aligned16(idx) || !aligned16(scales) || !aligned16(w_packed) ||
+      !aligned16(meta_packed) || !aligned16(s_packed))
+    return MARLIN_ERR_ALIGN;
+  cudaError_t err = launch_pack_sparse24(
+      qc_kpacked, idx, static_cast<uint16_t*>(scales), static_cast<uint32_t*>(const_cast<void*>(w_packed)),
+      static_cast<uint32_t*>(const_cast<void*>(meta_packed)), static_cast<uint16_t*>(const_cast<void*>(s_packed)), K, N,
+      G, true, static_cast<cudaStream_t>(stream));
+  return err == cudaSuccess ? MARLIN_OK : MARLIN_ERR_CUDA;
 }
-int marlin_gemm_sparse24(const void*, const void*, const void*, const void*, void*, int, int, int, int, void*, size_t,
-                         marlin_stream) {
-  return MARLIN_ERR_SHAPE;
+
+int marlin_gemm_sparse24(const void* A, const void* w_packed, const void* meta_packed, const void* s_packed, void* C,
+                         int M, int K, int N, int group_size, void* workspace, size_t workspace_bytes,
+                         marlin_stream stream) {
+  return gemm_common(A, w_packed, meta_packed, s_packed, C, M, K, N, group_size, workspace, workspace_bytes, stream,
+                     true);
 }
 
 int marlin_read_status(const void* workspace, marlin_stream stream) {
@@ -263,7 +298,7 @@ int marlin_plan_stripes(int M, int K, int N, int sm_count, int* n_tile, int* wor
   if (M < 1 || !shape_ok(K, N)) return MARLIN_ERR_SHAPE;
   DensePlan plan;
   const int m_slab = M < kMaxSlabM ? M : kMaxSlabM;
-  if (!make_dense_plan(m_slab, K, N, sm_count, &plan)) return MARLIN_ERR_SHAPE;
+  if (!make_dense_plan(m_slab, K, N, sm_count, false, &plan)) return MARLIN_ERR_SHAPE;
   if (cap < plan.workers + 1) return MARLIN_ERR_SHAPE;
   *n_tile = plan.nw * kChunkN;
   *workers = plan.workers;

@@ -142,6 +142,19 @@ __device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4],
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+// 2:4 sparse MMA: A = 16 x 32 with 16 stored values per row (the usual 16 x 16 A fragment), B = 32 x 8,
+// E = metadata word of the lanes the selector names (lane % 4 in {0, 1} for selector 0, {2, 3} for 1):
+// nibble x of that lane's word = positions (first | second << 2) of the two kept values of row
+// g + 8*(x / 4) in group 4*(lane % 2) + x % 4 of four consecutive rows of B.  (Layout confirmed on B200
+// with one-hot probes.)
+template <int SEL>
+__device__ __forceinline__ void mma_sp_16832(float (&d)[4], const uint32_t (&a)[4], const uint32_t (&b)[4], uint32_t e) {
+  asm("mma.sp::ordered_metadata.sync.aligned.m16n8k32.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
+      "{%8,%9,%10,%11}, {%0,%1,%2,%3}, %12, %13;"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]), "r"(b[2]), "r"(b[3]), "r"(e), "n"(SEL));
+}
+
 // Register re-allocation between warpgroups (all four warps of a warpgroup execute it together).
 template <int N>
 __device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }

@@ -55,15 +55,18 @@ constexpr int kBarBytes = 1024;  // full[32] at 0, empty[32] at 256, flags at 51
 // raised "unspecified launch failure" on long-K layers, was no faster, and is not built.
 constexpr int consumer_warps_for(int /*mb*/) { return 8; }
 
-template <int MB, int NW, int CW>
+template <int MB, int NW, int CW, bool SP>
 struct Geometry {
   static constexpr int SK = CW / NW;             // groups of warps that split K
   static constexpr int MPAD = MB * 8;
   static constexpr int NT = NW * kChunkN;
   static constexpr int A_HALF_BYTES = MPAD * 128;            // one 64-wide half of the A tile: MPAD rows x 128 B
   static constexpr int A_BYTES = 2 * A_HALF_BYTES;
-  static constexpr int W_BYTES = NW * kChunkBytes;
-  static constexpr int STAGE_BYTES = A_BYTES + W_BYTES;      // multiple of 1024
+  static constexpr int CODE_CHUNK = SP ? kSparseCodeChunkBytes : kChunkBytes;  // packed codes of one 64-column chunk
+  static constexpr int META_CHUNK = SP ? kSparseMetaChunkBytes : 0;            // 2:4 position metadata of one chunk
+  static constexpr int W_BYTES = NW * CODE_CHUNK;
+  static constexpr int META_BYTES = NW * META_CHUNK;
+  static constexpr int STAGE_BYTES = A_BYTES + W_BYTES + META_BYTES;  // multiple of 1024
   static constexpr int FRAG_F4 = MB * 4;                     // float4 accumulator registers per thread
   static constexpr int TILE_F4 = NW * FRAG_F4 * 32;          // float4s of one partial tile
   static constexpr int RED_BYTES = (SK / 2) * TILE_F4 * 16;
@@ -76,10 +79,10 @@ struct Geometry {
 // ---------------------------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------------------------
-template <int MB, int NW, int CW>
+template <int MB, int NW, int CW, bool SP>
 __global__ void __launch_bounds__((CW + 4) * 32, 1)
 gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a) {
-  using G = Geometry<MB, NW, CW>;
+  using G = Geometry<MB, NW, CW, SP>;
   constexpr int SK = G::SK;
   constexpr int kConsumerWarps = CW;
   constexpr int kConsumerThreads = CW * 32;
@@ -127,13 +130,19 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
     if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
     const uint64_t pol_w = policy_evict_first();
     const uint64_t pol_a = policy_evict_last();
-    constexpr uint32_t tx_bytes = G::W_BYTES + G::A_BYTES;  // out-of-range rows of the box count too
+    constexpr uint32_t tx_bytes = G::W_BYTES + G::META_BYTES + G::A_BYTES;  // out-of-range rows of the box count too
     const uint32_t nb64 = p.N / kChunkN;
     // weights of (kb, col): super-columns of four chunks, k-blocks contiguous inside a super-column
-    auto weight_src = [&](uint32_t col, uint32_t kb) -> const uint8_t* {
+    auto chunk_index = [&](uint32_t col, uint32_t kb) -> size_t {
       const uint32_t nb = col * NW;
       const uint32_t sc = nb >> 2, cs = min(4u, nb64 - 4u * sc);
-      return p.wq + ((size_t)sc * 4u * KB + (size_t)kb * cs + (nb & 3u)) * kChunkBytes;
+      return (size_t)sc * 4u * KB + (size_t)kb * cs + (nb & 3u);
+    };
+    auto weight_src = [&](uint32_t col, uint32_t kb) -> const uint8_t* {
+      return p.wq + chunk_index(col, kb) * G::CODE_CHUNK;
+    };
+    auto meta_src = [&](uint32_t col, uint32_t kb) -> const uint8_t* {
+      return p.meta + chunk_index(col, kb) * G::META_CHUNK;
     };
     // First pass over the ring: the packed weights do not depend on the previous kernel of the
     // stream, so their copies go out before the dependency wait and HBM keeps streaming across the
@@ -145,6 +154,9 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
         const uint32_t col = u / KB, kb = u - col * KB;
         mbar_expect_tx(&full[s], tx_bytes);
         bulk_g2s(stage0 + (size_t)s * G::STAGE_BYTES + G::A_BYTES, weight_src(col, kb), G::W_BYTES, &full[s], pol_w);
+        if constexpr (SP)
+          bulk_g2s(stage0 + (size_t)s * G::STAGE_BYTES + G::A_BYTES + G::W_BYTES, meta_src(col, kb), G::META_BYTES,
+                   &full[s], pol_w);
       }
     }
     __syncwarp();
@@ -170,6 +182,7 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
       if (lane == 0) {
         mbar_expect_tx(&full[s], tx_bytes);
         bulk_g2s(st + G::A_BYTES, wsrc, G::W_BYTES, &full[s], pol_w);
+        if constexpr (SP) bulk_g2s(st + G::A_BYTES + G::W_BYTES, meta_src(col, kb), G::META_BYTES, &full[s], pol_w);
       }
       __syncwarp();
       if (lane < 2) tma_load_2d(st + lane * G::A_HALF_BYTES, &tmap_a, (int)(kb * kTileK + lane * 64), 0, &full[s], pol_a);
@@ -254,6 +267,53 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
       mbar_wait(&full[s], ph, abort_flag, p.status);
       if (warp == 0 && x == off && it0 == 0) MARLIN_STAMP(4);
       const uint8_t* st = stage0 + (size_t)s * G::STAGE_BYTES;
+      if constexpr (SP) {
+        // 2:4 path (Section 4): the kept codes are the A operand of mma.sp.m16n8k32, the 2-bit positions
+        // its metadata; one word of codes = one MMA, and the four 32-row steps of the k-block alternate the
+        // sparsity selector so that every lane supplies metadata for half of them.
+        const uint4* cp = reinterpret_cast<const uint4*>(st + G::A_BYTES + wn * G::CODE_CHUNK) + lane;
+        const uint4* mp = reinterpret_cast<const uint4*>(st + G::A_BYTES + G::W_BYTES + wn * G::META_CHUNK) + lane;
+        uint32_t Cw[4][4], Mw[4][2];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint4 v = cp[j * 32];
+          Cw[j][0] = v.x; Cw[j][1] = v.y; Cw[j][2] = v.z; Cw[j][3] = v.w;
+        }
+#pragma unroll
+        for (int jh = 0; jh < 2; ++jh) {
+          const uint4 v = mp[jh * 32];
+          Mw[2 * jh][0] = v.x; Mw[2 * jh][1] = v.y; Mw[2 * jh + 1][0] = v.z; Mw[2 * jh + 1][1] = v.w;
+        }
+        // this lane's activations of a 32-row step: four 4-byte words, 8 bytes apart, starting at
+        // 32*(c/2) + 4*(c%2) bytes inside the step's 64 bytes (the step's groups of four rows are
+        // permuted so that they are)
+        const uint32_t b_off = (uint32_t)(32 * (c >> 1) + 4 * (c & 1));
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          uint32_t bf[MB][4];
+#pragma unroll
+          for (int mb = 0; mb < MB; ++mb) {
+            const uint8_t* arow = st + (t >> 1) * G::A_HALF_BYTES + mb * 1024 + g * 128;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const uint32_t o = (uint32_t)(64 * (t & 1) + 8 * i) + b_off;
+              bf[mb][i] = *reinterpret_cast<const uint32_t*>(arow + ((((o >> 4) ^ (uint32_t)g) << 4) | (o & 15u)));
+            }
+          }
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            uint32_t a[4];
+            dequant8(Cw[j][t], a);
+#pragma unroll
+            for (int mb = 0; mb < MB; ++mb) {
+              if (t & 1)
+                mma_sp_16832<1>(tmp[j * MB + mb], a, bf[mb], Mw[j][t >> 1]);
+              else
+                mma_sp_16832<0>(tmp[j * MB + mb], a, bf[mb], Mw[j][t >> 1]);
+            }
+          }
+        }
+      } else {
       const uint4* wp = reinterpret_cast<const uint4*>(st + G::A_BYTES + wn * kChunkBytes) + lane;
       // codes of this lane: columns g (X) and g + 8 (Y) of each 16-column block j, its 32 rows of the k-block
       uint32_t X[4][4], Y[4][4];
@@ -292,6 +352,7 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
             }
           }
         }
+      }
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty[s]);
@@ -464,10 +525,10 @@ bool make_a_tensor_map(CUtensorMap* map, const void* A, int M, int K, int mpad) 
 
 namespace {
 
-template <int MB, int NW>
+template <int MB, int NW, bool SP>
 cudaError_t launch_one(const DensePlan& plan, const GemmParams& p, cudaStream_t stream) {
   constexpr int CW = consumer_warps_for(MB);
-  auto kernel = gemm_dense_kernel<MB, NW, CW>;
+  auto kernel = gemm_dense_kernel<MB, NW, CW, SP>;
   static bool attr_set[64] = {};  // per device
   int dev = 0;
   cudaError_t err = cudaGetDevice(&dev);
@@ -492,9 +553,9 @@ cudaError_t launch_one(const DensePlan& plan, const GemmParams& p, cudaStream_t 
   return cudaLaunchKernelEx(&cfg, kernel, p, tmap);
 }
 
-template <int MB, int NW>
+template <int MB, int NW, bool SP>
 void fill_geometry(DensePlan* plan) {
-  using G = Geometry<MB, NW, consumer_warps_for(MB)>;
+  using G = Geometry<MB, NW, consumer_warps_for(MB), SP>;
   plan->stage_bytes = G::STAGE_BYTES;
   int stages = (kSmemBudget - G::FIXED_BYTES - G::ALIGN_SLACK) / G::STAGE_BYTES;
   if (stages > kMaxStages) stages = kMaxStages;
@@ -514,7 +575,7 @@ extern "C" __attribute__((visibility("default"))) int marlin_timing_read(void* h
 #define MARLIN_DISPATCH(MBV, NWV, STMT)         \
   if (plan_mb == MBV && plan_nw == NWV) { STMT; }
 
-bool make_dense_plan(int m_slab, int K, int N, int sm_count, DensePlan* plan) {
+bool make_dense_plan(int m_slab, int K, int N, int sm_count, bool sparse24, DensePlan* plan) {
   if (m_slab < 1 || m_slab > kMaxSlabM || K < kTileK || K % kTileK || N < kChunkN || N % kChunkN) return false;
   if (sm_count < 1) return false;
   int mb = m_slab <= 8 ? 1 : (m_slab <= 16 ? 2 : 4);
@@ -531,29 +592,29 @@ bool make_dense_plan(int m_slab, int K, int N, int sm_count, DensePlan* plan) {
   if (workers > plan->units) workers = plan->units;
   plan->workers = (int)workers;
   const int plan_mb = mb, plan_nw = nw;
-  MARLIN_DISPATCH(1, 1, (fill_geometry<1, 1>(plan)))
-  MARLIN_DISPATCH(1, 2, (fill_geometry<1, 2>(plan)))
-  MARLIN_DISPATCH(1, 4, (fill_geometry<1, 4>(plan)))
-  MARLIN_DISPATCH(2, 1, (fill_geometry<2, 1>(plan)))
-  MARLIN_DISPATCH(2, 2, (fill_geometry<2, 2>(plan)))
-  MARLIN_DISPATCH(2, 4, (fill_geometry<2, 4>(plan)))
-  MARLIN_DISPATCH(4, 1, (fill_geometry<4, 1>(plan)))
-  MARLIN_DISPATCH(4, 2, (fill_geometry<4, 2>(plan)))
-  MARLIN_DISPATCH(4, 4, (fill_geometry<4, 4>(plan)))
+  MARLIN_DISPATCH(1, 1, (sparse24 ? fill_geometry<1, 1, true>(plan) : fill_geometry<1, 1, false>(plan)))
+  MARLIN_DISPATCH(1, 2, (sparse24 ? fill_geometry<1, 2, true>(plan) : fill_geometry<1, 2, false>(plan)))
+  MARLIN_DISPATCH(1, 4, (sparse24 ? fill_geometry<1, 4, true>(plan) : fill_geometry<1, 4, false>(plan)))
+  MARLIN_DISPATCH(2, 1, (sparse24 ? fill_geometry<2, 1, true>(plan) : fill_geometry<2, 1, false>(plan)))
+  MARLIN_DISPATCH(2, 2, (sparse24 ? fill_geometry<2, 2, true>(plan) : fill_geometry<2, 2, false>(plan)))
+  MARLIN_DISPATCH(2, 4, (sparse24 ? fill_geometry<2, 4, true>(plan) : fill_geometry<2, 4, false>(plan)))
+  MARLIN_DISPATCH(4, 1, (sparse24 ? fill_geometry<4, 1, true>(plan) : fill_geometry<4, 1, false>(plan)))
+  MARLIN_DISPATCH(4, 2, (sparse24 ? fill_geometry<4, 2, true>(plan) : fill_geometry<4, 2, false>(plan)))
+  MARLIN_DISPATCH(4, 4, (sparse24 ? fill_geometry<4, 4, true>(plan) : fill_geometry<4, 4, false>(plan)))
   return plan->stages >= consumer_warps_for(mb) / nw && plan->stages >= kProducerWarps;
 }
 
-cudaError_t launch_gemm_dense(const DensePlan& plan, const GemmParams& p, cudaStream_t stream) {
+cudaError_t launch_gemm_dense(const DensePlan& plan, const GemmParams& p, bool sparse24, cudaStream_t stream) {
   const int plan_mb = plan.mb, plan_nw = plan.nw;
-  MARLIN_DISPATCH(1, 1, return (launch_one<1, 1>(plan, p, stream)))
-  MARLIN_DISPATCH(1, 2, return (launch_one<1, 2>(plan, p, stream)))
-  MARLIN_DISPATCH(1, 4, return (launch_one<1, 4>(plan, p, stream)))
-  MARLIN_DISPATCH(2, 1, return (launch_one<2, 1>(plan, p, stream)))
-  MARLIN_DISPATCH(2, 2, return (launch_one<2, 2>(plan, p, stream)))
-  MARLIN_DISPATCH(2, 4, return (launch_one<2, 4>(plan, p, stream)))
-  MARLIN_DISPATCH(4, 1, return (launch_one<4, 1>(plan, p, stream)))
-  MARLIN_DISPATCH(4, 2, return (launch_one<4, 2>(plan, p, stream)))
-  MARLIN_DISPATCH(4, 4, return (launch_one<4, 4>(plan, p, stream)))
+  MARLIN_DISPATCH(1, 1, return (sparse24 ? launch_one<1, 1, true>(plan, p, stream) : launch_one<1, 1, false>(plan, p, stream)))
+  MARLIN_DISPATCH(1, 2, return (sparse24 ? launch_one<1, 2, true>(plan, p, stream) : launch_one<1, 2, false>(plan, p, stream)))
+  MARLIN_DISPATCH(1, 4, return (sparse24 ? launch_one<1, 4, true>(plan, p, stream) : launch_one<1, 4, false>(plan, p, stream)))
+  MARLIN_DISPATCH(2, 1, return (sparse24 ? launch_one<2, 1, true>(plan, p, stream) : launch_one<2, 1, false>(plan, p, stream)))
+  MARLIN_DISPATCH(2, 2, return (sparse24 ? launch_one<2, 2, true>(plan, p, stream) : launch_one<2, 2, false>(plan, p, stream)))
+  MARLIN_DISPATCH(2, 4, return (sparse24 ? launch_one<2, 4, true>(plan, p, stream) : launch_one<2, 4, false>(plan, p, stream)))
+  MARLIN_DISPATCH(4, 1, return (sparse24 ? launch_one<4, 1, true>(plan, p, stream) : launch_one<4, 1, false>(plan, p, stream)))
+  MARLIN_DISPATCH(4, 2, return (sparse24 ? launch_one<4, 2, true>(plan, p, stream) : launch_one<4, 2, false>(plan, p, stream)))
+  MARLIN_DISPATCH(4, 4, return (sparse24 ? launch_one<4, 4, true>(plan, p, stream) : launch_one<4, 4, false>(plan, p, stream)))
   return cudaErrorInvalidValue;
 }
 

@@ -17,6 +17,8 @@ namespace marlin_b200 {
 constexpr int kTileK = 128;           // rows of W per k-block
 constexpr int kChunkN = 64;           // columns of W per chunk
 constexpr int kChunkBytes = 4096;     // dense chunk
+constexpr int kSparseCodeChunkBytes = 2048;  // 2:4 chunk: 64 kept codes per column
+constexpr int kSparseMetaChunkBytes = 1024;  // 2:4 chunk: 2-bit positions of the kept codes
 constexpr int kProducerWarps = 4;     // the warps of the third warpgroup that issue copies
 // The last warpgroup of a CTA issues the copies; it shrinks to kProducerRegs registers per thread
 // (setmaxnreg) and the consumer warpgroups share what that frees.
@@ -48,12 +50,13 @@ struct DensePlan {
 
 // Chooses tile width, worker count and pipeline depth for one slab of m_slab <= 32 rows.
 // Pure host arithmetic.  Returns false on an unsupported shape.
-bool make_dense_plan(int m_slab, int K, int N, int sm_count, DensePlan* plan);
+bool make_dense_plan(int m_slab, int K, int N, int sm_count, bool sparse24, DensePlan* plan);
 
 struct GemmParams {
   const uint16_t* A;
   const uint8_t* wq;
   const uint8_t* sq;
+  const uint8_t* meta;   // 2:4 variant only
   uint16_t* C;
   int M, K, N;
   uint32_t kb;       // K / 128
@@ -72,7 +75,9 @@ struct GemmParams {
   int slot_floats;   // floats per partial-tile slot
 };
 
-cudaError_t launch_gemm_dense(const DensePlan& plan, const GemmParams& p, cudaStream_t stream);
+cudaError_t launch_gemm_dense(const DensePlan& plan, const GemmParams& p, bool sparse24, cudaStream_t stream);
+cudaError_t launch_pack_sparse24(uint32_t* qc, uint8_t* idx, uint16_t* s, uint32_t* wq, uint32_t* meta, uint16_t* sq, int K,
+                                 int N, int G, bool inverse, cudaStream_t stream);
 
 // tcgen05 kernel (gemm_dense_tc.cu): 256-column tiles, up to 128 rows of A per launch.
 bool tc_path_supported(int m_slab, int K, int N);

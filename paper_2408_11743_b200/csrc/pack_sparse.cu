@@ -1,0 +1,177 @@
+// Offline re-layout of the 2:4 sparse W4A16 weights: kept codes, 2-bit position metadata and scales
+// (Section 4, "Quantized non-zero values" and "Metadata indices": both structures are reshuffled once so
+// that every thread's loads are contiguous and the metadata lands in the lanes the sparse MMA reads).
+//
+// Per chunk (128 rows of the ORIGINAL K = 64 kept rows, 64 columns), ordered like the dense chunks
+// (super-columns of four):
+//   codes, 2048 bytes: 16-byte vector j*32 + lane (lane = 4g + c) holds words t = 0..3, one per 32-row
+//     step of the k-block = one mma.sp.m16n8k32; nibble p of a word (r = p % 4, e = p / 4) is kept value
+//     e (first or second) of
+//       column 64*nb + 16*j + g + 8*(r & 1)
+//       group  gamma = c + 4*(r >> 1) of the step's eight groups of four rows, where MMA group gamma
+//              stands for the actual group Gamma(gamma) = 4*(gamma % 2) + gamma / 2 of the step
+//     (the permutation of groups makes a lane's activations four words 8 bytes apart);
+//   metadata, 1024 bytes: 16-byte vector (j/2)*32 + lane, word (j % 2)*2 + w: the word lane (g, c)
+//     supplies for step t = c/2 + 2*w (selector t % 2): nibble x = positions (first | second << 2) of
+//     the kept values of column 64*nb + 16*j + g + 8*(x / 4) in MMA group 4*(c % 2) + x % 4.
+//   scales: as in the dense layout, one row per scale group of the original K.
+#include "marlin_internal.cuh"
+
+namespace marlin_b200 {
+namespace {
+
+__device__ __forceinline__ long long sp_chunk_index(int kb, int nb, int KB, int nb64) {
+  int sc = nb >> 2;
+  int cs = min(4, nb64 - 4 * sc);
+  return (long long)sc * 4 * KB + (long long)kb * cs + (nb & 3);
+}
+__device__ __forceinline__ void sp_chunk_coords(long long chunk, int KB, int nb64, int* kb, int* nb) {
+  long long full = (long long)(nb64 >> 2) * 4 * KB;
+  if (chunk < full) {
+    int sc = (int)(chunk / (4 * KB));
+    int rem = (int)(chunk % (4 * KB));
+    *kb = rem >> 2;
+    *nb = 4 * sc + (rem & 3);
+  } else {
+    int cs = nb64 & 3;
+    int rem = (int)(chunk - full);
+    *kb = rem / cs;
+    *nb = 4 * (nb64 >> 2) + rem % cs;
+  }
+}
+__device__ __forceinline__ int actual_group(int gamma) { return 4 * (gamma & 1) + (gamma >> 1); }
+__device__ __forceinline__ int mma_group(int Gamma) { return 2 * (Gamma & 3) + (Gamma >> 2); }
+
+// codes: one thread per packed word
+__global__ void pack_sparse_codes_kernel(const uint32_t* __restrict__ qc, uint32_t* __restrict__ wq, int K, int N) {
+  const long long total = (long long)K * N / 16;
+  const int KB = K / 128, nb64 = N / 64;
+  for (long long wi = blockIdx.x * (long long)blockDim.x + threadIdx.x; wi < total;
+       wi += (long long)gridDim.x * blockDim.x) {
+    int kb, nb;
+    sp_chunk_coords(wi >> 9, KB, nb64, &kb, &nb);
+    const int in = (int)(wi & 511);
+    const int t = in & 3, lane = (in >> 2) & 31, j = in >> 7;
+    const int g = lane >> 2, c = lane & 3;
+    uint32_t out = 0;
+#pragma unroll
+    for (int p = 0; p < 8; ++p) {
+      const int r = p & 3, e = p >> 2;
+      const int n = 64 * nb + 16 * j + g + 8 * (r & 1);
+      const int gamma = c + 4 * (r >> 1);
+      const int T = 2 * (32 * kb + 8 * t + actual_group(gamma)) + e;  // kept-value row
+      const uint32_t code = (qc[(size_t)(T >> 3) * N + n] >> (4 * (T & 7))) & 15u;
+      out |= code << (4 * p);
+    }
+    wq[wi] = out;
+  }
+}
+
+// metadata: one thread per packed word
+__global__ void pack_sparse_meta_kernel(const uint8_t* __restrict__ idx, uint32_t* __restrict__ meta, int K, int N) {
+  const long long total = (long long)K * N / 32;
+  const int KB = K / 128, nb64 = N / 64;
+  for (long long wi = blockIdx.x * (long long)blockDim.x + threadIdx.x; wi < total;
+       wi += (long long)gridDim.x * blockDim.x) {
+    int kb, nb;
+    sp_chunk_coords(wi >> 8, KB, nb64, &kb, &nb);
+    const int in = (int)(wi & 255);
+    const int q = in & 3, lane = (in >> 2) & 31, jh = in >> 7;
+    const int j = 2 * jh + (q >> 1), w = q & 1;
+    const int g = lane >> 2, c = lane & 3;
+    const int t = (c >> 1) + 2 * w;
+    uint32_t out = 0;
+#pragma unroll
+    for (int x = 0; x < 8; ++x) {
+      const int n = 64 * nb + 16 * j + g + 8 * (x >> 2);
+      const int gamma = 4 * (c & 1) + (x & 3);
+      const long long G2 = 2LL * (32 * kb + 8 * t + actual_group(gamma));
+      const uint32_t i0 = idx[(size_t)G2 * N + n] & 3u, i1 = idx[(size_t)(G2 + 1) * N + n] & 3u;
+      out |= (i0 | (i1 << 2)) << (4 * x);
+    }
+    meta[wi] = out;
+  }
+}
+
+// inverse: one thread per canonical word of kept codes
+__global__ void unpack_sparse_codes_kernel(const uint32_t* __restrict__ wq, uint32_t* __restrict__ qc, int K, int N) {
+  const long long total = (long long)K * N / 16;
+  const int KB = K / 128, nb64 = N / 64;
+  for (long long qi = blockIdx.x * (long long)blockDim.x + threadIdx.x; qi < total;
+       qi += (long long)gridDim.x * blockDim.x) {
+    const int n = (int)(qi % N);
+    const int T8 = (int)(qi / N);
+    const int nb = n >> 6, j = (n >> 4) & 3, row = n & 15, g = row & 7, rlo = row >> 3;
+    uint32_t out = 0;
+#pragma unroll
+    for (int jn = 0; jn < 8; ++jn) {
+      const int T = 8 * T8 + jn;
+      const int e = T & 1, Gabs = T >> 1;
+      const int kb = Gabs >> 5, t = (Gabs >> 3) & 3, gamma = mma_group(Gabs & 7);
+      const int c = gamma & 3, r = rlo + 2 * (gamma >> 2), p = r + 4 * e;
+      const long long wi = sp_chunk_index(kb, nb, KB, nb64) * 512 + (j * 32 + 4 * g + c) * 4 + t;
+      out |= ((wq[wi] >> (4 * p)) & 15u) << (4 * jn);
+    }
+    qc[qi] = out;
+  }
+}
+
+// inverse: one thread per (group of four original rows, column): writes the two position bytes
+__global__ void unpack_sparse_meta_kernel(const uint32_t* __restrict__ meta, uint8_t* __restrict__ idx, int K, int N) {
+  const long long total = (long long)(K / 4) * N;
+  const int KB = K / 128, nb64 = N / 64;
+  for (long long x0 = blockIdx.x * (long long)blockDim.x + threadIdx.x; x0 < total;
+       x0 += (long long)gridDim.x * blockDim.x) {
+    const int n = (int)(x0 % N);
+    const int Gabs = (int)(x0 / N);
+    const int nb = n >> 6, j = (n >> 4) & 3, row = n & 15, g = row & 7, rlo = row >> 3;
+    const int kb = Gabs >> 5, t = (Gabs >> 3) & 3, gamma = mma_group(Gabs & 7);
+    const int c = (gamma >> 2) + 2 * (t & 1), w = t >> 1;
+    const int x = (gamma & 3) + 4 * rlo;
+    const long long wi = sp_chunk_index(kb, nb, KB, nb64) * 256 + ((j >> 1) * 32 + 4 * g + c) * 4 + (j & 1) * 2 + w;
+    const uint32_t nib = (meta[wi] >> (4 * x)) & 15u;
+    idx[(size_t)(2LL * Gabs) * N + n] = (uint8_t)(nib & 3u);
+    idx[(size_t)(2LL * Gabs + 1) * N + n] = (uint8_t)(nib >> 2);
+  }
+}
+
+__global__ void permute_scales_sp_kernel(const uint16_t* __restrict__ in, uint16_t* __restrict__ out, long long total,
+                                         bool inverse) {
+  for (long long x = blockIdx.x * (long long)blockDim.x + threadIdx.x; x < total;
+       x += (long long)gridDim.x * blockDim.x) {
+    const long long base = x & ~63LL;
+    const int pos = (int)(x & 63);
+    const int g = pos >> 3, j = (pos >> 1) & 3, b = pos & 1;
+    const long long canon = base + 16 * j + 8 * b + g;
+    if (inverse)
+      out[canon] = in[x];
+    else
+      out[x] = in[canon];
+  }
+}
+
+int grid_for(long long items, int threads) {
+  long long b = (items + threads - 1) / threads;
+  return (int)(b > 148 * 16 ? 148 * 16 : (b < 1 ? 1 : b));
+}
+
+}  // namespace
+
+cudaError_t launch_pack_sparse24(uint32_t* qc, uint8_t* idx, uint16_t* s, uint32_t* wq, uint32_t* meta, uint16_t* sq, int K,
+                                 int N, int G, bool inverse, cudaStream_t stream) {
+  const int threads = 256;
+  const long long code_words = (long long)K * N / 16, meta_words = (long long)K * N / 32;
+  const long long ns = (long long)(K / G) * N;
+  if (!inverse) {
+    pack_sparse_codes_kernel<<<grid_for(code_words, threads), threads, 0, stream>>>(qc, wq, K, N);
+    pack_sparse_meta_kernel<<<grid_for(meta_words, threads), threads, 0, stream>>>(idx, meta, K, N);
+    permute_scales_sp_kernel<<<grid_for(ns, threads), threads, 0, stream>>>(s, sq, ns, false);
+  } else {
+    unpack_sparse_codes_kernel<<<grid_for(code_words, threads), threads, 0, stream>>>(wq, qc, K, N);
+    unpack_sparse_meta_kernel<<<grid_for((long long)(K / 4) * N, threads), threads, 0, stream>>>(meta, idx, K, N);
+    permute_scales_sp_kernel<<<grid_for(ns, threads), threads, 0, stream>>>(sq, s, ns, true);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace marlin_b200
