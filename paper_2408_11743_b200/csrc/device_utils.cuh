@@ -49,11 +49,15 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 // kernel through their normal control flow (no barrier is left unattended) and the host sees
 // MARLIN_ERR_DEVICE_TIMEOUT instead of a hang.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
+// BACKOFF_NS > 0: sleep between polls.  The copy-issuing warps use it: their waits are long and not urgent,
+// and a warp that polls flat out takes issue slots from the compute warps of its scheduler.
+template <int BACKOFF_NS = 0>
 __device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
   if (mbar_try_wait(bar, parity)) return;
   uint32_t spins = 0;
   uint64_t t0 = 0;
   while (!mbar_try_wait(bar, parity)) {
+    if (BACKOFF_NS > 0) __nanosleep(BACKOFF_NS);
     if ((++spins & 255u) == 0) {
       if (*abort_flag) return;
       uint64_t now = global_timer_ns();
@@ -153,6 +157,24 @@ __device__ __forceinline__ void mma_sp_16832(float (&d)[4], const uint32_t (&a)[
       "{%8,%9,%10,%11}, {%0,%1,%2,%3}, %12, %13;"
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]), "r"(b[2]), "r"(b[3]), "r"(e), "n"(SEL));
+}
+
+// Explicit shared-space loads from a 32-bit shared address (the stage ring is addressed through a pointer
+// that is re-aligned at run time, which can hide the address space from the compiler).
+__device__ __forceinline__ uint4 lds128(uint32_t saddr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(saddr));
+  return v;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t saddr) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(saddr));
+  return v;
+}
+__device__ __forceinline__ uint32_t lds16(uint32_t saddr) {
+  uint16_t v;
+  asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(saddr));
+  return v;
 }
 
 // Register re-allocation between warpgroups (all four warps of a warpgroup execute it together).

@@ -72,8 +72,13 @@ struct Geometry {
   static constexpr int RED_BYTES = (SK / 2) * TILE_F4 * 16;
   static constexpr int CST_STRIDE = NT + 8;                  // halves
   static constexpr int CST_BYTES = MPAD * CST_STRIDE * 2;
-  static constexpr int FIXED_BYTES = ((kBarBytes + RED_BYTES + CST_BYTES + 1023) / 1024) * 1024;
+  static constexpr int SC_BYTES = NT * 2;                    // group scales of one stage (one row of the tile)
+  static constexpr int SC_OFF = kBarBytes + RED_BYTES + CST_BYTES;
   static constexpr int ALIGN_SLACK = 1024;                   // the stage ring is placed on a 1024-byte boundary
+  // stages: what fits after the fixed areas, each stage bringing its scale row along
+  static constexpr int STAGES_FIT = (kSmemBudget - ALIGN_SLACK - SC_OFF - 1023) / (STAGE_BYTES + SC_BYTES);
+  static constexpr int STAGES = STAGES_FIT > kMaxStages ? kMaxStages : STAGES_FIT;
+  static constexpr int FIXED_BYTES = ((SC_OFF + STAGES * SC_BYTES + 1023) / 1024) * 1024;
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -98,7 +103,9 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
   volatile int* last_flag = abort_flag + 1;
   float4* red = reinterpret_cast<float4*>(smem + kBarBytes);
   uint16_t* cst = reinterpret_cast<uint16_t*>(smem + kBarBytes + G::RED_BYTES);
+  uint8_t* sc_ring = smem + G::SC_OFF;  // [stage][NT] fp16 group scales, copied with the stage
   uint8_t* stage0 = smem + G::FIXED_BYTES;
+  const uint32_t stage0_s = smem_u32(stage0);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -130,7 +137,12 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
     if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
     const uint64_t pol_w = policy_evict_first();
     const uint64_t pol_a = policy_evict_last();
-    constexpr uint32_t tx_bytes = G::W_BYTES + G::META_BYTES + G::A_BYTES;  // out-of-range rows of the box count too
+    // out-of-range rows of the A box count too; grouped layers bring the scale row of the k-block along
+    const uint32_t tx_bytes = G::W_BYTES + G::META_BYTES + G::A_BYTES + (p.grouped ? G::SC_BYTES : 0);
+    auto scale_src = [&](uint32_t col, uint32_t kb) -> const uint8_t* {
+      const uint32_t gi = p.group_shift >= 0 ? (kb >> p.group_shift) : (kb / (uint32_t)p.kb_per_group);
+      return p.sq + ((size_t)gi * p.N + (size_t)col * G::NT) * 2;
+    };
     const uint32_t nb64 = p.N / kChunkN;
     // weights of (kb, col): super-columns of four chunks, k-blocks contiguous inside a super-column
     auto chunk_index = [&](uint32_t col, uint32_t kb) -> size_t {
@@ -157,6 +169,7 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
         if constexpr (SP)
           bulk_g2s(stage0 + (size_t)s * G::STAGE_BYTES + G::A_BYTES + G::W_BYTES, meta_src(col, kb), G::META_BYTES,
                    &full[s], pol_w);
+        if (p.grouped) bulk_g2s(sc_ring + (size_t)s * G::SC_BYTES, scale_src(col, kb), G::SC_BYTES, &full[s], pol_w);
       }
     }
     __syncwarp();
@@ -177,12 +190,13 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
     for (; u < u1; u += kProducerWarps) {
       const uint32_t col = u / KB, kb = u - col * KB;
       const uint8_t* wsrc = weight_src(col, kb);
-      mbar_wait(&empty[s], ph ^ 1u, abort_flag, p.status);
+      mbar_wait<200>(&empty[s], ph ^ 1u, abort_flag, p.status);
       uint8_t* st = stage0 + (size_t)s * G::STAGE_BYTES;
       if (lane == 0) {
         mbar_expect_tx(&full[s], tx_bytes);
         bulk_g2s(st + G::A_BYTES, wsrc, G::W_BYTES, &full[s], pol_w);
         if constexpr (SP) bulk_g2s(st + G::A_BYTES + G::W_BYTES, meta_src(col, kb), G::META_BYTES, &full[s], pol_w);
+        if (p.grouped) bulk_g2s(sc_ring + (size_t)s * G::SC_BYTES, scale_src(col, kb), G::SC_BYTES, &full[s], pol_w);
       }
       __syncwarp();
       if (lane < 2) tma_load_2d(st + lane * G::A_HALF_BYTES, &tmap_a, (int)(kb * kTileK + lane * 64), 0, &full[s], pol_a);
@@ -256,32 +270,35 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
     const uint32_t off = (grp + SK - (it0 % SK)) % SK;
     for (uint32_t x = off; x < len; x += SK) {
       const uint32_t kb = kb0 + x;
+      mbar_wait(&full[s], ph, abort_flag, p.status);
       if (p.grouped) {
         const int gi = p.group_shift >= 0 ? (int)(kb >> p.group_shift) : (int)(kb / (uint32_t)p.kb_per_group);
         if (gi != cur_group) {
           if (cur_group >= 0) close_group();
-          cur_raw = __ldg(reinterpret_cast<const uint4*>(srow + (size_t)gi * p.N));  // used when the group closes
+          // the group's scales came with the stage (a read from global memory here would be a cold DRAM
+          // access whose latency every warp would wait out once per stage)
+          cur_raw = lds128(smem_u32(sc_ring) + (uint32_t)s * G::SC_BYTES + (uint32_t)(wn * 64 + g * 8) * 2);
           cur_group = gi;
         }
       }
-      mbar_wait(&full[s], ph, abort_flag, p.status);
       if (warp == 0 && x == off && it0 == 0) MARLIN_STAMP(4);
       const uint8_t* st = stage0 + (size_t)s * G::STAGE_BYTES;
+      const uint32_t st_s = stage0_s + (uint32_t)s * G::STAGE_BYTES;  // the same as a shared-space address
       if constexpr (SP) {
         // 2:4 path (Section 4): the kept codes are the A operand of mma.sp.m16n8k32, the 2-bit positions
         // its metadata; one word of codes = one MMA, and the four 32-row steps of the k-block alternate the
         // sparsity selector so that every lane supplies metadata for half of them.
-        const uint4* cp = reinterpret_cast<const uint4*>(st + G::A_BYTES + wn * G::CODE_CHUNK) + lane;
-        const uint4* mp = reinterpret_cast<const uint4*>(st + G::A_BYTES + G::W_BYTES + wn * G::META_CHUNK) + lane;
+        const uint32_t cp = st_s + G::A_BYTES + wn * G::CODE_CHUNK + lane * 16;
+        const uint32_t mp = st_s + G::A_BYTES + G::W_BYTES + wn * G::META_CHUNK + lane * 16;
         uint32_t Cw[4][4], Mw[4][2];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          const uint4 v = cp[j * 32];
+          const uint4 v = lds128(cp + j * 512);
           Cw[j][0] = v.x; Cw[j][1] = v.y; Cw[j][2] = v.z; Cw[j][3] = v.w;
         }
 #pragma unroll
         for (int jh = 0; jh < 2; ++jh) {
-          const uint4 v = mp[jh * 32];
+          const uint4 v = lds128(mp + jh * 512);
           Mw[2 * jh][0] = v.x; Mw[2 * jh][1] = v.y; Mw[2 * jh + 1][0] = v.z; Mw[2 * jh + 1][1] = v.w;
         }
         // this lane's activations of a 32-row step: four 4-byte words, 8 bytes apart, starting at
@@ -293,11 +310,11 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
           uint32_t bf[MB][4];
 #pragma unroll
           for (int mb = 0; mb < MB; ++mb) {
-            const uint8_t* arow = st + (t >> 1) * G::A_HALF_BYTES + mb * 1024 + g * 128;
+            const uint32_t arow = st_s + (t >> 1) * G::A_HALF_BYTES + mb * 1024 + g * 128;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
               const uint32_t o = (uint32_t)(64 * (t & 1) + 8 * i) + b_off;
-              bf[mb][i] = *reinterpret_cast<const uint32_t*>(arow + ((((o >> 4) ^ (uint32_t)g) << 4) | (o & 15u)));
+              bf[mb][i] = lds32(arow + ((((o >> 4) ^ (uint32_t)g) << 4) | (o & 15u)));
             }
           }
 #pragma unroll
@@ -314,13 +331,13 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
           }
         }
       } else {
-      const uint4* wp = reinterpret_cast<const uint4*>(st + G::A_BYTES + wn * kChunkBytes) + lane;
+      const uint32_t wp = st_s + G::A_BYTES + wn * G::CODE_CHUNK + lane * 16;
       // codes of this lane: columns g (X) and g + 8 (Y) of each 16-column block j, its 32 rows of the k-block
       uint32_t X[4][4], Y[4][4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const uint4 xv = wp[(2 * j) * 32];
-        const uint4 yv = wp[(2 * j + 1) * 32];
+        const uint4 xv = lds128(wp + (2 * j) * 512);
+        const uint4 yv = lds128(wp + (2 * j + 1) * 512);
         X[j][0] = xv.x; X[j][1] = xv.y; X[j][2] = xv.z; X[j][3] = xv.w;
         Y[j][0] = yv.x; Y[j][1] = yv.y; Y[j][2] = yv.z; Y[j][3] = yv.w;
       }
@@ -329,9 +346,9 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
         uint32_t bf[MB][8];
 #pragma unroll
         for (int mb = 0; mb < MB; ++mb) {
-          const uint8_t* arow = st + h * G::A_HALF_BYTES + mb * 1024;
-          const uint4 v0 = *reinterpret_cast<const uint4*>(arow + a_off0);
-          const uint4 v1 = *reinterpret_cast<const uint4*>(arow + a_off1);
+          const uint32_t arow = st_s + h * G::A_HALF_BYTES + mb * 1024;
+          const uint4 v0 = lds128(arow + a_off0);
+          const uint4 v1 = lds128(arow + a_off1);
           bf[mb][0] = v0.x; bf[mb][1] = v0.y; bf[mb][2] = v0.z; bf[mb][3] = v0.w;
           bf[mb][4] = v1.x; bf[mb][5] = v1.y; bf[mb][6] = v1.z; bf[mb][7] = v1.w;
         }
@@ -557,8 +574,7 @@ template <int MB, int NW, bool SP>
 void fill_geometry(DensePlan* plan) {
   using G = Geometry<MB, NW, consumer_warps_for(MB), SP>;
   plan->stage_bytes = G::STAGE_BYTES;
-  int stages = (kSmemBudget - G::FIXED_BYTES - G::ALIGN_SLACK) / G::STAGE_BYTES;
-  if (stages > kMaxStages) stages = kMaxStages;
+  int stages = G::STAGES;
   if (const char* e = getenv("MARLIN_B200_STAGES")) { int v = atoi(e); if (v >= 2 && v < stages) stages = v; }
   plan->stages = stages;
   plan->smem_bytes = G::FIXED_BYTES + G::ALIGN_SLACK + stages * G::STAGE_BYTES;

@@ -135,7 +135,8 @@ struct TcGeometry {
   static constexpr int A_BYTES = 2 * A_HALF_BYTES;
   static constexpr int W_BYTES = 4 * kChunkBytes;
   static constexpr int STAGE_BYTES = A_BYTES + W_BYTES;
-  static constexpr int FIXED_BYTES = 1024;
+  static constexpr int SC_BYTES = kTileN * 2;                       // group scales of one stage
+  static constexpr int FIXED_BYTES = 1024 + kTcMaxStages * SC_BYTES; // barriers + scale ring
   static constexpr int ALIGN_SLACK = 1024;
   static constexpr int STAGES =
       (kSmemBudget - FIXED_BYTES - ALIGN_SLACK) / STAGE_BYTES > kTcMaxStages
@@ -168,6 +169,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
   uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(smem + 208);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + 212);
   volatile int* last_flag = reinterpret_cast<volatile int*>(smem + 216);
+  uint8_t* sc_ring = smem + 1024;  // [stage][256] fp16 scales, copied with the stage
   uint8_t* stage0 = smem + G::FIXED_BYTES;
 
   const int warp = threadIdx.x >> 5;
@@ -211,7 +213,11 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
       const uint64_t pol_w = policy_evict_first();
       const uint64_t pol_a = policy_evict_last();
-      constexpr uint32_t tx_bytes = G::W_BYTES + G::A_BYTES;
+      const uint32_t tx_bytes = G::W_BYTES + G::A_BYTES + (p.grouped ? G::SC_BYTES : 0);
+      auto scale_src = [&](uint32_t col, uint32_t kb) -> const uint8_t* {
+        const uint32_t gi = p.group_shift >= 0 ? (kb >> p.group_shift) : (kb / (uint32_t)p.kb_per_group);
+        return p.sq + ((size_t)gi * p.N + (size_t)col * kTileN) * 2;
+      };
       // weights of (kb, col): the four chunks of a 256-column tile are adjacent, k-blocks follow one another
       auto weight_src = [&](uint32_t col, uint32_t kb) -> const uint8_t* {
         return p.wq + ((size_t)col * KB + kb) * (size_t)G::W_BYTES;
@@ -224,6 +230,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
           const uint32_t col = u / KB, kb = u - col * KB;
           mbar_expect_tx(&full[s], tx_bytes);
           bulk_g2s(stage0 + (size_t)s * G::STAGE_BYTES + G::A_BYTES, weight_src(col, kb), G::W_BYTES, &full[s], pol_w);
+          if (p.grouped) bulk_g2s(sc_ring + (size_t)s * G::SC_BYTES, scale_src(col, kb), G::SC_BYTES, &full[s], pol_w);
         }
       }
       __syncwarp();
@@ -242,11 +249,12 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       s -= NSTAGES;
       for (; u < u1; u += kTcProducerWarps) {
         const uint32_t col = u / KB, kb = u - col * KB;
-        mbar_wait(&empty[s], ph ^ 1u, abort_flag, p.status);
+        mbar_wait<200>(&empty[s], ph ^ 1u, abort_flag, p.status);
         uint8_t* st = stage0 + (size_t)s * G::STAGE_BYTES;
         if (lane == 0) {
           mbar_expect_tx(&full[s], tx_bytes);
           bulk_g2s(st + G::A_BYTES, weight_src(col, kb), G::W_BYTES, &full[s], pol_w);
+          if (p.grouped) bulk_g2s(sc_ring + (size_t)s * G::SC_BYTES, scale_src(col, kb), G::SC_BYTES, &full[s], pol_w);
         }
         __syncwarp();
         if (lane < 2)
@@ -332,26 +340,27 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
     const uint32_t len = min(KB - kb0, u1 - u);
     const uint16_t* sptr = reinterpret_cast<const uint16_t*>(p.sq) + (size_t)col * kTileN + spos;
 
-    int cur_group = -1;
-    uint32_t s2 = 0;  // {scale, scale} of the open group
+    uint32_t s2 = 0;  // {scale, scale} of this thread's column for the current k-block
+    if (!p.grouped) {
+      const uint32_t sv = __ldg(sptr);
+      s2 = sv | (sv << 16);
+    }
     for (uint32_t x = 0; x < len; ++x, ++it) {
-      const uint32_t kb = kb0 + x;
-      const int gi = p.grouped ? (p.group_shift >= 0 ? (int)(kb >> p.group_shift) : (int)(kb / (uint32_t)p.kb_per_group)) : 0;
-      if (gi != cur_group) {
-        const uint32_t sv = __ldg(sptr + (size_t)gi * p.N);
-        s2 = sv | (sv << 16);
-        cur_group = gi;
-      }
       const int s = (int)(it % NSTAGES);
       const int slot = (int)(it % NSLOTS);
       const bool tr = (warp == 0 && it == 6);
       if (tr) MARLIN_STAMP(12);
       mbar_wait(&full[s], (it / NSTAGES) & 1u, abort_flag, p.status);
       if (tr) MARLIN_STAMP(13);
-      const uint8_t* wbase = stage0 + (size_t)s * G::STAGE_BYTES + G::A_BYTES + vec_off;
+      if (p.grouped) {
+        // the scale row of the k-block came with the stage (a global read here would be a cold DRAM access)
+        const uint32_t sv = lds16(smem_u32(sc_ring) + (uint32_t)s * G::SC_BYTES + (uint32_t)spos * 2);
+        s2 = sv | (sv << 16);
+      }
+      const uint32_t wbase = smem_u32(stage0) + (uint32_t)s * G::STAGE_BYTES + G::A_BYTES + vec_off;
       uint4 v[4];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) v[c] = *reinterpret_cast<const uint4*>(wbase + c * 16);
+      for (int c = 0; c < 4; ++c) v[c] = lds128(wbase + c * 16);
       // the codes are in registers: the weight part of the stage is free as far as this warp is concerned
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty[s]);
