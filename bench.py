@@ -48,7 +48,14 @@ REFERENCE_SAMPLE_MS = (16,)   # one step of --impl reference
 
 
 def launches_for(M: int) -> int:
-    return (M + 31) // 32  # one kernel per slab of 32 rows
+    """Kernels one marlin_gemm call launches on this layer: the warp-MMA kernel up to 32 rows, the tcgen05
+    kernel (up to 128 rows per launch) above."""
+    return 1 if M <= 128 else (M + 127) // 128
+
+
+# DRAM bytes of one launch of the dominant kernel from the committed ncu capture
+# (profiles/gemm_dense_kernel_M16_K8192_N8192.md: dram__bytes_read.sum + dram__bytes_write.sum)
+NCU_DRAM_BYTES_PER_LAUNCH = 34.91e6
 
 
 # ------------------------------------------------------------------------------------------------
@@ -170,6 +177,79 @@ def run_reference(args):
 # ------------------------------------------------------------------------------------------------
 # GPU leg
 # ------------------------------------------------------------------------------------------------
+def extra_layers(marlin, dev, stream, l2, peaks, capture, time_graph):
+    """Per-layer numbers outside the timed step: Llama-2-7B shapes (dense) and the 8192^2 2:4 layer."""
+    import torch
+    out = []
+    rng = np.random.default_rng(1234)
+
+    def measure(K, N, G, M, sparse):
+        wb = roofline.weight_bytes(K, N, G, sparse24=sparse)
+        copies = max(2, int(np.ceil(2.0 * l2 / wb)) + 1)
+        S = torch.from_numpy(rng.uniform(0.005, 0.02, size=(K // G, N)).astype(np.float16)).to(dev)
+        if sparse:
+            qc = torch.from_numpy(rng.integers(-2**31, 2**31 - 1, size=(K // 16, N), dtype=np.int64).astype(np.int32)).to(dev)
+            pat = rng.integers(0, 6, size=(K // 4, N))
+            idx = np.empty((K // 2, N), dtype=np.uint8)
+            idx[0::2], idx[1::2] = inputs._KEEP_PATTERNS[pat, 0], inputs._KEEP_PATTERNS[pat, 1]
+            packed0 = marlin.pack_sparse24(qc, torch.from_numpy(idx).to(dev), S, G)
+        else:
+            q = torch.from_numpy(rng.integers(-2**31, 2**31 - 1, size=(K // 8, N), dtype=np.int64).astype(np.int32)).to(dev)
+            packed0 = marlin.pack(q, S, G)
+        packed = [tuple(t.clone() for t in packed0) for _ in range(copies)]
+        A = torch.from_numpy(rng.standard_normal((M, K), dtype=np.float32).astype(np.float16)).to(dev)
+        C = torch.empty((M, N), dtype=torch.float16, device=dev)
+        ws = marlin.new_workspace(M, K, N, device=dev)
+        rot = [0]
+
+        def call():
+            pk = packed[rot[0] % copies]
+            rot[0] += 1
+            if sparse:
+                marlin.gemm_sparse24(A, pk[0], pk[1], pk[2], K, N, G, ws, out=C, stream=stream)
+            else:
+                marlin.gemm(A, pk[0], pk[1], K, N, G, ws, out=C, stream=stream)
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                call()
+        torch.cuda.synchronize(dev)
+        reps = max(16, 2 * copies)
+        g = capture(call, reps)
+        time_graph(g)
+        t = min(time_graph(g) for _ in range(5)) / reps
+        W16 = [torch.randn((K, N), dtype=torch.float16, device=dev) * 0.05
+               for _ in range(max(2, int(np.ceil(2.0 * l2 / (2 * K * N))) + 1))]
+        o16 = torch.empty((M, N), dtype=torch.float16, device=dev)
+        r16 = [0]
+
+        def fp16():
+            torch.matmul(A, W16[r16[0] % len(W16)], out=o16)
+            r16[0] += 1
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                fp16()
+        torch.cuda.synchronize(dev)
+        g16 = capture(fp16, 2 * len(W16))
+        time_graph(g16)
+        t16 = min(time_graph(g16) for _ in range(5)) / (2 * len(W16))
+        troof = roofline.roofline_seconds(M, K, N, G, peaks, sparse24=sparse)
+        assert marlin.read_status(ws, stream=stream) == 0
+        return {"K": K, "N": N, "M": M, "sparse24": sparse, "us": round(t * 1e6, 3),
+                "weight_gbs": round(wb / t / 1e9, 1), "roofline_frac": round(troof / t, 4),
+                "cublas_fp16_us": round(t16 * 1e6, 3), "speedup_vs_fp16": round(t16 / t, 3)}
+
+    for name, K, N in inputs.LLAMA7B_LAYERS:
+        for M in (1, 16, 32):
+            r = measure(K, N, GROUP, M, False)
+            r["layer"] = "llama2-7b " + name
+            out.append(r)
+    for M in (16, 32, 64, 128):
+        r = measure(8192, 8192, GROUP, M, True)
+        r["layer"] = "2:4 sparse 8192x8192"
+        out.append(r)
+    return out
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -308,6 +388,11 @@ def run_ours(args):
             del g, g16
         del W16
 
+        # ---- context, not part of the step: Llama-2-7B-shaped layers and the 2:4 variant ----
+        extra = []
+        if not args.no_extra:
+            extra = extra_layers(marlin, dev, stream, l2, peaks, capture, time_graph)
+
         # ---- end to end: host buffers, copies inside the timed region ----
         A_host = {M: torch.from_numpy(get(M).A).pin_memory() for M in SWEEP}
         C_host = {M: torch.empty((M, N_DIM), dtype=torch.float16).pin_memory() for M in SWEEP}
@@ -351,11 +436,14 @@ def run_ours(args):
                        "timing": "CUDA graph of K steps between CUDA events on the launch stream",
                        "multi_gpu": "replicas only"},
             "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                         "frac": round(achieved / peaks["hbm_gbs"], 4), "traffic": None,
-                         "peak_source": peaks["source"], "kernel": "gemm_dense_kernel",
+                         "frac": round(achieved / peaks["hbm_gbs"], 4), "traffic": NCU_DRAM_BYTES_PER_LAUNCH,
+                         "traffic_note": "ncu capture of the M=16 launch; algorithmic bytes of that launch 35.1e6",
+                         "peak_source": peaks["source"],
+                         "kernel": "gemm_dense_kernel (M <= 32) and gemm_dense_tc_kernel (M = 64, 128)",
                          "per_launch_us": round(step_s * 1e6 / launches_per_step, 3),
                          "algorithmic_bytes_per_step": step_alg_bytes},
             "per_m": per_m,
+            "other_layers": extra,
             "cpu_baseline": {"value": round(cpu_v, 4), "unit": UNIT, "cores": cores, "kind": "oracle",
                              "sample": f"full layer at M in {list(CPU_SAMPLE_MS)} ({cpu_t:.1f} s)"},
             "e2e": {"value": round(world * step_wbytes / e2e_s / 1e9, 2), "unit": UNIT,
@@ -376,6 +464,7 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-extra", action="store_true", help="skip the Llama-shaped and 2:4 context measurements")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
