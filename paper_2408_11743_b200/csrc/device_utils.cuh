@@ -62,9 +62,17 @@ __device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, volati
       if (*abort_flag) return;
       uint64_t now = global_timer_ns();
       if (t0 == 0) t0 = now;
-      if (now - t0 > kWaitLimitNs) {
+      if (now > t0 && now - t0 > kWaitLimitNs) {
         *abort_flag = 1;
-        atomicExch(status, (int)MARLIN_ERR_DEVICE_TIMEOUT);
+        // the first wait that gives up leaves a record behind the status word: who waited, on what, how long
+        if (atomicCAS(status, 0, (int)MARLIN_ERR_DEVICE_TIMEOUT) == 0) {
+          status[1] = (int)blockIdx.x;
+          status[2] = (int)threadIdx.x;
+          status[3] = (int)(smem_u32(bar) & 1023u);
+          status[4] = (int)parity;
+          status[5] = (int)spins;
+          status[6] = (int)((now - t0) >> 10);
+        }
         return;
       }
     }

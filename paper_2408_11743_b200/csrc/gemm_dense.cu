@@ -122,7 +122,8 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
   }
   if (threadIdx.x == 0) {
     *abort_flag = 0;
-    *last_flag = 0;
+    last_flag[0] = 0;
+    last_flag[1] = 0;
   }
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   __syncthreads();
@@ -404,6 +405,69 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
     // ---- stripe fix-up across CTAs and output ----
     const int first_w = (int)stripe_owner32(col * KB, U, P);
     const int last_w = (int)stripe_owner32((col + 1) * KB - 1, U, P);
+    if (u + len < u1) {
+      // A segment in the middle of the stripe: group 0 holds the tile and finishes it alone (its L2 round
+      // trips take a microsecond or two); the other groups go on with the k-blocks of the next segment.
+      if (grp == 0) {
+        constexpr int kG0 = NW * 32;
+        if (last_w > first_w) {
+          const int my_slot = 2 * (int)worker + (col != u0 / KB ? 1 : 0);
+          float4* mine = reinterpret_cast<float4*>(p.partials + (size_t)my_slot * p.slot_floats) +
+                         (size_t)wn * G::FRAG_F4 * 32 + lane;
+#pragma unroll
+          for (int r = 0; r < 4 * MB; ++r) mine[r * 32] = make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
+          named_bar_sync(2, kG0);
+          if (ctid == 0) {
+            const int old = atom_add_acq_rel_gpu(&p.counters[col], 1);
+            const int is_last = (old == last_w - first_w) ? 1 : 0;
+            if (is_last) p.counters[col] = 0;
+            last_flag[1] = is_last;
+          }
+          named_bar_sync(2, kG0);
+          if (last_flag[1]) {
+            // every thread re-reads its own fragment positions of all partials, in stripe order
+            for (int w = first_w; w <= last_w; ++w) {
+              const int slot = 2 * w + (col != stripe_begin32(w, U, P) / KB ? 1 : 0);
+              const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)slot * p.slot_floats) +
+                                  (size_t)wn * G::FRAG_F4 * 32 + lane;
+#pragma unroll
+              for (int r = 0; r < 4 * MB; ++r) {
+                const float4 v = ld_cg_f4(src + r * 32);
+                if (w == first_w) {
+                  acc[r][0] = v.x; acc[r][1] = v.y; acc[r][2] = v.z; acc[r][3] = v.w;
+                } else {
+                  acc[r][0] += v.x; acc[r][1] += v.y; acc[r][2] += v.z; acc[r][3] += v.w;
+                }
+              }
+            }
+          }
+        }
+        if (last_w == first_w || last_flag[1]) {
+#pragma unroll
+          for (int r = 0; r < 4 * MB; ++r) {
+            const int j = r / MB, mb = r % MB;
+            const int n = wn * 64 + 16 * j + g;
+            const int m = mb * 8 + 2 * c;
+            cst[m * G::CST_STRIDE + n] = __half_as_ushort(__float2half_rn(acc[r][0]));
+            cst[(m + 1) * G::CST_STRIDE + n] = __half_as_ushort(__float2half_rn(acc[r][1]));
+            cst[m * G::CST_STRIDE + n + 8] = __half_as_ushort(__float2half_rn(acc[r][2]));
+            cst[(m + 1) * G::CST_STRIDE + n + 8] = __half_as_ushort(__float2half_rn(acc[r][3]));
+          }
+          named_bar_sync(2, kG0);
+          constexpr int CH = NW * 8;
+          for (int x = ctid; x < p.M * CH; x += kG0) {
+            const int m = x / CH, ch = x % CH;
+            const uint4 v = *reinterpret_cast<const uint4*>(cst + m * G::CST_STRIDE + ch * 8);
+            *reinterpret_cast<uint4*>(p.C + (size_t)m * p.N + (size_t)col * G::NT + ch * 8) = v;
+          }
+        }
+        named_bar_sync(2, kG0);  // cst and last_flag[1] are free again
+      }
+      u += len;
+      it0 += len;
+      continue;
+    }
+    // ---- the last segment of the stripe: all consumer threads take part ----
     bool tile_in_cst = false;
     if (last_w > first_w) {
       // this column tile is shared: publish the partial, count arrivals
@@ -507,6 +571,10 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
     if (warp == 0) MARLIN_STAMP(8);
   }
   if (warp == 0) MARLIN_STAMP(9);
+  if (*abort_flag) {
+    // a wait gave up: copies may still be in flight towards this CTA's shared memory
+    for (int x = 0; x < 1000; ++x) __nanosleep(1000);
+  }
 }
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point (no link against libcuda).
@@ -595,8 +663,9 @@ bool make_dense_plan(int m_slab, int K, int N, int sm_count, bool sparse24, Dens
   if (m_slab < 1 || m_slab > kMaxSlabM || K < kTileK || K % kTileK || N < kChunkN || N % kChunkN) return false;
   if (sm_count < 1) return false;
   int mb = m_slab <= 8 ? 1 : (m_slab <= 16 ? 2 : 4);
-  // wide column tiles keep the bulk copies large (16 KB) whatever the batch size
-  int nw = 4;
+  // 128-column tiles (8 KB copies): measured best for the warp-MMA kernel; narrower tiles mean fewer CTAs per
+  // column tile in the stripe fix-up, wider ones fewer and larger copies
+  int nw = 2;
   if (const char* e = getenv("MARLIN_B200_NW")) { int v = atoi(e); if (v == 1 || v == 2 || v == 4) nw = v; }
   while (nw > 1 && N % (kChunkN * nw)) nw >>= 1;
   plan->mb = mb;

@@ -111,7 +111,7 @@ __host__ __device__ constexpr uint32_t instr_desc_f16(int m, int n) {
 }
 
 #ifdef MARLIN_TIMING
-__device__ long long g_timing_tc[kMaxWorkers][16];
+__device__ long long g_timing_tc[kMaxWorkers][24];
 #define MARLIN_STAMP(slot) do { if (lane == 0) g_timing_tc[blockIdx.x][slot] = (long long)global_timer_ns(); } while (0)
 #else
 #define MARLIN_STAMP(slot) do { } while (0)
@@ -282,9 +282,11 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         for (uint32_t x = 0; x < len; ++x, ++it) {
           const int s = (int)(it % NSTAGES);
           const int slot = (int)(it % NSLOTS);
+          if (it == 6) MARLIN_STAMP(19);
           mbar_wait(&full[s], (it / NSTAGES) & 1u, abort_flag, p.status);
           mbar_wait(&afull[slot], (it / NSLOTS) & 1u, abort_flag, p.status);
           if (it == 0) MARLIN_STAMP(4);
+          if (it == 6) MARLIN_STAMP(16);
           tc_fence_after_sync();
           if (lane == 0) {
             // descriptor of the first K = 16 step of the stage; the others differ in the address field only
@@ -299,9 +301,11 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
                 tc_mma_ts(d_tmem, a_tmem + ks * 8, bdesc, idesc, (x == 0 && ks == 0) ? 0u : 1u);
               }
             }
+            if (it == 6) MARLIN_STAMP(17);
             tc_commit(&aempty[slot]);  // the A slot may be rewritten
             tc_commit(&empty[s]);      // the activation tile of the stage may be refilled
             if (x + 1 == len) tc_commit(dfull);
+            if (it == 6) MARLIN_STAMP(18);
           }
           __syncwarp();
         }

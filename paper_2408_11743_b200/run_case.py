@@ -75,7 +75,12 @@ def main():
         e1.record(s)
     e1.synchronize()
     t = e0.elapsed_time(e1) * 1e-3 / args.iters
-    assert marlin.read_status(ws) == 0
+    if marlin.read_status(ws) != 0:
+        # a bounded wait inside the kernel expired: the words behind the status word say which one
+        rec = ws[:32].cpu().view(torch.int32).tolist()
+        print(f"device status {rec[0]}: block {rec[1]} thread {rec[2]} barrier offset {rec[3]} parity {rec[4]} "
+              f"polls {rec[5]} waited {rec[6]} us")
+        sys.exit(2)
     wb = roofline.weight_bytes(K, N, case.G, sparse24=args.sparse)
     print(f"M={M} K={K} N={N} G={case.G} sparse={args.sparse}: {t * 1e6:.2f} us  "
           f"{wb / t / 1e9:.0f} GB/s weights  {roofline.flops(M, K, N) / t / 1e12:.1f} TFLOP/s")
