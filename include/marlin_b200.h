@@ -95,8 +95,11 @@ MARLIN_API int marlin_unpack(const void* w_packed, const void* s_packed, uint32_
  *   C          device, out, fp16 [M][N] row-major, every element written
  *   workspace  device, at least marlin_workspace_bytes(M, K, N) bytes, zeroed once by the caller
  * Accumulation is fp32 (also across stripes); the result is rounded once to fp16 (nearest even).
- * Results are deterministic: the same inputs give the same bits on every call.
- * M > 32 is processed as consecutive slabs of rows.
+ * Up to 16 rows the warp-level kernel runs and the same inputs give the same bits on every call.
+ * From 17 rows the tcgen05 kernel takes over (128 rows per launch, N a multiple of 256; otherwise the
+ * warp-level kernel runs on slabs of 16 rows): there the partial sums of a column tile shared by
+ * several CTAs are added in fp32 in arrival order, so the last bit of an fp16 result can differ between
+ * two calls.
  * Errors: argument checks return before anything is queued.  A kernel whose bounded waits expire
  * sets the workspace status word; read it with marlin_read_status. */
 MARLIN_API int marlin_gemm(const void* A, const void* w_packed, const void* s_packed, void* C,

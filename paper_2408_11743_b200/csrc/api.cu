@@ -60,7 +60,7 @@ int tc_min_m() {
   static int v = -1;
   if (v < 0) {
     const char* e = getenv("MARLIN_B200_TC_MIN_M");  // tuning knob; default below
-    v = e ? atoi(e) : 33;
+    v = e ? atoi(e) : 17;
     if (v < 1) v = 1;
   }
   return v;

@@ -1,4 +1,4 @@
-// Dense W4A16 layer for sm_100a, decode batch sizes (one launch handles up to 32 rows of A).
+// Dense W4A16 layer for sm_100a, decode batch sizes (one launch handles up to 16 rows of A).
 //
 // Structure of one CTA (one per SM, persistent over its stripe of work units):
 //   warp 8        producer: per k-block ONE bulk-async copy (cp.async.bulk + mbarrier complete_tx) of
@@ -52,7 +52,10 @@ __device__ long long g_timing[kMaxWorkers][16];
 constexpr int kBarBytes = 1024;  // full[32] at 0, empty[32] at 256, flags at 512
 
 // Consumer warps per CTA.  Eight everywhere: a sixteen-warp variant of the one-block kernel (batch <= 8)
-// raised "unspecified launch failure" on long-K layers, was no faster, and is not built.
+// raised "unspecified launch failure" on long-K layers, was no faster, and is not built.  The same goes
+// for a four-block variant (32 rows of A per launch, the only one whose accumulators spilled): it raised
+// that error in two of three timing runs on the 8192 x 8192 layer; batches above 16 rows go to the
+// tcgen05 kernel, or through this one as slabs of 16 rows where that kernel does not apply.
 constexpr int consumer_warps_for(int /*mb*/) { return 8; }
 
 template <int MB, int NW, int CW, bool SP>
@@ -662,7 +665,7 @@ extern "C" __attribute__((visibility("default"))) int marlin_timing_read(void* h
 bool make_dense_plan(int m_slab, int K, int N, int sm_count, bool sparse24, DensePlan* plan) {
   if (m_slab < 1 || m_slab > kMaxSlabM || K < kTileK || K % kTileK || N < kChunkN || N % kChunkN) return false;
   if (sm_count < 1) return false;
-  int mb = m_slab <= 8 ? 1 : (m_slab <= 16 ? 2 : 4);
+  int mb = m_slab <= 8 ? 1 : 2;
   // 128-column tiles (8 KB copies): measured best for the warp-MMA kernel; narrower tiles mean fewer CTAs per
   // column tile in the stripe fix-up, wider ones fewer and larger copies
   int nw = 2;
@@ -683,9 +686,6 @@ bool make_dense_plan(int m_slab, int K, int N, int sm_count, bool sparse24, Dens
   MARLIN_DISPATCH(2, 1, (sparse24 ? fill_geometry<2, 1, true>(plan) : fill_geometry<2, 1, false>(plan)))
   MARLIN_DISPATCH(2, 2, (sparse24 ? fill_geometry<2, 2, true>(plan) : fill_geometry<2, 2, false>(plan)))
   MARLIN_DISPATCH(2, 4, (sparse24 ? fill_geometry<2, 4, true>(plan) : fill_geometry<2, 4, false>(plan)))
-  MARLIN_DISPATCH(4, 1, (sparse24 ? fill_geometry<4, 1, true>(plan) : fill_geometry<4, 1, false>(plan)))
-  MARLIN_DISPATCH(4, 2, (sparse24 ? fill_geometry<4, 2, true>(plan) : fill_geometry<4, 2, false>(plan)))
-  MARLIN_DISPATCH(4, 4, (sparse24 ? fill_geometry<4, 4, true>(plan) : fill_geometry<4, 4, false>(plan)))
   return plan->stages >= consumer_warps_for(mb) / nw && plan->stages >= kProducerWarps;
 }
 
@@ -697,9 +697,6 @@ cudaError_t launch_gemm_dense(const DensePlan& plan, const GemmParams& p, bool s
   MARLIN_DISPATCH(2, 1, return (sparse24 ? launch_one<2, 1, true>(plan, p, stream) : launch_one<2, 1, false>(plan, p, stream)))
   MARLIN_DISPATCH(2, 2, return (sparse24 ? launch_one<2, 2, true>(plan, p, stream) : launch_one<2, 2, false>(plan, p, stream)))
   MARLIN_DISPATCH(2, 4, return (sparse24 ? launch_one<2, 4, true>(plan, p, stream) : launch_one<2, 4, false>(plan, p, stream)))
-  MARLIN_DISPATCH(4, 1, return (sparse24 ? launch_one<4, 1, true>(plan, p, stream) : launch_one<4, 1, false>(plan, p, stream)))
-  MARLIN_DISPATCH(4, 2, return (sparse24 ? launch_one<4, 2, true>(plan, p, stream) : launch_one<4, 2, false>(plan, p, stream)))
-  MARLIN_DISPATCH(4, 4, return (sparse24 ? launch_one<4, 4, true>(plan, p, stream) : launch_one<4, 4, false>(plan, p, stream)))
   return cudaErrorInvalidValue;
 }
 

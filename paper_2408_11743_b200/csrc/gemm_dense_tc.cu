@@ -124,7 +124,8 @@ constexpr int kTcThreads = 384;
 constexpr int kDequantWarps = 8;
 constexpr int kDequantThreads = kDequantWarps * 32;
 constexpr int kTcProducerWarps = 2;
-constexpr int kMmaWarp = 10;
+constexpr int kMmaWarp = 10;        // first of the MMA-issuing warps (it also owns the TMEM allocation)
+constexpr int kMmaWarps = 2;        // one per 128-channel tile: issuing a tcgen05.mma occupies the thread for tens of cycles
 constexpr int kTcMaxStages = 8;
 constexpr int kTileN = 256;          // columns of W per CTA tile: two UMMA tiles of 128 channels
 constexpr int kTmemCols = 512;
@@ -183,13 +184,13 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
   if (threadIdx.x == 0) {
     for (int s = 0; s < NSTAGES; ++s) {
       mbar_init(&full[s], 1);
-      mbar_init(&empty[s], kDequantWarps + 1);
+      mbar_init(&empty[s], kDequantWarps + kMmaWarps);
     }
     for (int a = 0; a < NSLOTS; ++a) {
       mbar_init(&afull[a], kDequantWarps);
-      mbar_init(&aempty[a], 1);
+      mbar_init(&aempty[a], kMmaWarps);
     }
-    mbar_init(dfull, 1);
+    mbar_init(dfull, kMmaWarps);
     mbar_init(dempty, kDequantWarps);
     *abort_flag = 0;
     *last_flag = 0;
@@ -268,9 +269,11 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       }
       return;
     }
-    if (warp == kMmaWarp) {
-      // ------------------------------- MMA issuer ---------------------------------------------
+    if (warp >= kMmaWarp && warp < kMmaWarp + kMmaWarps) {
+      // ------------------------------- MMA issuers --------------------------------------------
       constexpr uint32_t idesc = instr_desc_f16(128, MPAD);
+      const int t = warp - kMmaWarp;  // this warp's 128-channel tile
+      const uint32_t d_tmem = tmem_base + (uint32_t)(t * MPAD);
       uint32_t it = 0;   // stage counter of this CTA
       uint32_t seg = 0;  // segment counter
       uint32_t u = u0;
@@ -282,37 +285,33 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         for (uint32_t x = 0; x < len; ++x, ++it) {
           const int s = (int)(it % NSTAGES);
           const int slot = (int)(it % NSLOTS);
-          if (it == 6) MARLIN_STAMP(19);
+          if (it == 6 && t == 0) MARLIN_STAMP(19);
           mbar_wait(&full[s], (it / NSTAGES) & 1u, abort_flag, p.status);
           mbar_wait(&afull[slot], (it / NSLOTS) & 1u, abort_flag, p.status);
-          if (it == 0) MARLIN_STAMP(4);
-          if (it == 6) MARLIN_STAMP(16);
+          if (it == 0 && t == 0) MARLIN_STAMP(4);
+          if (it == 6 && t == 0) MARLIN_STAMP(16);
           tc_fence_after_sync();
           if (lane == 0) {
             // descriptor of the first K = 16 step of the stage; the others differ in the address field only
             const uint64_t desc0 = smem_desc_k_sw128(smem_u32(stage0 + (size_t)s * G::STAGE_BYTES));
+            const uint32_t a_tmem = tmem_base + (uint32_t)(G::A_COL0 + (slot * 2 + t) * 64);
 #pragma unroll
-            for (int t = 0; t < 2; ++t) {
-              const uint32_t d_tmem = tmem_base + (uint32_t)(t * MPAD);
-              const uint32_t a_tmem = tmem_base + (uint32_t)(G::A_COL0 + (slot * 2 + t) * 64);
-#pragma unroll
-              for (int ks = 0; ks < 8; ++ks) {
-                const uint64_t bdesc = desc0 + (uint64_t)(((ks >> 2) * G::A_HALF_BYTES + (ks & 3) * 32) >> 4);
-                tc_mma_ts(d_tmem, a_tmem + ks * 8, bdesc, idesc, (x == 0 && ks == 0) ? 0u : 1u);
-              }
+            for (int ks = 0; ks < 8; ++ks) {
+              const uint64_t bdesc = desc0 + (uint64_t)(((ks >> 2) * G::A_HALF_BYTES + (ks & 3) * 32) >> 4);
+              tc_mma_ts(d_tmem, a_tmem + ks * 8, bdesc, idesc, (x == 0 && ks == 0) ? 0u : 1u);
             }
-            if (it == 6) MARLIN_STAMP(17);
+            if (it == 6 && t == 0) MARLIN_STAMP(17);
             tc_commit(&aempty[slot]);  // the A slot may be rewritten
             tc_commit(&empty[s]);      // the activation tile of the stage may be refilled
             if (x + 1 == len) tc_commit(dfull);
-            if (it == 6) MARLIN_STAMP(18);
+            if (it == 6 && t == 0) MARLIN_STAMP(18);
           }
           __syncwarp();
         }
         u += len;
         ++seg;
       }
-      MARLIN_STAMP(5);
+      if (t == 0) MARLIN_STAMP(5);
     }
     // ---- the TMEM owner waits for everybody who touches tensor memory, then frees it ----
     if (warp == kMmaWarp) {

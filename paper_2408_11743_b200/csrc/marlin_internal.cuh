@@ -25,7 +25,7 @@ constexpr int kProducerWarps = 4;     // the warps of the third warpgroup that i
 constexpr int kProducerRegs = 40;
 constexpr int kMaxStages = 32;
 constexpr int kMaxWorkers = 160;      // grid size cap (a B200 has 148 SMs)
-constexpr int kMaxSlabM = 32;         // rows of A handled by one launch of the mma.sync kernel
+constexpr int kMaxSlabM = 16;         // rows of A handled by one launch of the mma.sync kernel
 constexpr int kTcMaxSlabM = 128;      // rows of A handled by one launch of the tcgen05 kernel
 constexpr int kSmemBudget = 227 * 1024;
 

@@ -67,7 +67,7 @@ def test_same_layer_many_batch_sizes_and_repeatability(marlin, oracle_lib):
         # but the bound's rms is over the compared block
         _assert_close(oracle_lib, C, np.ascontiguousarray(C_ref[:M]))
         C2 = layer(case.A[:M])
-        if M <= 32:
+        if M <= 16:
             # warp-MMA kernel: partial tiles are summed in stripe order, the result is reproducible bit for bit
             assert np.array_equal(C.view(np.uint16), C2.view(np.uint16))
         else:
