@@ -439,7 +439,7 @@ def run_ours(args):
                          "frac": round(achieved / peaks["hbm_gbs"], 4), "traffic": NCU_DRAM_BYTES_PER_LAUNCH,
                          "traffic_note": "ncu capture of the M=16 launch; algorithmic bytes of that launch 35.1e6",
                          "peak_source": peaks["source"],
-                         "kernel": "gemm_dense_kernel (M <= 32) and gemm_dense_tc_kernel (M = 64, 128)",
+                         "kernel": "gemm_dense_kernel (M <= 16) and gemm_dense_tc_kernel (M = 32, 64, 128)",
                          "per_launch_us": round(step_s * 1e6 / launches_per_step, 3),
                          "algorithmic_bytes_per_step": step_alg_bytes},
             "per_m": per_m,

@@ -155,10 +155,13 @@ MARLIN_API int marlin_read_status(const void* workspace, marlin_stream stream);
 
 /* ---- host-side planning, exposed for inspection and tests (no GPU needed) ----------------------- */
 
-/* The striped partition of Section 3.4 "Striped Partitioning": the (column tile, 128-row k-block)
- * units of the weight matrix are numbered column by column, top to bottom, and worker i of
- * `workers` owns units [bounds[i], bounds[i+1]).  Fills n_tile (columns per tile: 64, 128 or 256),
- * workers (<= sm_count) and bounds[0..workers] (host pointers; `cap` entries available in bounds).
+/* The partition of Section 3.4 "Striped Partitioning" as the warp-level kernel uses it for this shape:
+ * the (column tile, 128-row k-block) units of the weight matrix are numbered column tile by column tile,
+ * top to bottom, and worker i of `workers` owns units [bounds[i], bounds[i+1]).  Two forms: where the
+ * column tiles divide the SMs well, every tile is cut into the same number of equal k-ranges, one per
+ * worker (no stripe crosses a tile boundary); otherwise the units are cut into `workers` even stripes,
+ * the paper's form.  Fills n_tile (columns per tile: 64, 128 or 256), workers (<= sm_count) and
+ * bounds[0..workers] (host pointers; `cap` entries available in bounds).
  * Returns MARLIN_ERR_SHAPE if cap is too small or the shape is invalid. */
 MARLIN_API int marlin_plan_stripes(int M, int K, int N, int sm_count, int* n_tile, int* workers,
                         int64_t* bounds, int cap);

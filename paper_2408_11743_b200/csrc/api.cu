@@ -191,6 +191,7 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
     p.partials = reinterpret_cast<float*>(ws + kWsPartialOff);
     p.tc_tiles = use_tc ? reinterpret_cast<float*>(ws + ((workspace_bytes & ~(size_t)255) - tc_tile_bytes(m_slab, N)))
                         : nullptr;
+    p.split = 0;
     p.slot_floats = kWsSlotCols * (slab_mpad(m_slab) < kMaxSlabM ? slab_mpad(m_slab) : kMaxSlabM);
     if (use_tc) {
       if (launch_gemm_dense_tc(p, info.sm_count, static_cast<cudaStream_t>(stream)) != cudaSuccess)
@@ -201,6 +202,7 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
       p.ncols = plan.ncols;
       p.units = (uint32_t)plan.units;
       p.workers = (uint32_t)plan.workers;
+      p.split = (uint32_t)plan.split;
       p.stages = plan.stages;
       p.stage_bytes = plan.stage_bytes;
       if (launch_gemm_dense(plan, p, sparse24, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MARLIN_ERR_CUDA;
@@ -302,7 +304,14 @@ int marlin_plan_stripes(int M, int K, int N, int sm_count, int* n_tile, int* wor
   if (cap < plan.workers + 1) return MARLIN_ERR_SHAPE;
   *n_tile = plan.nw * kChunkN;
   *workers = plan.workers;
-  for (int w = 0; w <= plan.workers; ++w) bounds[w] = stripe_begin(w, plan.units, plan.workers);
+  for (int w = 0; w <= plan.workers; ++w) {
+    if (plan.split) {
+      const long long t = w / plan.split, r = w % plan.split;
+      bounds[w] = t * plan.kb + (r * plan.kb) / plan.split;
+    } else {
+      bounds[w] = stripe_begin(w, plan.units, plan.workers);
+    }
+  }
   return MARLIN_OK;
 }
 

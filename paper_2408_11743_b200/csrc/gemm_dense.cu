@@ -114,7 +114,9 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
   const int lane = threadIdx.x & 31;
   const uint32_t worker = blockIdx.x;
   const uint32_t U = p.units, P = p.workers, KB = p.kb;
-  const uint32_t u0 = stripe_begin32(worker, U, P), u1 = stripe_begin32(worker + 1, U, P);
+  // split > 0: one k-range of one column tile per CTA instead of an even stripe over all units
+  const uint32_t u0 = p.split ? split_begin32(worker, KB, p.split) : stripe_begin32(worker, U, P);
+  const uint32_t u1 = p.split ? split_begin32(worker + 1, KB, p.split) : stripe_begin32(worker + 1, U, P);
   const int nstages = p.stages;
 
   pdl_launch_dependents();
@@ -233,6 +235,10 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
 
   float acc[4 * MB][4];
   float tmp[4 * MB][4];
+  // Dense path: the weights enter the MMAs as 1024 + q and 64 + q (dequant8_biased), and bias[mb] collects
+  // sum_k a[k] * (1032 or 72) of the open group with one more MMA per 16 rows of k whose weight operand is
+  // that constant: the same number in every output channel, taken off when the group closes.
+  float bias[SP ? 1 : MB][4];
   uint4 cur_raw = make_uint4(0, 0, 0, 0);  // 8 fp16 scales of the open group: columns 16j+g and 16j+8+g, j = 0..3
 
   auto close_group = [&]() {
@@ -243,12 +249,23 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
 #pragma unroll
       for (int mb = 0; mb < MB; ++mb) {
         const int r = j * MB + mb;
-        acc[r][0] += sc2.x * tmp[r][0];
-        acc[r][1] += sc2.x * tmp[r][1];
-        acc[r][2] += sc2.y * tmp[r][2];
-        acc[r][3] += sc2.y * tmp[r][3];
+        if constexpr (SP) {
+          acc[r][0] += sc2.x * tmp[r][0];
+          acc[r][1] += sc2.x * tmp[r][1];
+          acc[r][2] += sc2.y * tmp[r][2];
+          acc[r][3] += sc2.y * tmp[r][3];
+        } else {
+          acc[r][0] += sc2.x * (tmp[r][0] - bias[mb][0]);
+          acc[r][1] += sc2.x * (tmp[r][1] - bias[mb][1]);
+          acc[r][2] += sc2.y * (tmp[r][2] - bias[mb][2]);
+          acc[r][3] += sc2.y * (tmp[r][3] - bias[mb][3]);
+        }
         tmp[r][0] = tmp[r][1] = tmp[r][2] = tmp[r][3] = 0.f;
       }
+    }
+    if constexpr (!SP) {
+#pragma unroll
+      for (int mb = 0; mb < MB; ++mb) bias[mb][0] = bias[mb][1] = bias[mb][2] = bias[mb][3] = 0.f;
     }
   };
 
@@ -264,11 +281,12 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
     for (int r = 0; r < 4 * MB; ++r)
 #pragma unroll
       for (int x = 0; x < 4; ++x) { acc[r][x] = 0.f; tmp[r][x] = 0.f; }
-    int cur_group = -1;
-    if (!p.grouped) {
-      cur_raw = __ldg(reinterpret_cast<const uint4*>(srow));
-      cur_group = 0;
+    if constexpr (!SP) {
+#pragma unroll
+      for (int mb = 0; mb < MB; ++mb) bias[mb][0] = bias[mb][1] = bias[mb][2] = bias[mb][3] = 0.f;
     }
+    int cur_group = -1;
+    if (!p.grouped) cur_raw = __ldg(reinterpret_cast<const uint4*>(srow));
 
     // iterations of this segment that belong to this group: x = off, off + SK, ...
     const uint32_t off = (grp + SK - (it0 % SK)) % SK;
@@ -282,6 +300,14 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
           // the group's scales came with the stage (a read from global memory here would be a cold DRAM
           // access whose latency every warp would wait out once per stage)
           cur_raw = lds128(smem_u32(sc_ring) + (uint32_t)s * G::SC_BYTES + (uint32_t)(wn * 64 + g * 8) * 2);
+          cur_group = gi;
+        }
+      } else {
+        // one scale per column: the sums are still folded into `acc` every 1024 rows of k, so that the
+        // offsets carried in `tmp` never cost more than a few of its low bits
+        const int gi = (int)(kb >> 3);
+        if (gi != cur_group) {
+          if (cur_group >= 0) close_group();
           cur_group = gi;
         }
       }
@@ -362,14 +388,23 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             uint32_t x[4], y[4];
-            dequant8(X[j][2 * h + u], x);
-            dequant8(Y[j][2 * h + u], y);
+            dequant8_biased(X[j][2 * h + u], x);
+            dequant8_biased(Y[j][2 * h + u], y);
+            // registers 0, 1 of a fragment are its rows k < 8 (lower nibbles), 2, 3 its rows k >= 8 (upper)
             const uint32_t a0[4] = {x[0], y[0], x[1], y[1]};
             const uint32_t a1[4] = {x[2], y[2], x[3], y[3]};
 #pragma unroll
             for (int mb = 0; mb < MB; ++mb) {
               mma_16816(tmp[j * MB + mb], a0, bf[mb][4 * u], bf[mb][4 * u + 1]);
               mma_16816(tmp[j * MB + mb], a1, bf[mb][4 * u + 2], bf[mb][4 * u + 3]);
+            }
+          }
+          {
+            const uint32_t kc[4] = {kBiasLo, kBiasLo, kBiasHi, kBiasHi};
+#pragma unroll
+            for (int mb = 0; mb < MB; ++mb) {
+              mma_16816(bias[mb], kc, bf[mb][4 * u], bf[mb][4 * u + 1]);
+              mma_16816(bias[mb], kc, bf[mb][4 * u + 2], bf[mb][4 * u + 3]);
             }
           }
         }
@@ -406,8 +441,8 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
 
     if (warp == 0) MARLIN_STAMP(7);
     // ---- stripe fix-up across CTAs and output ----
-    const int first_w = (int)stripe_owner32(col * KB, U, P);
-    const int last_w = (int)stripe_owner32((col + 1) * KB - 1, U, P);
+    const int first_w = p.split ? (int)(col * p.split) : (int)stripe_owner32(col * KB, U, P);
+    const int last_w = p.split ? (int)(col * p.split + p.split - 1) : (int)stripe_owner32((col + 1) * KB - 1, U, P);
     if (u + len < u1) {
       // A segment in the middle of the stripe: group 0 holds the tile and finishes it alone (its L2 round
       // trips take a microsecond or two); the other groups go on with the k-blocks of the next segment.
@@ -430,7 +465,7 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
           if (last_flag[1]) {
             // every thread re-reads its own fragment positions of all partials, in stripe order
             for (int w = first_w; w <= last_w; ++w) {
-              const int slot = 2 * w + (col != stripe_begin32(w, U, P) / KB ? 1 : 0);
+              const int slot = 2 * w + ((!p.split && col != stripe_begin32(w, U, P) / KB) ? 1 : 0);
               const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)slot * p.slot_floats) +
                                   (size_t)wn * G::FRAG_F4 * 32 + lane;
 #pragma unroll
@@ -502,7 +537,7 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
           for (int d = 0; d < BATCH; ++d) {
             const int ww = w + d;
             if (ww <= last_w) {
-              const int slot = 2 * ww + (col != stripe_begin32(ww, U, P) / KB ? 1 : 0);
+              const int slot = 2 * ww + ((!p.split && col != stripe_begin32(ww, U, P) / KB) ? 1 : 0);
               const float4* src = reinterpret_cast<const float4*>(p.partials + (size_t)slot * p.slot_floats);
 #pragma unroll
               for (int e = 0; e < PER; ++e) {
@@ -666,17 +701,44 @@ bool make_dense_plan(int m_slab, int K, int N, int sm_count, bool sparse24, Dens
   if (m_slab < 1 || m_slab > kMaxSlabM || K < kTileK || K % kTileK || N < kChunkN || N % kChunkN) return false;
   if (sm_count < 1) return false;
   int mb = m_slab <= 8 ? 1 : 2;
-  // 128-column tiles (8 KB copies): measured best for the warp-MMA kernel; narrower tiles mean fewer CTAs per
-  // column tile in the stripe fix-up, wider ones fewer and larger copies
-  int nw = 2;
-  if (const char* e = getenv("MARLIN_B200_NW")) { int v = atoi(e); if (v == 1 || v == 2 || v == 4) nw = v; }
-  while (nw > 1 && N % (kChunkN * nw)) nw >>= 1;
+  const int kb = K / kTileK;
+  const long long max_workers = sm_count < kMaxWorkers ? sm_count : kMaxWorkers;
+  // Partition (Section 3.4 "Striped Partitioning", adapted).  Two forms.  Tile-aligned: every column tile
+  // is cut into S equal k-ranges, one per CTA, so that all CTAs do the same work and run the fix-up once
+  // (S = 1: not at all), with the tile width (64, 128 or 256 columns) that suits the shape.  Even stripes
+  // over all units (the paper's form, 128-column tiles): every SM is busy to the end, but a CTA whose
+  // stripe crosses a tile boundary pays the fix-up twice and finishes microseconds after the others.  A
+  // cost in units of one 4 KB chunk (about 0.1 us of a CTA's time), fitted to measurements on B200, picks
+  // between them: chunks per CTA, plus 0.6 per chunk-width and partial tile of the fix-up, plus 22 for the
+  // late finishers of even stripes.
+  int forced_nw = 0;
+  if (const char* e = getenv("MARLIN_B200_NW")) { int v = atoi(e); if (v == 1 || v == 2 || v == 4) forced_nw = v; }
+  bool allow_split = true;
+  if (const char* e = getenv("MARLIN_B200_SPLIT")) allow_split = atoi(e) != 0;
+  int even_nw = forced_nw ? forced_nw : 2;
+  while (even_nw > 1 && N % (kChunkN * even_nw)) even_nw >>= 1;
+  const long long even_units = (long long)(N / (kChunkN * even_nw)) * kb;
+  const long long even_workers = even_units < max_workers ? even_units : max_workers;
+  double best = (double)((even_units + even_workers - 1) / even_workers * even_nw) + 22.0;
+  int nw = even_nw, split = 0;
+  for (int cand = 1; cand <= 4 && allow_split; cand *= 2) {
+    if (forced_nw && cand != forced_nw) continue;
+    if (N % (kChunkN * cand)) continue;
+    const long long ncols = N / (kChunkN * cand);
+    long long S = max_workers / ncols;
+    if (S > kb) S = kb;
+    if (S < 1) continue;
+    const long long stages_per_cta = (kb + S - 1) / S;
+    const double cost = (double)(stages_per_cta * cand) + (S > 1 ? 0.6 * (double)(S * cand) : 0.0);
+    if (cost < best) { nw = cand; split = (int)S; best = cost; }
+  }
   plan->mb = mb;
   plan->nw = nw;
-  plan->kb = K / kTileK;
+  plan->kb = kb;
   plan->ncols = N / (kChunkN * nw);
   plan->units = (long long)plan->ncols * plan->kb;
-  long long workers = sm_count < kMaxWorkers ? sm_count : kMaxWorkers;
+  plan->split = split;
+  long long workers = split ? (long long)split * plan->ncols : max_workers;
   if (workers > plan->units) workers = plan->units;
   plan->workers = (int)workers;
   const int plan_mb = mb, plan_nw = nw;

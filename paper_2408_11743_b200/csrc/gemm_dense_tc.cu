@@ -120,15 +120,16 @@ __device__ long long g_timing_tc[kMaxWorkers][24];
 // ---------------------------------------------------------------------------------------------
 // geometry
 // ---------------------------------------------------------------------------------------------
-constexpr int kTcThreads = 384;
+constexpr int kTcThreads = 512;
 constexpr int kDequantWarps = 8;
 constexpr int kDequantThreads = kDequantWarps * 32;
-constexpr int kTcProducerWarps = 2;
-constexpr int kMmaWarp = 10;        // first of the MMA-issuing warps (it also owns the TMEM allocation)
-constexpr int kMmaWarps = 2;        // one per 128-channel tile: issuing a tcgen05.mma occupies the thread for tens of cycles
+constexpr int kTcProducerWarps = 2;  // warps 8, 9
+constexpr int kMmaWarp = 10;         // first of the MMA-issuing warps (it also owns the TMEM allocation)
 constexpr int kTcMaxStages = 8;
 constexpr int kTileN = 256;          // columns of W per CTA tile: two UMMA tiles of 128 channels
 constexpr int kTmemCols = 512;
+constexpr int kAuxRegs = 40;         // registers per thread of the copy and MMA warps
+constexpr int kDequantRegs = 216;    // 512 threads start with 128 each: 2 x 128 x (128 - 40) / 256 = 88 more
 
 template <int MPAD>
 struct TcGeometry {
@@ -144,9 +145,15 @@ struct TcGeometry {
           ? kTcMaxStages
           : (kSmemBudget - FIXED_BYTES - ALIGN_SLACK) / STAGE_BYTES;
   static constexpr int SMEM_BYTES = FIXED_BYTES + ALIGN_SLACK + STAGES * STAGE_BYTES;
-  // tensor memory: accumulators of the two 128-channel tiles in columns [0, 2*MPAD), then as many
-  // A-operand slots (2 tiles x 64 columns each) as fit in the 512 columns
-  static constexpr int A_SLOTS = (kTmemCols - 2 * MPAD) / 128 > 4 ? 4 : (kTmemCols - 2 * MPAD) / 128;
+  // Issuing one tcgen05.mma occupies its thread for about 75 cycles, more than a 128 x 64 x 16 product takes
+  // to execute, so up to batch 64 four warps issue: one per 128-channel tile and half of the k-block, each
+  // half into an accumulator of its own (the epilogue adds the two).  At batch 128 execution is the longer
+  // and two warps, one per tile, are enough.
+  static constexpr int MMA_WARPS = MPAD <= 64 ? 4 : 2;
+  static constexpr int KH = MMA_WARPS / 2;                 // accumulators per tile
+  static constexpr int D_COLS = 2 * KH * MPAD;             // accumulator of (tile t, half h) at column (t * KH + h) * MPAD
+  // then as many A-operand slots (2 tiles x 64 columns each) as fit in the 512 columns
+  static constexpr int A_SLOTS = (kTmemCols - D_COLS) / 128 > 4 ? 4 : (kTmemCols - D_COLS) / 128;
   static constexpr int A_COL0 = kTmemCols - A_SLOTS * 128;
 };
 
@@ -159,17 +166,19 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
   using G = TcGeometry<MPAD>;
   constexpr int NSTAGES = G::STAGES;
   constexpr int NSLOTS = G::A_SLOTS;
+  constexpr int NM = G::MMA_WARPS;
+  constexpr int KH = G::KH;
   extern __shared__ __align__(128) uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   uint64_t* full = reinterpret_cast<uint64_t*>(smem);          // [8]  TMA data of a stage has landed
-  uint64_t* empty = reinterpret_cast<uint64_t*>(smem + 64);    // [8]  stage may be refilled
+  uint64_t* empty = reinterpret_cast<uint64_t*>(smem + 64);    // [8]  the codes of a stage are in registers
   uint64_t* afull = reinterpret_cast<uint64_t*>(smem + 128);   // [4]  A-operand slot written
-  uint64_t* aempty = reinterpret_cast<uint64_t*>(smem + 160);  // [4]  A-operand slot consumed by the MMAs
-  uint64_t* dfull = reinterpret_cast<uint64_t*>(smem + 192);   //      accumulators of a segment complete
-  uint64_t* dempty = reinterpret_cast<uint64_t*>(smem + 200);  //      accumulators read out
-  uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(smem + 208);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + 212);
-  volatile int* last_flag = reinterpret_cast<volatile int*>(smem + 216);
+  uint64_t* mdone = reinterpret_cast<uint64_t*>(smem + 160);   // [8]  the MMAs of a stage have completed
+  uint64_t* dfull = reinterpret_cast<uint64_t*>(smem + 224);   //      accumulators of a segment complete
+  uint64_t* dempty = reinterpret_cast<uint64_t*>(smem + 232);  //      accumulators read out
+  uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(smem + 240);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + 244);
+  volatile int* last_flag = reinterpret_cast<volatile int*>(smem + 248);
   uint8_t* sc_ring = smem + 1024;  // [stage][256] fp16 scales, copied with the stage
   uint8_t* stage0 = smem + G::FIXED_BYTES;
 
@@ -177,20 +186,20 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
   const int lane = threadIdx.x & 31;
   const uint32_t worker = blockIdx.x;
   const uint32_t U = p.units, P = p.workers, KB = p.kb;
-  const uint32_t u0 = stripe_begin32(worker, U, P), u1 = stripe_begin32(worker + 1, U, P);
+  // split > 0: one k-range of one column tile per CTA (the last range of a tile ends where the next tile begins)
+  const uint32_t u0 = p.split ? split_begin32(worker, KB, p.split) : stripe_begin32(worker, U, P);
+  const uint32_t u1 = p.split ? split_begin32(worker + 1, KB, p.split) : stripe_begin32(worker + 1, U, P);
 
   pdl_launch_dependents();
   if (warp == 0) MARLIN_STAMP(10);
   if (threadIdx.x == 0) {
     for (int s = 0; s < NSTAGES; ++s) {
       mbar_init(&full[s], 1);
-      mbar_init(&empty[s], kDequantWarps + kMmaWarps);
+      mbar_init(&empty[s], kDequantWarps);
+      mbar_init(&mdone[s], NM);
     }
-    for (int a = 0; a < NSLOTS; ++a) {
-      mbar_init(&afull[a], kDequantWarps);
-      mbar_init(&aempty[a], kMmaWarps);
-    }
-    mbar_init(dfull, kMmaWarps);
+    for (int a = 0; a < NSLOTS; ++a) mbar_init(&afull[a], kDequantWarps);
+    mbar_init(dfull, NM);
     mbar_init(dempty, kDequantWarps);
     *abort_flag = 0;
     *last_flag = 0;
@@ -207,7 +216,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
   if (warp == 0) MARLIN_STAMP(0);
 
   if (warp >= kDequantWarps) {
-    setmaxnreg_dec<56>();
+    setmaxnreg_dec<kAuxRegs>();
     if (warp < kDequantWarps + kTcProducerWarps) {
       // ------------------------------- producers --------------------------------------------
       const int pw = warp - kDequantWarps;
@@ -250,7 +259,9 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       s -= NSTAGES;
       for (; u < u1; u += kTcProducerWarps) {
         const uint32_t col = u / KB, kb = u - col * KB;
+        // the stage is free when its codes are in registers and the MMAs that read its activations are done
         mbar_wait<200>(&empty[s], ph ^ 1u, abort_flag, p.status);
+        mbar_wait<200>(&mdone[s], ph ^ 1u, abort_flag, p.status);
         uint8_t* st = stage0 + (size_t)s * G::STAGE_BYTES;
         if (lane == 0) {
           mbar_expect_tx(&full[s], tx_bytes);
@@ -269,11 +280,14 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       }
       return;
     }
-    if (warp >= kMmaWarp && warp < kMmaWarp + kMmaWarps) {
+    if (warp >= kMmaWarp && warp < kMmaWarp + NM) {
       // ------------------------------- MMA issuers --------------------------------------------
       constexpr uint32_t idesc = instr_desc_f16(128, MPAD);
-      const int t = warp - kMmaWarp;  // this warp's 128-channel tile
-      const uint32_t d_tmem = tmem_base + (uint32_t)(t * MPAD);
+      constexpr int KS = 8 / KH;           // K = 16 steps per warp and stage
+      const int mw = warp - kMmaWarp;
+      const int t = mw & 1;                // 128-channel tile
+      const int h = mw >> 1;               // half of the k-block (always 0 with two warps)
+      const uint32_t d_tmem = tmem_base + (uint32_t)((t * KH + h) * MPAD);
       uint32_t it = 0;   // stage counter of this CTA
       uint32_t seg = 0;  // segment counter
       uint32_t u = u0;
@@ -285,33 +299,34 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         for (uint32_t x = 0; x < len; ++x, ++it) {
           const int s = (int)(it % NSTAGES);
           const int slot = (int)(it % NSLOTS);
-          if (it == 6 && t == 0) MARLIN_STAMP(19);
+          if (it == 6 && mw == 0) MARLIN_STAMP(19);
           mbar_wait(&full[s], (it / NSTAGES) & 1u, abort_flag, p.status);
           mbar_wait(&afull[slot], (it / NSLOTS) & 1u, abort_flag, p.status);
-          if (it == 0 && t == 0) MARLIN_STAMP(4);
-          if (it == 6 && t == 0) MARLIN_STAMP(16);
+          if (it == 0 && mw == 0) MARLIN_STAMP(4);
+          if (it == 6 && mw == 0) MARLIN_STAMP(16);
           tc_fence_after_sync();
           if (lane == 0) {
             // descriptor of the first K = 16 step of the stage; the others differ in the address field only
             const uint64_t desc0 = smem_desc_k_sw128(smem_u32(stage0 + (size_t)s * G::STAGE_BYTES));
             const uint32_t a_tmem = tmem_base + (uint32_t)(G::A_COL0 + (slot * 2 + t) * 64);
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
+            for (int k2 = 0; k2 < KS; ++k2) {
+              const int ks = h * KS + k2;
               const uint64_t bdesc = desc0 + (uint64_t)(((ks >> 2) * G::A_HALF_BYTES + (ks & 3) * 32) >> 4);
-              tc_mma_ts(d_tmem, a_tmem + ks * 8, bdesc, idesc, (x == 0 && ks == 0) ? 0u : 1u);
+              tc_mma_ts(d_tmem, a_tmem + ks * 8, bdesc, idesc, (x == 0 && k2 == 0) ? 0u : 1u);
             }
-            if (it == 6 && t == 0) MARLIN_STAMP(17);
-            tc_commit(&aempty[slot]);  // the A slot may be rewritten
-            tc_commit(&empty[s]);      // the activation tile of the stage may be refilled
+            if (it == 6 && mw == 0) MARLIN_STAMP(17);
+            // one arrival when these MMAs are done: the A slot may be rewritten, the activation tile refilled
+            tc_commit(&mdone[s]);
             if (x + 1 == len) tc_commit(dfull);
-            if (it == 6 && t == 0) MARLIN_STAMP(18);
+            if (it == 6 && mw == 0) MARLIN_STAMP(18);
           }
           __syncwarp();
         }
         u += len;
         ++seg;
       }
-      if (t == 0) MARLIN_STAMP(5);
+      if (mw == 0) MARLIN_STAMP(5);
     }
     // ---- the TMEM owner waits for everybody who touches tensor memory, then frees it ----
     if (warp == kMmaWarp) {
@@ -323,7 +338,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
   }
 
   // --------------------------------- dequantisers / epilogue ----------------------------------
-  setmaxnreg_inc<224>();
+  setmaxnreg_inc<kDequantRegs>();
   const int tile = warp >> 2;                 // which 128 channels of the 256-column tile
   const uint32_t lane_win = (uint32_t)(warp & 3) * 32u;  // this warp's TMEM lanes
   const int n256 = tile * 128 + (int)lane_win + lane;    // column of the thread inside the CTA tile
@@ -368,7 +383,11 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty[s]);
 
-      mbar_wait(&aempty[slot], ((it / NSLOTS) & 1u) ^ 1u, abort_flag, p.status);
+      if (it >= (uint32_t)NSLOTS) {
+        // the slot was last read by the MMAs of stage it - NSLOTS
+        const uint32_t jt = it - NSLOTS;
+        mbar_wait(&mdone[jt % NSTAGES], (jt / NSTAGES) & 1u, abort_flag, p.status);
+      }
       if (tr) MARLIN_STAMP(14);
       tc_fence_after_sync();
       const uint32_t a_col = tmem_lane + (uint32_t)(G::A_COL0 + (slot * 2 + tile) * 64);
@@ -376,16 +395,16 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       for (int c = 0; c < 4; ++c) {
         const uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
+        for (int hh = 0; hh < 2; ++hh) {
           uint32_t lo[4], hi[4], r[8];
-          dequant8(w[2 * h], lo);      // rows 64h + 16c + 0..7
-          dequant8(w[2 * h + 1], hi);  // rows 64h + 16c + 8..15
+          dequant8(w[2 * hh], lo);      // rows 64hh + 16c + 0..7
+          dequant8(w[2 * hh + 1], hi);  // rows 64hh + 16c + 8..15
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             r[e] = hmul2_u32(lo[e], s2);
             r[4 + e] = hmul2_u32(hi[e], s2);
           }
-          tc_st_x8(a_col + (uint32_t)(32 * h + 8 * c), r);  // column = row / 2
+          tc_st_x8(a_col + (uint32_t)(32 * hh + 8 * c), r);  // column = row / 2
         }
       }
       if (tr) MARLIN_STAMP(15);
@@ -401,40 +420,54 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
     mbar_wait(dfull, seg & 1u, abort_flag, p.status);
     if (warp == 0) MARLIN_STAMP(7);
     tc_fence_after_sync();
-    float acc[MPAD];
-#pragma unroll
-    for (int cc = 0; cc < MPAD / 32; ++cc) {
-      float part[32];
-      tc_ld_x32(tmem_lane + (uint32_t)(tile * MPAD + cc * 32), part);
-      tc_wait_ld();
-#pragma unroll
-      for (int e = 0; e < 32; ++e) acc[cc * 32 + e] = part[e];
-    }
-    tc_fence_before_sync();
-    __syncwarp();
-    if (lane == 0) mbar_arrive(dempty);
     ++seg;
-
     if (!waited_for_prior_grid) {
       // first write to C or the workspace: the previous kernel of the stream must be done with them
       pdl_wait_prior_grids();
       waited_for_prior_grid = true;
     }
-    const int first_w = (int)stripe_owner32(col * KB, U, P);
-    const int last_w = (int)stripe_owner32((col + 1) * KB - 1, U, P);
-    bool store = true;
-    if (last_w > first_w) {
-      // The column tile is shared by several CTAs.  With up to 128 rows a partial tile is large and
-      // a small layer splits every column many ways, so the sum is left to the L2: every contributor
-      // adds its partial into the tile's fp32 accumulation buffer with fire-and-forget reductions
-      // (float4 index = (m / 4) * 256 + column: coalesced over columns), the last arriver reads the
-      // total, clears the buffer for the next call and stores C.  (The order of these fp32 additions
-      // is not fixed, so the last bits of a shared tile can differ from run to run.)
-      float* tile_acc = p.tc_tiles + (size_t)col * (kTileN * MPAD);
-      float4* mine = reinterpret_cast<float4*>(tile_acc) + n256;
+    const int first_w = p.split ? (int)(col * p.split) : (int)stripe_owner32(col * KB, U, P);
+    const int last_w = p.split ? (int)(col * p.split + p.split - 1) : (int)stripe_owner32((col + 1) * KB - 1, U, P);
+    const bool shared_tile = last_w > first_w;
+    // The column tile may be shared by several CTAs.  With up to 128 rows a partial tile is large and
+    // a small layer splits every column many ways, so the sum is left to the L2: every contributor
+    // adds its partial into the tile's fp32 accumulation buffer with fire-and-forget reductions
+    // (float4 index = (m / 4) * 256 + column: coalesced over columns), the last arriver reads the
+    // total, clears the buffer for the next call and stores C.  (The order of these fp32 additions
+    // is not fixed, so the last bits of a shared tile can differ from run to run.)
+    float4* mine = reinterpret_cast<float4*>(p.tc_tiles + (size_t)col * (kTileN * MPAD)) + n256;
+    uint16_t* cptr = p.C + (size_t)col * kTileN + n256;
+    // 32 batch rows at a time: accumulators out of tensor memory, then either to the L2 or straight to C
+#pragma unroll 1
+    for (int cc = 0; cc < MPAD / 32; ++cc) {
+      float part[32];
+      tc_ld_x32(tmem_lane + (uint32_t)(tile * KH * MPAD + cc * 32), part);
+      if constexpr (KH == 2) {
+        float part2[32];
+        tc_ld_x32(tmem_lane + (uint32_t)((tile * KH + 1) * MPAD + cc * 32), part2);
+        tc_wait_ld();
 #pragma unroll
-      for (int m4 = 0; m4 < MPAD / 4; ++m4)
-        red_add_f32x4(mine + m4 * kTileN, acc[4 * m4], acc[4 * m4 + 1], acc[4 * m4 + 2], acc[4 * m4 + 3]);
+        for (int e = 0; e < 32; ++e) part[e] += part2[e];
+      } else {
+        tc_wait_ld();
+      }
+      if (shared_tile) {
+#pragma unroll
+        for (int m4 = 0; m4 < 8; ++m4)
+          red_add_f32x4(mine + (cc * 8 + m4) * kTileN, part[4 * m4], part[4 * m4 + 1], part[4 * m4 + 2], part[4 * m4 + 3]);
+      } else {
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          const int m = cc * 32 + e;
+          if (m < p.M) cptr[(size_t)m * p.N] = __half_as_ushort(__float2half_rn(part[e]));
+        }
+      }
+    }
+    tc_fence_before_sync();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(dempty);
+
+    if (shared_tile) {
       named_bar_sync(1, kDequantThreads);
       if (ctid == 0) {
         const int old = atom_add_acq_rel_gpu(&p.counters[col], 1);
@@ -443,23 +476,23 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         *last_flag = is_last;
       }
       named_bar_sync(1, kDequantThreads);
-      store = (*last_flag != 0);
-      if (store) {
+      if (*last_flag != 0) {
+        // all loads of the total in flight at once: this CTA is alone on the critical path of the tile
+        float4 t4[MPAD / 4];
 #pragma unroll
-        for (int m4 = 0; m4 < MPAD / 4; ++m4) {
-          const float4 t4 = ld_cg_f4(mine + m4 * kTileN);
-          acc[4 * m4] = t4.x; acc[4 * m4 + 1] = t4.y; acc[4 * m4 + 2] = t4.z; acc[4 * m4 + 3] = t4.w;
-        }
+        for (int m4 = 0; m4 < MPAD / 4; ++m4) t4[m4] = ld_cg_f4(mine + m4 * kTileN);
 #pragma unroll
         for (int m4 = 0; m4 < MPAD / 4; ++m4) mine[m4 * kTileN] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int m4 = 0; m4 < MPAD / 4; ++m4) {
+          const int m = 4 * m4;
+          if (m < p.M) cptr[(size_t)m * p.N] = __half_as_ushort(__float2half_rn(t4[m4].x));
+          if (m + 1 < p.M) cptr[(size_t)(m + 1) * p.N] = __half_as_ushort(__float2half_rn(t4[m4].y));
+          if (m + 2 < p.M) cptr[(size_t)(m + 2) * p.N] = __half_as_ushort(__float2half_rn(t4[m4].z));
+          if (m + 3 < p.M) cptr[(size_t)(m + 3) * p.N] = __half_as_ushort(__float2half_rn(t4[m4].w));
+        }
       }
       named_bar_sync(1, kDequantThreads);  // last_flag may be rewritten by the next segment
-    }
-    if (store) {
-      uint16_t* cptr = p.C + (size_t)col * kTileN + n256;
-#pragma unroll
-      for (int m = 0; m < MPAD; ++m)
-        if (m < p.M) cptr[(size_t)m * p.N] = __half_as_ushort(__float2half_rn(acc[m]));
     }
     u += len;
     if (warp == 0) MARLIN_STAMP(8);
@@ -519,6 +552,20 @@ cudaError_t launch_gemm_dense_tc(GemmParams p, int sm_count, cudaStream_t stream
   if (workers > units) workers = units;
   p.ncols = p.N / kTileN;
   p.units = (uint32_t)units;
+  // With up to 128 rows the epilogue of a segment (accumulators out of tensor memory, L2 reductions, arrival
+  // count) takes microseconds during which the CTA converts nothing, and under even stripes most CTAs run it
+  // twice.  Where the tiles divide the SMs well, each tile is cut into S k-ranges instead, one per CTA: one
+  // epilogue per CTA, all CTAs alike.  Otherwise (few CTAs per tile would idle many SMs) even stripes stay.
+  p.split = 0;
+  {
+    long long S = workers / p.ncols;
+    if (S > (long long)p.kb) S = p.kb;
+    const char* e = getenv("MARLIN_B200_TC_SPLIT");  // tuning knob: 0 forces even stripes
+    if (S >= 2 && S * p.ncols * 100 >= workers * 85 && !(e && atoi(e) == 0)) {
+      p.split = (uint32_t)S;
+      workers = S * p.ncols;
+    }
+  }
   p.workers = (uint32_t)workers;
   const int mpad = tc_mpad(p.M);
   if (mpad == 32) return launch_tc<32>(p, (int)workers, stream);

@@ -43,6 +43,7 @@ struct DensePlan {
   int ncols;       // N / (64 * nw)
   long long units; // ncols * kb
   int workers;     // CTAs
+  int split;       // 0: even stripes; S > 0: S k-ranges per column tile, one per CTA
   int stages;
   int stage_bytes;
   int smem_bytes;
@@ -73,6 +74,8 @@ struct GemmParams {
   float* partials;   // warp-MMA kernel: partial-tile slots
   float* tc_tiles;   // tcgen05 kernel: one fp32 accumulation tile per 256-column tile
   int slot_floats;   // floats per partial-tile slot
+  uint32_t split;    // tcgen05 kernel: 0 = even stripes over all units; S > 0 = every column tile is cut into S
+                     // k-ranges and worker w owns range w % S of tile w / S (one segment per CTA)
 };
 
 cudaError_t launch_gemm_dense(const DensePlan& plan, const GemmParams& p, bool sparse24, cudaStream_t stream);
@@ -97,5 +100,11 @@ __host__ __device__ inline int stripe_owner(long long x, long long U, long long 
 // the same in 32-bit arithmetic for the device (U * P < 2^32 is checked on the host)
 __device__ inline uint32_t stripe_begin32(uint32_t w, uint32_t U, uint32_t P) { return (w * U) / P; }
 __device__ inline uint32_t stripe_owner32(uint32_t x, uint32_t U, uint32_t P) { return ((x + 1) * P - 1) / U; }
+// The tile-aligned variant of the partition: tile t = w / S, k-range r = w % S covers k-blocks
+// [r * KB / S, (r + 1) * KB / S) of the tile (S <= KB, so no range is empty).
+__device__ inline uint32_t split_begin32(uint32_t w, uint32_t KB, uint32_t S) {
+  const uint32_t t = w / S, r = w - t * S;
+  return t * KB + (r * KB) / S;
+}
 
 }  // namespace marlin_b200

@@ -81,18 +81,30 @@ SHAPES = [(4096, 4096), (8192, 8192), (4096, 12288), (4096, 22016), (11008, 4096
 def test_stripe_partition_covers_every_unit_once(marlin, K, N, M, sms):
     n_tile, workers, bounds = marlin.plan_stripes(M, K, N, sms)
     assert n_tile in (64, 128, 256) and N % n_tile == 0
-    units = (N // n_tile) * (K // 128)
-    assert workers == min(sms, units)
+    kb = K // 128
+    units = (N // n_tile) * kb
+    assert 1 <= workers <= min(sms, units)
     assert bounds[0] == 0 and bounds[-1] == units and len(bounds) == workers + 1
     sizes = [b - a for a, b in zip(bounds, bounds[1:])]
-    assert min(sizes) >= 1 and max(sizes) - min(sizes) <= 1          # contiguous, balanced stripes
-    # the device finds the owner of unit x as floor(((x + 1) * P - 1) / U): check it against the bounds
-    import bisect
-    step = max(1, units // 997)
-    for x in list(range(0, units, step)) + [units - 1]:
-        owner = ((x + 1) * workers - 1) // units
-        assert bounds[owner] <= x < bounds[owner + 1]
-        assert owner == bisect.bisect_right(bounds, x) - 1
+    assert min(sizes) >= 1                                           # contiguous, nobody idle
+    if max(sizes) - min(sizes) <= 1 and workers == min(sms, units):
+        # even stripes: the device finds the owner of unit x as floor(((x + 1) * P - 1) / U)
+        import bisect
+        step = max(1, units // 997)
+        for x in list(range(0, units, step)) + [units - 1]:
+            owner = ((x + 1) * workers - 1) // units
+            assert bounds[owner] <= x < bounds[owner + 1]
+            assert owner == bisect.bisect_right(bounds, x) - 1
+    else:
+        # tile-aligned form: the same number S of k-ranges in every column tile, none crossing a tile
+        # boundary, their lengths within one k-block of each other
+        ncols = N // n_tile
+        assert workers % ncols == 0
+        S = workers // ncols
+        assert S <= kb
+        for w in range(workers):
+            assert bounds[w] // kb == (bounds[w + 1] - 1) // kb == w // S
+        assert max(sizes) - min(sizes) <= 1
 
 
 def test_byte_model_matches_paper():
