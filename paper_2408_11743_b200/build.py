@@ -16,7 +16,7 @@ _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libmarlin_b200.so")
 SOURCES = ["api.cu", "pack.cu", "pack_sparse.cu", "gemm_dense.cu", "gemm_dense_tc.cu"]
-HEADERS = [os.path.join(CSRC, "marlin_internal.cuh"), os.path.join(CSRC, "device_utils.cuh"), os.path.join(_ROOT, "include", "marlin_b200.h")]
+HEADERS = [os.path.join(CSRC, "marlin_internal.cuh"), os.path.join(CSRC, "device_utils.cuh"), os.path.join(CSRC, "tc_utils.cuh"), os.path.join(_ROOT, "include", "marlin_b200.h")]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

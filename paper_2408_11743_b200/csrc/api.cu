@@ -50,11 +50,6 @@ int device_info(DeviceInfo* out) {
   return MARLIN_OK;
 }
 
-// rows of the widest launch a call with this M can make, padded the way that launch pads them
-int slab_mpad(int max_M) {
-  return max_M <= 8 ? 8 : (max_M <= 16 ? 16 : (max_M <= 32 ? 32 : (max_M <= 64 ? 64 : 128)));
-}
-
 // Batch size from which the tcgen05 kernel takes over from the warp-level MMA kernel.
 int tc_min_m() {
   static int v = -1;
@@ -104,9 +99,9 @@ size_t marlin_packed_meta_bytes(int K, int N) {
 // Workspace map: [status word, counters: 8192 bytes][partial-tile slots of the warp-MMA kernel]
 // ... [fp32 accumulation tiles of the tcgen05 kernel, placed at the END of the buffer].  Everything is
 // zero at rest; both kernels leave it that way.
-static size_t mma_slot_bytes(int max_M) {
-  const int rows = slab_mpad(max_M) < kMaxSlabM ? slab_mpad(max_M) : kMaxSlabM;
-  return (size_t)2 * kMaxWorkers * kWsSlotCols * rows * sizeof(float);
+static size_t mma_slot_bytes(int /*max_M*/) {
+  // two slots per worker, each the widest partial tile of the small-batch kernels: 16 rows x 256 columns
+  return (size_t)2 * kMaxWorkers * kWsSlotCols * kMaxSlabM * sizeof(float);
 }
 static size_t tc_tile_bytes(int max_M, int N) {
   if (max_M < tc_min_m() || N % 256) return 0;
@@ -192,7 +187,7 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
     p.tc_tiles = use_tc ? reinterpret_cast<float*>(ws + ((workspace_bytes & ~(size_t)255) - tc_tile_bytes(m_slab, N)))
                         : nullptr;
     p.split = 0;
-    p.slot_floats = kWsSlotCols * (slab_mpad(m_slab) < kMaxSlabM ? slab_mpad(m_slab) : kMaxSlabM);
+    p.slot_floats = kWsSlotCols * kMaxSlabM;
     if (use_tc) {
       if (launch_gemm_dense_tc(p, info.sm_count, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return MARLIN_ERR_CUDA;
