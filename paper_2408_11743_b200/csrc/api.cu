@@ -187,6 +187,7 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
     p.tc_tiles = use_tc ? reinterpret_cast<float*>(ws + ((workspace_bytes & ~(size_t)255) - tc_tile_bytes(m_slab, N)))
                         : nullptr;
     p.split = 0;
+    p.cluster = 0;
     p.slot_floats = kWsSlotCols * kMaxSlabM;
     if (use_tc) {
       if (launch_gemm_dense_tc(p, info.sm_count, static_cast<cudaStream_t>(stream)) != cudaSuccess)

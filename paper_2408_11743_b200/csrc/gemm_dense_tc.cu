@@ -204,9 +204,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       if (*abort_flag) {
         for (int x = 0; x < 1000; ++x) __nanosleep(1000);
       }
-      return;
-    }
-    if (warp >= kMmaWarp && warp < kMmaWarp + NM) {
+    } else if (warp >= kMmaWarp && warp < kMmaWarp + NM) {
       // ------------------------------- MMA issuers --------------------------------------------
       constexpr uint32_t idesc = instr_desc_f16(128, MPAD);
       constexpr int KS = 8 / KH;           // K = 16 steps per warp and stage
@@ -253,6 +251,11 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         ++seg;
       }
       if (mw == 0) MARLIN_STAMP(5);
+    }
+    if (p.cluster) {
+      // every thread of every CTA of the cluster takes part in the two barriers of the epilogue
+      cluster_sync_all();
+      cluster_sync_all();
     }
     // ---- the TMEM owner waits for everybody who touches tensor memory, then frees it ----
     if (warp == kMmaWarp) {
@@ -355,6 +358,63 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
     const int first_w = p.split ? (int)(col * p.split) : (int)stripe_owner32(col * KB, U, P);
     const int last_w = p.split ? (int)(col * p.split + p.split - 1) : (int)stripe_owner32((col + 1) * KB - 1, U, P);
     const bool shared_tile = last_w > first_w;
+    if (p.cluster) {
+      // The CTAs of this column tile form a thread-block cluster and finish side by side, so the partial
+      // tiles never leave the SMs: the batch rows are dealt out to the S CTAs in blocks of four, every CTA
+      // sends each block of its partial tile into the shared memory of the block's owner (the stage ring is
+      // free by now), and each owner adds the S partials of its rows in rank order and stores that part of C.
+      // Fixed order of the fp32 sum, no atomics, no workspace.
+      constexpr int R4 = MPAD / 4;              // blocks of four batch rows
+      const int S = (int)p.split;
+      const int rmax = (R4 + S - 1) / S;        // blocks per owner, at most
+      const int r = (int)cluster_ctarank();
+      cluster_sync_all();                       // all CTAs of the tile are done with their stage rings
+      const uint32_t recv = smem_u32(stage0);   // [source rank][block][256 columns] float4
+      uint16_t* cptr = p.C + (size_t)col * kTileN + n256;
+#pragma unroll 1
+      for (int cc = 0; cc < MPAD / 32; ++cc) {
+        float part[32];
+        tc_ld_x32(tmem_lane + (uint32_t)(tile * KH * MPAD + cc * 32), part);
+        if constexpr (KH == 2) {
+          float part2[32];
+          tc_ld_x32(tmem_lane + (uint32_t)((tile * KH + 1) * MPAD + cc * 32), part2);
+          tc_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) part[e] += part2[e];
+        } else {
+          tc_wait_ld();
+        }
+#pragma unroll
+        for (int m4 = 0; m4 < 8; ++m4) {
+          const int blk = cc * 8 + m4;
+          const int owner = ((blk + 1) * S - 1) / R4;   // owner o holds blocks [o * R4 / S, (o + 1) * R4 / S)
+          const int li = blk - owner * R4 / S;
+          st_cluster_f32x4(recv + (uint32_t)(((r * rmax + li) * kTileN + n256) * 16), (uint32_t)owner, part[4 * m4],
+                           part[4 * m4 + 1], part[4 * m4 + 2], part[4 * m4 + 3]);
+        }
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(dempty);
+      cluster_sync_all();                       // everybody's blocks have arrived
+      const int b0 = r * R4 / S, b1 = (r + 1) * R4 / S;
+      for (int blk = b0; blk < b1; ++blk) {
+        const int li = blk - b0;
+        float4 sum = *reinterpret_cast<const float4*>(stage0 + (size_t)((0 * rmax + li) * kTileN + n256) * 16);
+        for (int src = 1; src < S; ++src) {
+          const float4 v = *reinterpret_cast<const float4*>(stage0 + (size_t)((src * rmax + li) * kTileN + n256) * 16);
+          sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
+        }
+        const int m = 4 * blk;
+        if (m < p.M) cptr[(size_t)m * p.N] = __half_as_ushort(__float2half_rn(sum.x));
+        if (m + 1 < p.M) cptr[(size_t)(m + 1) * p.N] = __half_as_ushort(__float2half_rn(sum.y));
+        if (m + 2 < p.M) cptr[(size_t)(m + 2) * p.N] = __half_as_ushort(__float2half_rn(sum.z));
+        if (m + 3 < p.M) cptr[(size_t)(m + 3) * p.N] = __half_as_ushort(__float2half_rn(sum.w));
+      }
+      u += len;
+      if (warp == 0) MARLIN_STAMP(8);
+      continue;
+    }
     // The column tile may be shared by several CTAs.  With up to 128 rows a partial tile is large and
     // a small layer splits every column many ways, so the sum is left to the L2: every contributor
     // adds its partial into the tile's fp32 accumulation buffer with fire-and-forget reductions
@@ -449,12 +509,35 @@ cudaError_t launch_tc(const GemmParams& p, int workers, cudaStream_t stream) {
   cfg.blockDim = dim3(kTcThreads);
   cfg.dynamicSmemBytes = G::SMEM_BYTES;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kernel, p, tmap);
+  GemmParams q = p;
+  q.cluster = 0;
+  if (p.cluster) {
+    // the S CTAs of a column tile as one thread-block cluster, if this device can co-schedule such a cluster
+    // (all of them at once: a GPC holds only so many clusters of a size, and a second wave would cost far
+    // more than the reduction through the L2 that is the alternative)
+    static int cluster_ok[64][9] = {};  // per device and cluster size: 0 unknown, 1 yes, -1 no
+    const int S = (int)p.split;
+    int ok = (dev >= 0 && dev < 64) ? cluster_ok[dev][S] : 0;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = (unsigned)S;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    if (ok == 0) {
+      cfg.numAttrs = 2;
+      int n = 0;
+      ok = (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) == cudaSuccess && n * S >= workers) ? 1 : -1;
+      (void)cudaGetLastError();
+      if (dev >= 0 && dev < 64) cluster_ok[dev][S] = ok;
+    }
+    cfg.numAttrs = ok > 0 ? 2 : 1;
+    q.cluster = ok > 0 ? 1u : 0u;
+  }
+  return cudaLaunchKernelEx(&cfg, kernel, q, tmap);
 }
 
 }  // namespace
@@ -486,11 +569,17 @@ cudaError_t launch_gemm_dense_tc(GemmParams p, int sm_count, cudaStream_t stream
   {
     long long S = workers / p.ncols;
     if (S > (long long)p.kb) S = p.kb;
+    if (S > 8) S = 8;  // the CTAs of a tile form a thread-block cluster: at most the portable size
     const char* e = getenv("MARLIN_B200_TC_SPLIT");  // tuning knob: 0 forces even stripes
     if (S >= 2 && S * p.ncols * 100 >= workers * 85 && !(e && atoi(e) == 0)) {
       p.split = (uint32_t)S;
       workers = S * p.ncols;
     }
+  }
+  {
+    const char* e = getenv("MARLIN_B200_TC_CLUSTER");  // tuning knob: 0 = reduce through the L2 instead
+    // from 33 rows up: below that the partial tiles are small and the L2 path is as fast
+    p.cluster = (p.split >= 2 && p.M > 32 && !(e && atoi(e) == 0)) ? 1u : 0u;
   }
   p.workers = (uint32_t)workers;
   const int mpad = tc_mpad(p.M);

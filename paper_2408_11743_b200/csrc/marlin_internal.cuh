@@ -74,6 +74,7 @@ struct GemmParams {
   float* partials;   // warp-MMA kernel: partial-tile slots
   float* tc_tiles;   // tcgen05 kernel: one fp32 accumulation tile per 256-column tile
   int slot_floats;   // floats per partial-tile slot
+  uint32_t cluster;  // tcgen05 kernel: 1 = launched as thread-block clusters of `split` CTAs (the CTAs of one column tile)
   uint32_t split;    // tcgen05 kernel: 0 = even stripes over all units; S > 0 = every column tile is cut into S
                      // k-ranges and worker w owns range w % S of tile w / S (one segment per CTA)
 };
