@@ -72,7 +72,7 @@ struct Geometry {
   static constexpr int STAGE_BYTES = A_BYTES + W_BYTES + META_BYTES;  // multiple of 1024
   static constexpr int FRAG_F4 = MB * 4;                     // float4 accumulator registers per thread
   static constexpr int TILE_F4 = NW * FRAG_F4 * 32;          // float4s of one partial tile
-  static constexpr int RED_BYTES = (SK / 2) * TILE_F4 * 16;
+  static constexpr int RED_BYTES = (SK - 1) * TILE_F4 * 16;  // parked tiles of groups 1 .. SK - 1
   static constexpr int CST_STRIDE = NT + 8;                  // halves
   static constexpr int CST_BYTES = MPAD * CST_STRIDE * 2;
   static constexpr int SC_BYTES = NT * 2;                    // group scales of one stage (one row of the tile)
@@ -213,6 +213,11 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
     if (*abort_flag) {
       // give copies that may still be in flight time to land before the CTA's shared memory goes away
       for (int x = 0; x < 1000; ++x) __nanosleep(1000);
+    }
+    if (p.cluster) {
+      // every thread of every CTA of the cluster takes part in the two barriers of the fix-up
+      cluster_sync_all();
+      cluster_sync_all();
     }
     return;
   }
@@ -419,25 +424,27 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
     if (warp == 0) MARLIN_STAMP(5);
     if (warp == kConsumerWarps - 1) MARLIN_STAMP(6);
 
-    // ---- reduce the SK groups of this CTA (the last step of Algorithm 1, as a tree) ----
+    // ---- reduce the SK groups of this CTA (the last step of Algorithm 1) ----
+    // Every group but the first parks its tile in shared memory; after one barrier group 0 adds them to its
+    // own in group order (one pass instead of a tree: a barrier costs more here than a few shared loads).
+    if (grp > 0) {
+      float4* dst = red + (size_t)(grp - 1) * G::TILE_F4 + (size_t)wn * G::FRAG_F4 * 32 + lane;
 #pragma unroll
-    for (int half = SK / 2; half >= 1; half >>= 1) {
-      if (grp >= half && grp < 2 * half) {
-        float4* dst = red + (size_t)(grp - half) * G::TILE_F4 + (size_t)wn * G::FRAG_F4 * 32 + lane;
+      for (int r = 0; r < 4 * MB; ++r) dst[r * 32] = make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
+    }
+    named_bar_sync(1, kConsumerThreads);
+    if (grp == 0) {
 #pragma unroll
-        for (int r = 0; r < 4 * MB; ++r) dst[r * 32] = make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
-      }
-      named_bar_sync(1, kConsumerThreads);
-      if (grp < half) {
-        const float4* src = red + (size_t)grp * G::TILE_F4 + (size_t)wn * G::FRAG_F4 * 32 + lane;
+      for (int gq = 1; gq < SK; ++gq) {
+        const float4* src = red + (size_t)(gq - 1) * G::TILE_F4 + (size_t)wn * G::FRAG_F4 * 32 + lane;
 #pragma unroll
         for (int r = 0; r < 4 * MB; ++r) {
           const float4 v = src[r * 32];
           acc[r][0] += v.x; acc[r][1] += v.y; acc[r][2] += v.z; acc[r][3] += v.w;
         }
       }
-      named_bar_sync(1, kConsumerThreads);
     }
+    named_bar_sync(1, kConsumerThreads);  // `red` may be written again
 
     if (warp == 0) MARLIN_STAMP(7);
     // ---- stripe fix-up across CTAs and output ----
@@ -507,7 +514,43 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
     }
     // ---- the last segment of the stripe: all consumer threads take part ----
     bool tile_in_cst = false;
-    if (last_w > first_w) {
+    if (p.cluster) {
+      // The CTAs of this column tile form a thread-block cluster and finish side by side.  The partial tiles
+      // go straight into the shared memory of the cluster's first CTA (its stage ring is free by now), which
+      // adds them to its own in rank order: the order of the workspace path, without its L2 round trips.
+      const int rank = (int)worker - first_w;
+      cluster_sync_all();  // every CTA of the tile is done with its stage ring
+      if (rank != 0 && grp == 0) {
+        const uint32_t dst = stage0_s + (uint32_t)(((rank - 1) * G::TILE_F4 + wn * G::FRAG_F4 * 32 + lane) * 16);
+#pragma unroll
+        for (int r = 0; r < 4 * MB; ++r) st_cluster_f32x4(dst + (uint32_t)(r * 32 * 16), 0u, acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
+      }
+      cluster_sync_all();  // the partial tiles have arrived
+      if (rank == 0) {
+        if (grp == 0) {
+          for (int src = 1; src <= last_w - first_w; ++src) {
+            const uint32_t from = stage0_s + (uint32_t)(((src - 1) * G::TILE_F4 + wn * G::FRAG_F4 * 32 + lane) * 16);
+#pragma unroll
+            for (int r = 0; r < 4 * MB; ++r) {
+              const uint4 v = lds128(from + (uint32_t)(r * 32 * 16));
+              acc[r][0] += __uint_as_float(v.x); acc[r][1] += __uint_as_float(v.y);
+              acc[r][2] += __uint_as_float(v.z); acc[r][3] += __uint_as_float(v.w);
+            }
+          }
+#pragma unroll
+          for (int r = 0; r < 4 * MB; ++r) {
+            const int j = r / MB, mb = r % MB;
+            const int n = wn * 64 + 16 * j + g;
+            const int m = mb * 8 + 2 * c;
+            cst[m * G::CST_STRIDE + n] = __half_as_ushort(__float2half_rn(acc[r][0]));
+            cst[(m + 1) * G::CST_STRIDE + n] = __half_as_ushort(__float2half_rn(acc[r][1]));
+            cst[m * G::CST_STRIDE + n + 8] = __half_as_ushort(__float2half_rn(acc[r][2]));
+            cst[(m + 1) * G::CST_STRIDE + n + 8] = __half_as_ushort(__float2half_rn(acc[r][3]));
+          }
+        }
+        tile_in_cst = true;
+      }
+    } else if (last_w > first_w) {
       // this column tile is shared: publish the partial, count arrivals
       if (grp == 0) {
         const int my_slot = 2 * (int)worker + (col != u0 / KB ? 1 : 0);
@@ -651,6 +694,7 @@ namespace {
 template <int MB, int NW, bool SP>
 cudaError_t launch_one(const DensePlan& plan, const GemmParams& p, cudaStream_t stream) {
   constexpr int CW = consumer_warps_for(MB);
+  constexpr size_t G_TILE_BYTES = (size_t)Geometry<MB, NW, CW, SP>::TILE_F4 * 16;
   auto kernel = gemm_dense_kernel<MB, NW, CW, SP>;
   static bool attr_set[64] = {};  // per device
   int dev = 0;
@@ -668,12 +712,35 @@ cudaError_t launch_one(const DensePlan& plan, const GemmParams& p, cudaStream_t 
   cfg.blockDim = dim3((CW + 4) * 32);
   cfg.dynamicSmemBytes = plan.smem_bytes;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kernel, p, tmap);
+  GemmParams q = p;
+  q.cluster = 0;
+  const int S = plan.split;
+  const char* e = getenv("MARLIN_B200_CLUSTER");  // tuning knob: 0 = fix-up through the workspace
+  if (S >= 2 && S <= 8 && (size_t)(S - 1) * G_TILE_BYTES <= (size_t)plan.stages * plan.stage_bytes && !(e && atoi(e) == 0)) {
+    // the S CTAs of a column tile as one thread-block cluster, if all clusters of the grid fit on the device
+    // at once (a GPC holds only so many clusters of a size; a second wave would cost more than it saves)
+    static int cluster_ok[64][9] = {};  // per device and cluster size: 0 unknown, 1 yes, -1 no
+    int ok = (dev >= 0 && dev < 64) ? cluster_ok[dev][S] : 0;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = (unsigned)S;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    if (ok == 0) {
+      cfg.numAttrs = 2;
+      int n = 0;
+      ok = (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) == cudaSuccess && n * S >= plan.workers) ? 1 : -1;
+      (void)cudaGetLastError();
+      if (dev >= 0 && dev < 64) cluster_ok[dev][S] = ok;
+    }
+    cfg.numAttrs = ok > 0 ? 2 : 1;
+    q.cluster = ok > 0 ? 1u : 0u;
+  }
+  return cudaLaunchKernelEx(&cfg, kernel, q, tmap);
 }
 
 template <int MB, int NW, bool SP>

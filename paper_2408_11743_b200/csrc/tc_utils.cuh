@@ -66,21 +66,6 @@ __device__ __forceinline__ void tc_ld_x16(uint32_t taddr, float (&r)[16]) {
       : "r"(taddr)
       : "memory");
 }
-// Thread-block cluster: hardware barrier over all threads of all CTAs of the cluster (release / acquire), and
-// a 16-byte store into the shared memory of the CTA with rank `cta` at the address that `local_addr` has here.
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-__device__ __forceinline__ void st_cluster_f32x4(uint32_t local_addr, uint32_t cta, float a, float b, float c, float d) {
-  uint32_t remote;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(cta));
-  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(remote), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
-}
 // fire-and-forget fp32 vector reduction at the L2
 __device__ __forceinline__ void red_add_f32x4(float4* addr, float a, float b, float c, float d) {
   asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
