@@ -97,9 +97,10 @@ MARLIN_API int marlin_unpack(const void* w_packed, const void* s_packed, uint32_
  * Accumulation is fp32 (also across stripes); the result is rounded once to fp16 (nearest even).
  * Up to 16 rows the warp-level kernel runs and the same inputs give the same bits on every call.
  * From 17 rows the tcgen05 kernel takes over (128 rows per launch, N a multiple of 256; otherwise the
- * warp-level kernel runs on slabs of 16 rows): there the partial sums of a column tile shared by
- * several CTAs are added in fp32 in arrival order, so the last bit of an fp16 result can differ between
- * two calls.
+ * warp-level kernel runs on slabs of 16 rows).  Where it adds the partial sums of a column tile shared
+ * by several CTAs through the L2 (up to 32 rows, or shapes whose CTAs do not fit as one wave of
+ * thread-block clusters) the fp32 additions happen in arrival order, so the last bit of an fp16 result
+ * can differ between two calls; otherwise the order is fixed there too.
  * Errors: argument checks return before anything is queued.  A kernel whose bounded waits expire
  * sets the workspace status word; read it with marlin_read_status. */
 MARLIN_API int marlin_gemm(const void* A, const void* w_packed, const void* s_packed, void* C,

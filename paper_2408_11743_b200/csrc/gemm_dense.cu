@@ -1,27 +1,33 @@
-// Dense W4A16 layer for sm_100a, decode batch sizes (one launch handles up to 16 rows of A).
+// W4A16 layer for sm_100a, decode batch sizes (one launch handles up to 16 rows of A), dense and 2:4 sparse.
 //
-// Structure of one CTA (one per SM, persistent over its stripe of work units):
-//   warp 8        producer: per k-block ONE bulk-async copy (cp.async.bulk + mbarrier complete_tx) of
-//                 the contiguous packed weights of the column tile and one TMA tensor-tile copy per
-//                 64-wide half of the A tile (128-byte swizzle, rows beyond M zero-filled by the
-//                 hardware) into a ring of shared-memory stages.  Weights carry an L2 evict-first
-//                 policy (each byte is read once), activations evict-last (re-read by every tile).
-//                 Issuing a bulk copy costs the producer on the order of a hundred cycles whatever
-//                 its size, so the design keeps copies few and large.
+// Structure of one CTA (one per SM, 384 threads, persistent over its share of the work units):
+//   warps 8..11   producers.  Per k-block ONE bulk-async copy (cp.async.bulk + mbarrier complete_tx) of
+//                 the contiguous packed weights of the column tile, one of the tile's row of group scales,
+//                 and one TMA tensor-tile copy per 64-wide half of the A tile (128-byte swizzle, rows beyond M
+//                 zero-filled by the hardware) into a ring of shared-memory stages.  Weights carry an L2
+//                 evict-first policy (each byte is read once), activations evict-last (re-read by every
+//                 tile).  Issuing a bulk copy occupies a warp for a few hundred cycles whatever its size, so
+//                 copies are few and large and four warps take the stages round-robin.  The weights of the
+//                 first pass over the ring are requested before the programmatic dependency wait.
 //   warps 0..7    consumers, arranged as SK groups of NW warps.  Stage number `it` of the CTA is
 //                 consumed by group it % SK; inside a group warp wn owns 64 output columns.  A warp
-//                 reads its 16-byte weight vectors, converts the 4-bit codes to fp16 (q - 8) with the
-//                 exponent-bias trick, and feeds mma.sync.m16n8k16 with the WEIGHTS as the 16-wide
-//                 operand and the batch on the 8-wide one, so that batch sizes 1..8 cost one MMA per
-//                 256 weights.  The group scale is not applied to the weights: each group of k
-//                 accumulates into `tmp`, and `acc += s * tmp` in fp32 when the group ends; the
-//                 scales themselves are read straight from global memory (one 16-byte load per lane
-//                 and group, issued a whole stage before its use).
-//   end of a column segment: tree reduction of the SK groups through shared memory, then the stripe
-//                 fix-up across CTAs: partial tiles go to the workspace in fp32, an arrival counter
-//                 (acq_rel atomic) tells the last CTA of a column tile to add them in stripe order,
-//                 with all its threads and all loads in flight at once, and write fp16 C.
-//                 Nobody spins on another CTA.
+//                 reads its 16-byte weight vectors, turns the 4-bit codes into fp16 with the exponent-bias
+//                 trick, and feeds mma.sync.m16n8k16 with the WEIGHTS as the 16-wide operand and the batch
+//                 on the 8-wide one, so that batch sizes 1..8 cost one MMA per 256 weights.
+//                 Dense layers skip the subtraction of the bias trick: the weights enter the MMA as 1024 + q
+//                 and 64 + q, one more MMA per 16 rows of k with a constant weight operand collects
+//                 sum_k a[k] * (1032 or 72), and the difference is taken when the group closes (five ALU
+//                 instructions per eight weights instead of nine).  2:4 layers convert exactly (the
+//                 correction would depend on the metadata).
+//                 The group scale is not applied to the weights: each group of k accumulates into `tmp`,
+//                 and `acc += s * (tmp - bias)` in fp32 when the group ends.
+//   end of a column segment: the groups of the CTA add their tiles through shared memory; then the fix-up
+//                 across the CTAs that share the column tile, one of three ways: through the shared memory of
+//                 the first CTA of a thread-block cluster (tile-aligned partition, clusters fit in one wave);
+//                 or partial tiles to the workspace in fp32 and an arrival counter (acq_rel atomic) that
+//                 tells the last CTA to add them in worker order; a segment in the middle of an even stripe
+//                 is handled that way by warp group 0 alone while the others go on.  Always the same order
+//                 of the fp32 sum; nobody spins on another CTA.
 //
 // Paper correspondence (Section 3.4): weight streaming and evict-first ("Maximizing Loading
 // Bandwidth"), multi-stage pipeline ("Memory Load Pipelining"), warps splitting K with a shared

@@ -8,25 +8,32 @@
 //     D_t[128 channels x MPAD batch rows] += W_t^T[128 x 128] . A^T[128 x MPAD],   t = 0, 1
 // with UMMA shape M = 128 (output channels on the TMEM lanes), N = MPAD (batch), K = 16.
 //
-// One CTA per SM, 384 threads:
-//   warps 0..7   dequantisers: thread = one output channel of the tile.  It reads its 128 codes of the
-//                k-block (four 16-byte shared loads), converts them to fp16 (q - 8) with the
-//                exponent-bias trick (Section 3.4 "Dequantization and Tensor Cores"), multiplies by the
-//                group scale (Section 3.4 "Groups and Instruction Ordering": applied in the main loop)
-//                and writes the 128 values into its TMEM lane with tcgen05.st (64 columns, two k per
-//                column).  Two A-operand slots let conversion of k-block i+1 overlap the MMAs of i.
-//                At the end of a column segment the same warps read the accumulator back (tcgen05.ld),
-//                run the stripe fix-up and store C.
-//   warps 8, 9   producers: per k-block one 16 KB bulk copy of packed weights (evict-first) and one TMA
-//                tensor tile per 64-wide half of the activations (128-byte swizzle = the canonical
-//                K-major UMMA layout, rows >= M zero-filled), into a ring of shared-memory stages.
-//   warp 10      MMA issuer: one thread issues 2 x 8 tcgen05.mma per k-block (A from TMEM, B = the
-//                activation tile through a shared-memory descriptor), then tcgen05.commit to the
-//                barriers that free the A slot and the stage.  It also owns the TMEM allocation.
-//   warp 11      idle (completes the producer warpgroup for setmaxnreg).
+// One CTA per SM, 512 threads:
+//   warps 0..7    dequantisers: thread = one output channel of the tile.  It reads its 128 codes of the
+//                 k-block (four 16-byte shared loads), converts them to fp16 (q - 8) with the
+//                 exponent-bias trick (Section 3.4 "Dequantization and Tensor Cores"), multiplies by the
+//                 group scale (Section 3.4 "Groups and Instruction Ordering": applied in the main loop)
+//                 and writes the 128 values into its TMEM lane with tcgen05.st (64 columns, two k per
+//                 column).  Two or three A-operand slots let conversion of k-block i+1 overlap the MMAs of i.
+//                 At the end of a column segment the same warps read the accumulators back (tcgen05.ld),
+//                 run the fix-up and store C.
+//   warps 8, 9    producers: per k-block one 16 KB bulk copy of packed weights (evict-first), the row of
+//                 group scales, and one TMA tensor tile per 64-wide half of the activations (128-byte
+//                 swizzle = the canonical K-major UMMA layout, rows >= M zero-filled), into a ring of stages.
+//   warps 10..13  MMA issuers.  Issuing one tcgen05.mma occupies its thread for about 75 cycles, more than a
+//                 128 x 64 x 16 product takes to execute, so up to batch 64 four warps issue (tile t, half h
+//                 of the k-block, each half into an accumulator of its own); at batch 128 two.  One
+//                 tcgen05.commit per stage and warp signals that the A slot and the stage are free.  Warp 10
+//                 owns the TMEM allocation.
+//   warps 14, 15  idle (they complete the last warpgroup for setmaxnreg).
 //
-// Stripe partition, bounded waits and programmatic dependent launch are those of the small-batch kernel
-// (gemm_dense.cu); the stripe fix-up adds the partial tiles with L2 reductions instead of gathering them.
+// Partition: every column tile is cut into S k-ranges, one per CTA, where that keeps most SMs busy (one
+// epilogue per CTA, all CTAs alike); else even stripes over all units.  Fix-up of a shared tile: above 32
+// rows and when the S CTAs of every tile fit on the device as one wave of thread-block clusters, the
+// partial tiles are exchanged through distributed shared memory and every CTA finishes a share of the
+// batch rows (fixed order of the sum); otherwise every contributor adds its partial tile into an fp32 tile
+// in the workspace with L2 reductions and the last arriver stores C.  Bounded waits and programmatic
+// dependent launch are those of the small-batch kernel (gemm_dense.cu).
 #include <stdlib.h>
 
 #include "device_utils.cuh"
