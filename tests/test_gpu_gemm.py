@@ -48,6 +48,32 @@ def test_gemm_matches_oracle(marlin, oracle_lib, M, K, N, G):
     _assert_close(oracle_lib, C, C_ref)
 
 
+# The planner picks a partition and a fix-up per shape, so the default run exercises only one of them for a
+# given shape.  The tuning switches of the library force the others: even stripes instead of the tile-aligned
+# partition, the workspace fix-up instead of thread-block clusters, each tile width.
+MODES = [
+    {"MARLIN_B200_SPLIT": "0", "MARLIN_B200_TC_SPLIT": "0"},             # even stripes in both kernels
+    {"MARLIN_B200_CLUSTER": "0", "MARLIN_B200_TC_CLUSTER": "0"},         # no clusters: fix-up through the workspace
+    {"MARLIN_B200_NW": "1"}, {"MARLIN_B200_NW": "2"}, {"MARLIN_B200_NW": "4"},
+    {"MARLIN_B200_NW": "4", "MARLIN_B200_SPLIT": "0"}, {"MARLIN_B200_NW": "1", "MARLIN_B200_CLUSTER": "0"},
+]
+MODE_SHAPES = [(1, 4096, 4096, 128), (8, 2048, 1536, 128), (16, 1024, 768, -1), (13, 11008, 512, 128),
+               (40, 4096, 4096, 128), (128, 2048, 1024, 128), (64, 8192, 8192, 128)]
+
+
+@pytest.mark.parametrize("mode", range(len(MODES)))
+def test_every_partition_and_fixup_path_matches_oracle(marlin, oracle_lib, mode, monkeypatch):
+    for k, v in MODES[mode].items():
+        monkeypatch.setenv(k, v)
+    for M, K, N, G in MODE_SHAPES:
+        case = inputs.make_dense(M, K, N, G, seed=31 * mode + M + K + N)
+        layer = DenseLayer(marlin, case.q_kpacked, case.S, G, max_M=M)
+        C = layer(case.A)
+        _assert_close(oracle_lib, C, oracle_lib.gemm(case.A, case.q_kpacked, case.S, case.G))
+        counters = to_host(layer.ws[256:8192])
+        assert np.all(counters == 0)
+
+
 def test_config1_single_layer(marlin, oracle_lib):
     name, M, K, N, G, seed = next(inputs.iter_cases(1))
     case = inputs.make_dense(M, K, N, G, seed)

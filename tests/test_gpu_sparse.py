@@ -68,6 +68,23 @@ def test_sparse_gemm_matches_oracle(marlin, oracle_lib, M, K, N, G):
     assert bad == 0, f"{bad} elements out of tolerance, worst ratio {worst:.3f}, rms {rms:.3f}"
 
 
+# the partition and the fix-up the planner did not pick for a shape, forced through the library's tuning switches
+SPARSE_MODES = [{"MARLIN_B200_SPLIT": "0"}, {"MARLIN_B200_CLUSTER": "0"}, {"MARLIN_B200_NW": "1"},
+                {"MARLIN_B200_NW": "2"}, {"MARLIN_B200_NW": "4", "MARLIN_B200_SPLIT": "0"}]
+
+
+@pytest.mark.parametrize("mode", range(len(SPARSE_MODES)))
+def test_sparse_every_partition_and_fixup_path(marlin, oracle_lib, mode, monkeypatch):
+    for k, v in SPARSE_MODES[mode].items():
+        monkeypatch.setenv(k, v)
+    for M, K, N, G in [(1, 4096, 4096, 128), (8, 2048, 1536, 128), (16, 1024, 768, -1), (40, 4096, 1024, 128)]:
+        case = inputs.make_sparse24(M, K, N, G, seed=17 * mode + M + K + N)
+        C = SparseLayer(marlin, case, M)(case.A)
+        C_ref = oracle_lib.gemm_sparse24(case.A, case.qc_kpacked, case.idx, case.S, case.G)
+        bad, worst, rms = oracle_lib.check_tolerance(C, C_ref)
+        assert bad == 0, f"{bad} elements out of tolerance, worst ratio {worst:.3f}, rms {rms:.3f}"
+
+
 def test_sparse_equals_dense_kernel_on_the_expanded_matrix(marlin, oracle_lib):
     # the dense kernel on the matrix with code 8 (value 0) at the pruned positions computes the same layer
     M, K, N, G = 16, 2048, 1024, 128
