@@ -39,7 +39,7 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
-from paper_2408_11743_b200 import inputs, roofline  # noqa: E402
+from paper_2408_11743_b200 import inputs, replicas, roofline  # noqa: E402
 
 K_DIM, N_DIM, GROUP = 8192, 8192, 128
 SWEEP = (1, 2, 4, 8, 16, 32, 64, 128)
@@ -344,13 +344,10 @@ def run_ours(args):
     barrier()
     sampler.stop()
     clocks = sampler.summary(t_wall0, t_wall1)
-    if world > 1:
-        t = torch.tensor([elapsed], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed = float(t.item())
+    elapsed = replicas.max_over_ranks(elapsed, dev)
     step_s = elapsed / args.steps
     step_wbytes = wbytes * len(SWEEP)
-    value = world * step_wbytes / step_s / 1e9
+    value = replicas.job_throughput(step_wbytes, world, step_s) / 1e9
     step_alg_bytes = sum(roofline.algorithmic_bytes(M, K_DIM, N_DIM, GROUP) for M in SWEEP)
     launches_per_step = sum(launches_for(M) for M in SWEEP)
 
