@@ -93,7 +93,9 @@ struct TcGeometry {
 // ---------------------------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------------------------
-template <int MPAD>
+// GR: the layer has group scales (multiplied into the weights in the loop); otherwise one scale per column,
+// applied to the accumulators in the epilogue.
+template <int MPAD, bool GR>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a) {
   using G = TcGeometry<MPAD>;
@@ -294,11 +296,9 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
     const uint32_t len = min(KB - kb0, u1 - u);
     const uint16_t* sptr = reinterpret_cast<const uint16_t*>(p.sq) + (size_t)col * kTileN + spos;
 
-    uint32_t s2 = 0;  // {scale, scale} of this thread's column for the current k-block
-    if (!p.grouped) {
-      const uint32_t sv = __ldg(sptr);
-      s2 = sv | (sv << 16);
-    }
+    uint32_t s2 = 0;    // {scale, scale} of this thread's column for the current k-block
+    float sc_col = 1.f;  // the column's single scale
+    if constexpr (!GR) sc_col = __half2float(__ushort_as_half(__ldg(sptr)));
     for (uint32_t x = 0; x < len; ++x, ++it) {
       const int s = (int)(it % NSTAGES);
       const int slot = (int)(it % NSLOTS);
@@ -306,7 +306,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       if (tr) MARLIN_STAMP(12);
       mbar_wait(&full[s], (it / NSTAGES) & 1u, abort_flag, p.status);
       if (tr) MARLIN_STAMP(13);
-      if (p.grouped) {
+      if constexpr (GR) {
         // the scale row of the k-block came with the stage (a global read here would be a cold DRAM access)
         const uint32_t sv = lds16(smem_u32(sc_ring) + (uint32_t)s * G::SC_BYTES + (uint32_t)spos * 2);
         s2 = sv | (sv << 16);
@@ -337,8 +337,8 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
           dequant8(w[2 * hh + 1], hi);  // rows 64hh + 16c + 8..15
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            r[e] = hmul2_u32(lo[e], s2);
-            r[4 + e] = hmul2_u32(hi[e], s2);
+            r[e] = GR ? hmul2_u32(lo[e], s2) : lo[e];
+            r[4 + e] = GR ? hmul2_u32(hi[e], s2) : hi[e];
           }
           tc_st_x8(a_col + (uint32_t)(32 * hh + 8 * c), r);  // column = row / 2
         }
@@ -390,6 +390,10 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
           for (int e = 0; e < 32; ++e) part[e] += part2[e];
         } else {
           tc_wait_ld();
+        }
+        if constexpr (!GR) {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) part[e] *= sc_col;
         }
 #pragma unroll
         for (int m4 = 0; m4 < 8; ++m4) {
@@ -444,6 +448,10 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       } else {
         tc_wait_ld();
       }
+      if constexpr (!GR) {
+#pragma unroll
+        for (int e = 0; e < 32; ++e) part[e] *= sc_col;
+      }
       if (shared_tile) {
 #pragma unroll
         for (int m4 = 0; m4 < 8; ++m4)
@@ -496,10 +504,10 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
   named_bar_sync(2, kDequantThreads + 32);
 }
 
-template <int MPAD>
+template <int MPAD, bool GR>
 cudaError_t launch_tc(const GemmParams& p, int workers, cudaStream_t stream) {
   using G = TcGeometry<MPAD>;
-  auto kernel = gemm_dense_tc_kernel<MPAD>;
+  auto kernel = gemm_dense_tc_kernel<MPAD, GR>;
   static bool attr_set[64] = {};
   int dev = 0;
   cudaError_t err = cudaGetDevice(&dev);
@@ -590,9 +598,14 @@ cudaError_t launch_gemm_dense_tc(GemmParams p, int sm_count, cudaStream_t stream
   }
   p.workers = (uint32_t)workers;
   const int mpad = tc_mpad(p.M);
-  if (mpad == 32) return launch_tc<32>(p, (int)workers, stream);
-  if (mpad == 64) return launch_tc<64>(p, (int)workers, stream);
-  return launch_tc<128>(p, (int)workers, stream);
+  if (p.grouped) {
+    if (mpad == 32) return launch_tc<32, true>(p, (int)workers, stream);
+    if (mpad == 64) return launch_tc<64, true>(p, (int)workers, stream);
+    return launch_tc<128, true>(p, (int)workers, stream);
+  }
+  if (mpad == 32) return launch_tc<32, false>(p, (int)workers, stream);
+  if (mpad == 64) return launch_tc<64, false>(p, (int)workers, stream);
+  return launch_tc<128, false>(p, (int)workers, stream);
 }
 
 }  // namespace marlin_b200
