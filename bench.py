@@ -11,8 +11,9 @@ twice the L2 capacity.
 
 Prints ONE JSON line.  `value` = packed weight bytes (codes + scales) streamed per second over the
 whole step, inputs resident in HBM, timed with CUDA events around a CUDA graph of K steps.
-`e2e` = the same metric with A copied from pinned host memory and C copied back inside the timed
-region (weights stay resident: they are the model).  `roofline` is that of the dominant kernel (the
+`e2e` = the same metric with every step's A copied from pinned host memory and its C copied back inside
+the timed region (one transfer each way per step, on copy streams that overlap the neighbouring steps'
+kernels; weights stay resident: they are the model).  `roofline` is that of the dominant kernel (the
 instance that serves M = 1, 2, 4, 8): its algorithmic bytes (weights + scales + A + C, each once) per
 second of its own live launch time against the measured HBM peak, with the same figure for the whole
 step under `whole_step`.  `per_m` lists each
@@ -393,38 +394,63 @@ def run_ours(args):
             extra = extra_layers(marlin, dev, stream, l2, peaks, capture, time_graph)
 
         # ---- end to end: host buffers, copies inside the timed region ----
-        # the inputs of a step arrive in one pinned host buffer and its results leave in one: one copy each way
-        # per step (all eight activation matrices, all eight results), the eight calls in between
+        # The inputs of a step arrive in one pinned host buffer and its results leave in one: one copy each way
+        # per step (all eight activation matrices, all eight results), the eight calls in between.  Copy-in,
+        # compute and copy-out run on three streams over two sets of device buffers, so the copies of one step
+        # overlap the kernels of its neighbours; every step still copies its own inputs in and its results out.
         rows = sum(SWEEP)
         A_host = torch.empty((rows, K_DIM), dtype=torch.float16).pin_memory()
-        C_host = torch.empty((rows, N_DIM), dtype=torch.float16).pin_memory()
-        A_all = torch.empty((rows, K_DIM), dtype=torch.float16, device=dev)
-        C_all = torch.empty((rows, N_DIM), dtype=torch.float16, device=dev)
-        A_e2e, C_e2e, r0 = {}, {}, 0
+        C_host = [torch.empty((rows, N_DIM), dtype=torch.float16).pin_memory() for _ in range(2)]
+        A_all = [torch.empty((rows, K_DIM), dtype=torch.float16, device=dev) for _ in range(2)]
+        C_all = [torch.empty((rows, N_DIM), dtype=torch.float16, device=dev) for _ in range(2)]
+        A_e2e, C_e2e, r0 = [{}, {}], [{}, {}], 0
         for M in SWEEP:
             A_host[r0:r0 + M].copy_(torch.from_numpy(get(M).A))
-            A_e2e[M], C_e2e[M] = A_all[r0:r0 + M], C_all[r0:r0 + M]
+            for b in range(2):
+                A_e2e[b][M], C_e2e[b][M] = A_all[b][r0:r0 + M], C_all[b][r0:r0 + M]
             r0 += M
+        s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+        ev_in = [torch.cuda.Event() for _ in range(2)]    # inputs of the buffer set are on the device
+        ev_cmp = [torch.cuda.Event() for _ in range(2)]   # its kernels are done (A may be overwritten, C read)
+        ev_out = [torch.cuda.Event() for _ in range(2)]   # its results are on the host (C may be overwritten)
+        step_no = [0]
 
         def e2e_step():
-            A_all.copy_(A_host, non_blocking=True)
-            for M in SWEEP:
-                w, s = packed[rot[0] % copies]
-                rot[0] += 1
-                marlin.gemm(A_e2e[M], w, s, K_DIM, N_DIM, GROUP, ws, out=C_e2e[M], stream=stream)
-            C_host.copy_(C_all, non_blocking=True)
+            b = step_no[0] % 2
+            first_use = step_no[0] < 2
+            step_no[0] += 1
+            with torch.cuda.stream(s_in):
+                if not first_use:
+                    s_in.wait_event(ev_cmp[b])
+                A_all[b].copy_(A_host, non_blocking=True)
+                ev_in[b].record(s_in)
+            with torch.cuda.stream(stream):
+                stream.wait_event(ev_in[b])
+                if not first_use:
+                    stream.wait_event(ev_out[b])
+                for M in SWEEP:
+                    w, s = packed[rot[0] % copies]
+                    rot[0] += 1
+                    marlin.gemm(A_e2e[b][M], w, s, K_DIM, N_DIM, GROUP, ws, out=C_e2e[b][M], stream=stream)
+                ev_cmp[b].record(stream)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_cmp[b])
+                C_host[b].copy_(C_all[b], non_blocking=True)
+                ev_out[b].record(s_out)
 
-        with torch.cuda.stream(stream):
-            for _ in range(3):
-                e2e_step()
+        for _ in range(4):
+            e2e_step()
         torch.cuda.synchronize(dev)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        with torch.cuda.stream(stream):
-            e0.record(stream)
-            for _ in range(args.steps):
-                e2e_step()
-            e1.record(stream)
+        # the timed region starts on the copy-in stream and ends when the last results are on the host
+        e0.record(s_in)
+        for _ in range(args.steps):
+            e2e_step()
+        s_out.wait_stream(stream)
+        s_out.wait_stream(s_in)
+        e1.record(s_out)
         e1.synchronize()
+        torch.cuda.synchronize(dev)
         e2e_s = e0.elapsed_time(e1) * 1e-3 / args.steps
         h2d = sum(2 * M * K_DIM for M in SWEEP)
         d2h = sum(2 * M * N_DIM for M in SWEEP)
