@@ -17,8 +17,9 @@
  *     Every function that can fail returns a marlin_status; 0 is success.
  *   - There is no CPU path and no other-architecture path: on a device that is not compute
  *     capability 10.x the calls return MARLIN_ERR_ARCH.
- *   - Shapes: K % 128 == 0, N % 64 == 0, M >= 1.  group_size is a multiple of 128 that divides K,
- *     or K itself (also written -1): one scale per column.
+ *   - Shapes: K % 128 == 0, K <= 2^20, N % 64 == 0, N <= 65536, M >= 1 (any number of rows: a call splits
+ *     them over as many launches as it needs).  group_size is a multiple of 128 that divides K, or K itself
+ *     (also written -1): one scale per column.
  *   - The packed device layout is opaque (documented in the design doc); only marlin_pack* writes it and
  *     only marlin_unpack* / marlin_gemm* read it.
  */

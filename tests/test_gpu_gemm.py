@@ -36,6 +36,8 @@ SMALL = [
     (33, 1024, 512, 128), (64, 2048, 1024, 128), (100, 1024, 640, -1), (128, 2048, 2048, 128),
     (7, 11008, 256, 128), (1, 8192, 8192, 128), (4, 4096, 12288, 128), (16, 28672, 1024, -1),
     (16, 28672, 1024, 128), (32, 4096, 22016, 128),
+    # groups of three k-blocks (no power of two), in both kernels; more rows than one launch takes
+    (8, 1152, 256, 384), (40, 1152, 512, 384), (200, 1024, 512, 128), (150, 512, 192, 128),
 ]
 
 
