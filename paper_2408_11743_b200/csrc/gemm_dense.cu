@@ -14,11 +14,12 @@
 //                 reads its 16-byte weight vectors, turns the 4-bit codes into fp16 with the exponent-bias
 //                 trick, and feeds mma.sync.m16n8k16 with the WEIGHTS as the 16-wide operand and the batch
 //                 on the 8-wide one, so that batch sizes 1..8 cost one MMA per 256 weights.
-//                 Dense layers skip the subtraction of the bias trick: the weights enter the MMA as 1024 + q
+//                 Dense layers with up to 8 rows skip the subtraction of the bias trick: the weights enter the MMA as 1024 + q
 //                 and 64 + q, one more MMA per 16 rows of k with a constant weight operand collects
 //                 sum_k a[k] * (1032 or 72), and the difference is taken when the group closes (five ALU
-//                 instructions per eight weights instead of nine).  2:4 layers convert exactly (the
-//                 correction would depend on the metadata).
+//                 instructions per eight weights instead of nine).  With 9..16 rows the extra MMAs cost more
+//                 than they save, and 2:4 layers cannot use the trick (the correction would depend on the
+//                 metadata): both convert exactly.
 //                 The group scale is not applied to the weights: each group of k accumulates into `tmp`,
 //                 and `acc += s * (tmp - bias)` in fp32 when the group ends.
 //   end of a column segment: the groups of the CTA add their tiles through shared memory; then the fix-up
@@ -246,10 +247,13 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
 
   float acc[4 * MB][4];
   float tmp[4 * MB][4];
-  // Dense path: the weights enter the MMAs as 1024 + q and 64 + q (dequant8_biased), and bias[mb] collects
-  // sum_k a[k] * (1032 or 72) of the open group with one more MMA per 16 rows of k whose weight operand is
-  // that constant: the same number in every output channel, taken off when the group closes.
-  float bias[SP ? 1 : MB][4];
+  // Dense layers, one block of eight batch rows: the weights enter the MMAs as 1024 + q and 64 + q
+  // (dequant8_biased), and bias[mb] collects sum_k a[k] * (1032 or 72) of the open group with one more MMA per
+  // 16 rows of k whose weight operand is that constant: the same number in every output channel, taken off
+  // when the group closes.  With two blocks the MMAs are the larger part of the time and the extra ones cost
+  // more than the shorter conversion saves (measured), so those kernels convert exactly, as the 2:4 path must.
+  constexpr bool kBiased = !SP && MB == 1;
+  float bias[kBiased ? MB : 1][4];
   uint4 cur_raw = make_uint4(0, 0, 0, 0);  // 8 fp16 scales of the open group: columns 16j+g and 16j+8+g, j = 0..3
 
   auto close_group = [&]() {
@@ -260,7 +264,7 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
 #pragma unroll
       for (int mb = 0; mb < MB; ++mb) {
         const int r = j * MB + mb;
-        if constexpr (SP) {
+        if constexpr (!kBiased) {
           acc[r][0] += sc2.x * tmp[r][0];
           acc[r][1] += sc2.x * tmp[r][1];
           acc[r][2] += sc2.y * tmp[r][2];
@@ -274,7 +278,7 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
         tmp[r][0] = tmp[r][1] = tmp[r][2] = tmp[r][3] = 0.f;
       }
     }
-    if constexpr (!SP) {
+    if constexpr (kBiased) {
 #pragma unroll
       for (int mb = 0; mb < MB; ++mb) bias[mb][0] = bias[mb][1] = bias[mb][2] = bias[mb][3] = 0.f;
     }
@@ -292,7 +296,7 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
     for (int r = 0; r < 4 * MB; ++r)
 #pragma unroll
       for (int x = 0; x < 4; ++x) { acc[r][x] = 0.f; tmp[r][x] = 0.f; }
-    if constexpr (!SP) {
+    if constexpr (kBiased) {
 #pragma unroll
       for (int mb = 0; mb < MB; ++mb) bias[mb][0] = bias[mb][1] = bias[mb][2] = bias[mb][3] = 0.f;
     }
@@ -399,8 +403,13 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             uint32_t x[4], y[4];
-            dequant8_biased(X[j][2 * h + u], x);
-            dequant8_biased(Y[j][2 * h + u], y);
+            if constexpr (kBiased) {
+              dequant8_biased(X[j][2 * h + u], x);
+              dequant8_biased(Y[j][2 * h + u], y);
+            } else {
+              dequant8(X[j][2 * h + u], x);
+              dequant8(Y[j][2 * h + u], y);
+            }
             // registers 0, 1 of a fragment are its rows k < 8 (lower nibbles), 2, 3 its rows k >= 8 (upper)
             const uint32_t a0[4] = {x[0], y[0], x[1], y[1]};
             const uint32_t a1[4] = {x[2], y[2], x[3], y[3]};
@@ -410,7 +419,7 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
               mma_16816(tmp[j * MB + mb], a1, bf[mb][4 * u + 2], bf[mb][4 * u + 3]);
             }
           }
-          {
+          if constexpr (kBiased) {
             const uint32_t kc[4] = {kBiasLo, kBiasLo, kBiasHi, kBiasHi};
 #pragma unroll
             for (int mb = 0; mb < MB; ++mb) {
