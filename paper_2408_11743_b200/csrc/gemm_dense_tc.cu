@@ -328,20 +328,22 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       tc_fence_after_sync();
       const uint32_t a_col = tmem_lane + (uint32_t)(G::A_COL0 + (slot * 2 + tile) * 64);
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
+      for (int hh = 0; hh < 2; ++hh) {
+        // 64 rows of k = 32 columns of the slot, written with one store
+        uint32_t r[32];
 #pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {
-          uint32_t lo[4], hi[4], r[8];
-          dequant8(w[2 * hh], lo);      // rows 64hh + 16c + 0..7
-          dequant8(w[2 * hh + 1], hi);  // rows 64hh + 16c + 8..15
+        for (int c = 0; c < 4; ++c) {
+          const uint32_t w0 = hh == 0 ? v[c].x : v[c].z, w1 = hh == 0 ? v[c].y : v[c].w;
+          uint32_t lo[4], hi[4];
+          dequant8(w0, lo);  // rows 64hh + 16c + 0..7
+          dequant8(w1, hi);  // rows 64hh + 16c + 8..15
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            r[e] = GR ? hmul2_u32(lo[e], s2) : lo[e];
-            r[4 + e] = GR ? hmul2_u32(hi[e], s2) : hi[e];
+            r[8 * c + e] = GR ? hmul2_u32(lo[e], s2) : lo[e];
+            r[8 * c + 4 + e] = GR ? hmul2_u32(hi[e], s2) : hi[e];
           }
-          tc_st_x8(a_col + (uint32_t)(32 * hh + 8 * c), r);  // column = row / 2
         }
+        tc_st_x32(a_col + (uint32_t)(32 * hh), r);  // column = row / 2
       }
       if (tr) MARLIN_STAMP(15);
       tc_wait_st();
