@@ -20,7 +20,7 @@
  *   - Shapes: K % 128 == 0, K <= 2^20, N % 64 == 0, N <= 65536, M >= 1 (any number of rows: a call splits
  *     them over as many launches as it needs).  group_size is a multiple of 128 that divides K, or K itself
  *     (also written -1): one scale per column.
- *   - The packed device layout is opaque (documented in the design doc); only marlin_pack* writes it and
+ *   - The packed device layout is opaque (the design notes of this repository describe it); only marlin_pack* writes it and
  *     only marlin_unpack* / marlin_gemm* read it.
  */
 #ifndef MARLIN_B200_H_

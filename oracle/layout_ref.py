@@ -1,6 +1,6 @@
 """CPU restatement of the device weight layout -- TEST INFRASTRUCTURE ONLY.
 
-Written from the layout description in DESIGN.md ("Packed layout"), not from the CUDA source;
+Written from the written description of the packed layout (the design notes of this repository), not from the CUDA source;
 used only to compare bytes with what ``marlin_pack`` writes on the GPU.  Nothing in the product
 imports this file.
 
