@@ -105,7 +105,8 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
   constexpr int KH = G::KH;
   extern __shared__ __align__(128) uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem);          // [8]  TMA data of a stage has landed
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem);          // [8]  weights and scales of a stage have landed
+  uint64_t* xfull = reinterpret_cast<uint64_t*>(smem + 256);   // [8]  activation tile of a stage has landed
   uint64_t* empty = reinterpret_cast<uint64_t*>(smem + 64);    // [8]  the codes of a stage are in registers
   uint64_t* afull = reinterpret_cast<uint64_t*>(smem + 128);   // [4]  A-operand slot written
   uint64_t* mdone = reinterpret_cast<uint64_t*>(smem + 160);   // [8]  the MMAs of a stage have completed
@@ -130,6 +131,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
   if (threadIdx.x == 0) {
     for (int s = 0; s < NSTAGES; ++s) {
       mbar_init(&full[s], 1);
+      mbar_init(&xfull[s], 1);
       mbar_init(&empty[s], kDequantWarps);
       mbar_init(&mdone[s], NM);
     }
@@ -158,7 +160,9 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
       const uint64_t pol_w = policy_evict_first();
       const uint64_t pol_a = policy_evict_last();
-      const uint32_t tx_bytes = G::W_BYTES + G::A_BYTES + (p.grouped ? G::SC_BYTES : 0);
+      // weights and activations complete barriers of their own: the converting warps need only the former, and
+      // on the first pass over the ring those arrive before the dependency wait
+      const uint32_t tx_bytes = G::W_BYTES + (p.grouped ? G::SC_BYTES : 0);
       auto scale_src = [&](uint32_t col, uint32_t kb) -> const uint8_t* {
         const uint32_t gi = p.group_shift >= 0 ? (kb >> p.group_shift) : (kb / (uint32_t)p.kb_per_group);
         return p.sq + ((size_t)gi * p.N + (size_t)col * kTileN) * 2;
@@ -186,9 +190,11 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       s = pw;
       for (; u < u1 && s < NSTAGES; u += kTcProducerWarps, s += kTcProducerWarps) {
         const uint32_t col = u / KB, kb = u - col * KB;
+        if (lane == 0) mbar_expect_tx(&xfull[s], G::A_BYTES);
+        __syncwarp();
         if (lane < 2)
           tma_load_2d(stage0 + (size_t)s * G::STAGE_BYTES + lane * G::A_HALF_BYTES, &tmap_a,
-                      (int)(kb * kTileK + lane * 64), 0, &full[s], pol_a);
+                      (int)(kb * kTileK + lane * 64), 0, &xfull[s], pol_a);
       }
       uint32_t ph = 1;
       s -= NSTAGES;
@@ -202,10 +208,11 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
           mbar_expect_tx(&full[s], tx_bytes);
           bulk_g2s(st + G::A_BYTES, weight_src(col, kb), G::W_BYTES, &full[s], pol_w);
           if (p.grouped) bulk_g2s(sc_ring + (size_t)s * G::SC_BYTES, scale_src(col, kb), G::SC_BYTES, &full[s], pol_w);
+          mbar_expect_tx(&xfull[s], G::A_BYTES);
         }
         __syncwarp();
         if (lane < 2)
-          tma_load_2d(st + lane * G::A_HALF_BYTES, &tmap_a, (int)(kb * kTileK + lane * 64), 0, &full[s], pol_a);
+          tma_load_2d(st + lane * G::A_HALF_BYTES, &tmap_a, (int)(kb * kTileK + lane * 64), 0, &xfull[s], pol_a);
         s += kTcProducerWarps;
         if (s >= NSTAGES) { s -= NSTAGES; ph ^= 1u; }
       }
@@ -233,7 +240,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
           const int s = (int)(it % NSTAGES);
           const int slot = (int)(it % NSLOTS);
           if (it == 6 && mw == 0) MARLIN_STAMP(19);
-          mbar_wait(&full[s], (it / NSTAGES) & 1u, abort_flag, p.status);
+          mbar_wait(&xfull[s], (it / NSTAGES) & 1u, abort_flag, p.status);
           mbar_wait(&afull[slot], (it / NSLOTS) & 1u, abort_flag, p.status);
           if (it == 0 && mw == 0) MARLIN_STAMP(4);
           if (it == 6 && mw == 0) MARLIN_STAMP(16);
