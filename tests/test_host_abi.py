@@ -108,6 +108,22 @@ def test_stripe_partition_covers_every_unit_once(marlin, K, N, M, sms):
         assert max(sizes) - min(sizes) <= 1
 
 
+@pytest.mark.parametrize("K,N,tile,workers,form", [
+    (8192, 8192, 64, 128, "aligned"),      # one 64-column tile and all of K per CTA: no fix-up across CTAs
+    (4096, 4096, 128, 128, "aligned"),     # 32 tiles x 4 k-ranges
+    (4096, 12288, 256, 144, "aligned"),    # 48 tiles x 3 k-ranges
+    (11008, 4096, 64, 128, "aligned"),     # 64 tiles x 2 k-ranges
+    (4096, 22016, 128, 148, "even"),       # 172 tiles do not divide 148 SMs: even stripes
+    (28672, 8192, 128, 148, "even"),       # long K: idle SMs would cost more than the late finishers
+])
+def test_partition_chosen_for_the_layer_shapes_of_the_benchmarks(marlin, K, N, tile, workers, form):
+    n_tile, w, bounds = marlin.plan_stripes(1, K, N, 148)
+    assert (n_tile, w) == (tile, workers)
+    kb = K // 128
+    crosses = any(bounds[i] // kb != (bounds[i + 1] - 1) // kb for i in range(w))
+    assert crosses == (form == "even")
+
+
 def test_byte_model_matches_paper():
     from paper_2408_11743_b200 import roofline
     rows = [l.split() for l in open(os.path.join(GOLDEN, "byte_model.txt")) if l.strip() and l[0] != "#"]
