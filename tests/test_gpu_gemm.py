@@ -105,6 +105,44 @@ def test_same_layer_many_batch_sizes_and_repeatability(marlin, oracle_lib):
             assert bad == 0 and worst < 0.25
 
 
+@pytest.mark.parametrize("M,K,N,exact", [
+    (1, 4096, 4096, True),      # tile-aligned, two k-ranges per tile: thread-block clusters
+    (16, 2048, 8192, True),     # one CTA per tile, no fix-up
+    (8, 4096, 22016, True),     # even stripes, workspace fix-up, mid-stripe segments
+    (64, 8192, 8192, True),     # tcgen05 kernel, clusters of four
+    (40, 4096, 4096, False),    # tcgen05 kernel, L2 reductions (arrival order: last bit may differ)
+])
+def test_a_long_stream_of_overlapping_launches_is_stable(marlin, oracle_lib, M, K, N, exact):
+    # Consecutive launches overlap (the next kernel starts its prologue and its weight copies while the previous
+    # one drains) and share one workspace.  120 launches alternating two inputs and two outputs must give, at
+    # the end, exactly what a single launch gives.
+    import torch
+    case0 = inputs.make_dense(M, K, N, 128, seed=5 + M)
+    case1 = inputs.make_dense(M, K, N, 128, seed=6 + M)
+    layer = DenseLayer(marlin, case0.q_kpacked, case0.S, 128, max_M=M)
+    A = [to_dev(case0.A), to_dev(case1.A)]
+    want = []
+    for a in A:
+        want.append(to_host(marlin.gemm(a, layer.w, layer.s, K, N, 128, layer.ws)).copy())
+        torch.cuda.synchronize()
+    C = [torch.empty((M, N), dtype=torch.float16, device="cuda") for _ in range(2)]
+    for rep in range(3):
+        for c in C:
+            c.fill_(float("nan"))
+        for i in range(120):
+            marlin.gemm(A[i % 2], layer.w, layer.s, K, N, 128, layer.ws, out=C[i % 2])
+        torch.cuda.synchronize()
+        assert marlin.read_status(layer.ws) == 0
+        for i in range(2):
+            got = to_host(C[i])
+            if exact:
+                assert np.array_equal(got.view(np.uint16), want[i].view(np.uint16)), f"repetition {rep}, buffer {i}"
+            else:
+                bad, worst, _ = oracle_lib.check_tolerance(got, want[i])
+                assert bad == 0 and worst < 0.25
+    _assert_close(oracle_lib, to_host(C[0]), oracle_lib.gemm(case0.A, case0.q_kpacked, case0.S, 128))
+
+
 def test_zero_codes_give_zero(marlin):
     K, N = 1024, 256
     q = inputs.kpack(np.full((K, N), 8, dtype=np.uint8))

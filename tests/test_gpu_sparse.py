@@ -85,6 +85,28 @@ def test_sparse_every_partition_and_fixup_path(marlin, oracle_lib, mode, monkeyp
         assert bad == 0, f"{bad} elements out of tolerance, worst ratio {worst:.3f}, rms {rms:.3f}"
 
 
+@pytest.mark.parametrize("M,K,N", [(1, 4096, 4096), (16, 4096, 22016), (40, 2048, 1024)])
+def test_sparse_long_stream_of_overlapping_launches_is_stable(marlin, oracle_lib, M, K, N):
+    # 120 launches that overlap on the stream and share one workspace, two inputs and two outputs in turn:
+    # at the end each output holds exactly what a single launch gives (the sum order is fixed in this kernel)
+    import torch
+    case = inputs.make_sparse24(M, K, N, 128, seed=9 + M)
+    other = inputs.make_sparse24(M, K, N, 128, seed=10 + M)
+    layer = SparseLayer(marlin, case, M)
+    A = [to_dev(case.A), to_dev(other.A)]
+    want = [layer(case.A).copy(), layer(other.A).copy()]
+    C = [torch.empty((M, N), dtype=torch.float16, device="cuda") for _ in range(2)]
+    for rep in range(2):
+        for c in C:
+            c.fill_(float("nan"))
+        for i in range(120):
+            marlin.gemm_sparse24(A[i % 2], layer.w, layer.meta, layer.s, K, N, 128, layer.ws, out=C[i % 2])
+        torch.cuda.synchronize()
+        assert marlin.read_status(layer.ws) == 0
+        for i in range(2):
+            assert np.array_equal(to_host(C[i]).view(np.uint16), want[i].view(np.uint16)), f"repetition {rep}, buffer {i}"
+
+
 def test_sparse_equals_dense_kernel_on_the_expanded_matrix(marlin, oracle_lib):
     # the dense kernel on the matrix with code 8 (value 0) at the pruned positions computes the same layer
     M, K, N, G = 16, 2048, 1024, 128
