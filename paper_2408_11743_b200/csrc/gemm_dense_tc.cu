@@ -21,8 +21,9 @@
 //                 group scales, and one TMA tensor tile per 64-wide half of the activations (128-byte
 //                 swizzle = the canonical K-major UMMA layout, rows >= M zero-filled), into a ring of stages.
 //   warps 10..13  MMA issuers.  Issuing one tcgen05.mma occupies its thread for about 75 cycles, more than a
-//                 128 x 64 x 16 product takes to execute, so up to batch 64 four warps issue (tile t, half h
-//                 of the k-block, each half into an accumulator of its own); at batch 128 two.  One
+//                 128 x 64 x 16 product takes to execute, so four warps issue: up to batch 64 per tile t and half
+//                 h of the k-block (each half into an accumulator of its own), at batch 128 per tile and half of
+//                 the batch rows (N = 64).  One
 //                 tcgen05.commit per stage and warp signals that the A slot and the stage are free.  Warp 10
 //                 owns the TMEM allocation.
 //   warps 14, 15  idle (they complete the last warpgroup for setmaxnreg).
@@ -79,11 +80,15 @@ struct TcGeometry {
           : (kSmemBudget - FIXED_BYTES - ALIGN_SLACK) / STAGE_BYTES;
   static constexpr int SMEM_BYTES = FIXED_BYTES + ALIGN_SLACK + STAGES * STAGE_BYTES;
   // Issuing one tcgen05.mma occupies its thread for about 75 cycles, more than a 128 x 64 x 16 product takes
-  // to execute, so up to batch 64 four warps issue: one per 128-channel tile and half of the k-block, each
-  // half into an accumulator of its own (the epilogue adds the two).  At batch 128 execution is the longer
-  // and two warps, one per tile, are enough.
-  static constexpr int MMA_WARPS = MPAD <= 64 ? 4 : 2;
-  static constexpr int KH = MMA_WARPS / 2;                 // accumulators per tile
+  // to execute, and a commit or a wait costs the thread as much again while the pipe drains.  So four warps
+  // issue, two per 128-channel tile.  Up to batch 64 they split the k-block, each half into an accumulator of
+  // its own (the epilogue adds the two).  At batch 128 there is no room for four full accumulators: the two
+  // warps of a tile split the batch instead, 64 rows each (N = 64), which are the two halves of the tile's one
+  // 128-column accumulator.
+  static constexpr int MMA_WARPS = 4;
+  static constexpr int KH = MPAD <= 64 ? 2 : 1;            // k-halves with accumulators of their own
+  static constexpr int NH = MPAD <= 64 ? 1 : 2;            // halves of the batch per tile
+  static constexpr int MMA_N = MPAD / NH;                  // N of one MMA
   static constexpr int D_COLS = 2 * KH * MPAD;             // accumulator of (tile t, half h) at column (t * KH + h) * MPAD
   // then as many A-operand slots (2 tiles x 64 columns each) as fit in the 512 columns
   static constexpr int A_SLOTS = (kTmemCols - D_COLS) / 128 > 4 ? 4 : (kTmemCols - D_COLS) / 128;
@@ -222,12 +227,15 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       }
     } else if (warp >= kMmaWarp && warp < kMmaWarp + NM) {
       // ------------------------------- MMA issuers --------------------------------------------
-      constexpr uint32_t idesc = instr_desc_f16(128, MPAD);
+      constexpr uint32_t idesc = instr_desc_f16(128, G::MMA_N);
       constexpr int KS = 8 / KH;           // K = 16 steps per warp and stage
       const int mw = warp - kMmaWarp;
       const int t = mw & 1;                // 128-channel tile
-      const int h = mw >> 1;               // half of the k-block (always 0 with two warps)
-      const uint32_t d_tmem = tmem_base + (uint32_t)((t * KH + h) * MPAD);
+      const int h = KH == 2 ? mw >> 1 : 0;        // half of the k-block
+      const int nh = G::NH == 2 ? mw >> 1 : 0;    // half of the batch rows
+      const uint32_t d_tmem = tmem_base + (uint32_t)((t * KH + h) * MPAD + nh * G::MMA_N);
+      // rows 64 nh .. of the activation tile: eight 1024-byte groups of eight rows further on
+      const uint32_t b_rows_off = (uint32_t)(nh * G::MMA_N * 128);
       uint32_t it = 0;   // stage counter of this CTA
       uint32_t seg = 0;  // segment counter
       uint32_t u = u0;
@@ -247,7 +255,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
           tc_fence_after_sync();
           if (lane == 0) {
             // descriptor of the first K = 16 step of the stage; the others differ in the address field only
-            const uint64_t desc0 = smem_desc_k_sw128(smem_u32(stage0 + (size_t)s * G::STAGE_BYTES));
+            const uint64_t desc0 = smem_desc_k_sw128(smem_u32(stage0 + (size_t)s * G::STAGE_BYTES) + b_rows_off);
             const uint32_t a_tmem = tmem_base + (uint32_t)(G::A_COL0 + (slot * 2 + t) * 64);
 #pragma unroll
             for (int k2 = 0; k2 < KS; ++k2) {
@@ -378,15 +386,17 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       // The CTAs of this column tile form a thread-block cluster and finish side by side, so the partial
       // tiles never leave the SMs: the batch rows are dealt out to the S CTAs in blocks of four, every CTA
       // sends each block of its partial tile into the shared memory of the block's owner (the stage ring is
-      // free by now), and each owner adds the S partials of its rows in rank order and stores that part of C.
+      // free by now; these remote stores run at about 30 GB/s per SM, asynchronous ones counting on an mbarrier
+      // of the owner were slower still), and each owner adds the S partials of its rows in rank order and stores
+      // that part of C.
       // Fixed order of the fp32 sum, no atomics, no workspace.
       constexpr int R4 = MPAD / 4;              // blocks of four batch rows
       const int S = (int)p.split;
       const int rmax = (R4 + S - 1) / S;        // blocks per owner, at most
       const int r = (int)cluster_ctarank();
       cluster_sync_all();                       // all CTAs of the tile are done with their stage rings
+      if (warp == 0) MARLIN_STAMP(20);
       const uint32_t recv = smem_u32(stage0);   // [source rank][block][256 columns] float4
-      uint16_t* cptr = p.C + (size_t)col * kTileN + n256;
 #pragma unroll 1
       for (int cc = 0; cc < MPAD / 32; ++cc) {
         float part[32];
@@ -416,8 +426,13 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(dempty);
+      if (warp == 0) MARLIN_STAMP(21);
       cluster_sync_all();                       // everybody's blocks have arrived
+      if (warp == 0) MARLIN_STAMP(22);
       const int b0 = r * R4 / S, b1 = (r + 1) * R4 / S;
+      // the sums go through a row-major fp16 tile behind the receive buffer, so that C is written with 16-byte
+      // stores along its rows
+      uint16_t* out = reinterpret_cast<uint16_t*>(stage0 + (size_t)S * rmax * kTileN * 16);
       for (int blk = b0; blk < b1; ++blk) {
         const int li = blk - b0;
         float4 sum = *reinterpret_cast<const float4*>(stage0 + (size_t)((0 * rmax + li) * kTileN + n256) * 16);
@@ -425,11 +440,21 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
           const float4 v = *reinterpret_cast<const float4*>(stage0 + (size_t)((src * rmax + li) * kTileN + n256) * 16);
           sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
         }
-        const int m = 4 * blk;
-        if (m < p.M) cptr[(size_t)m * p.N] = __half_as_ushort(__float2half_rn(sum.x));
-        if (m + 1 < p.M) cptr[(size_t)(m + 1) * p.N] = __half_as_ushort(__float2half_rn(sum.y));
-        if (m + 2 < p.M) cptr[(size_t)(m + 2) * p.N] = __half_as_ushort(__float2half_rn(sum.z));
-        if (m + 3 < p.M) cptr[(size_t)(m + 3) * p.N] = __half_as_ushort(__float2half_rn(sum.w));
+        out[(4 * li + 0) * kTileN + n256] = __half_as_ushort(__float2half_rn(sum.x));
+        out[(4 * li + 1) * kTileN + n256] = __half_as_ushort(__float2half_rn(sum.y));
+        out[(4 * li + 2) * kTileN + n256] = __half_as_ushort(__float2half_rn(sum.z));
+        out[(4 * li + 3) * kTileN + n256] = __half_as_ushort(__float2half_rn(sum.w));
+      }
+      named_bar_sync(1, kDequantThreads);
+      {
+        const int rows_here = 4 * (b1 - b0);
+        for (int vec = ctid; vec < rows_here * (kTileN / 8); vec += kDequantThreads) {
+          const int row = vec / (kTileN / 8), c16 = vec % (kTileN / 8);
+          const int m = 4 * b0 + row;
+          if (m < p.M)
+            *reinterpret_cast<uint4*>(p.C + (size_t)m * p.N + (size_t)col * kTileN + c16 * 8) =
+                *reinterpret_cast<const uint4*>(out + row * kTileN + c16 * 8);
+        }
       }
       u += len;
       if (warp == 0) MARLIN_STAMP(8);
