@@ -30,9 +30,9 @@
 //
 // Partition: every column tile is cut into S k-ranges, one per CTA, where that keeps most SMs busy (one
 // epilogue per CTA, all CTAs alike); else even stripes over all units.  Fix-up of a shared tile: above 32
-// rows and when the S CTAs of every tile fit on the device as one wave of thread-block clusters, the
-// partial tiles are exchanged through distributed shared memory and every CTA finishes a share of the
-// batch rows (fixed order of the sum); otherwise every contributor adds its partial tile into an fp32 tile
+// rows and when the S CTAs of every tile fit on the device as one wave of thread-block clusters, every CTA
+// fetches its share of the batch rows from the partial tiles in the other CTAs' shared memory (fixed order
+// of the sum); otherwise every contributor adds its partial tile into an fp32 tile
 // in the workspace with L2 reductions and the last arriver stores C.  Bounded waits and programmatic
 // dependent launch are those of the small-batch kernel (gemm_dense.cu).
 #include <stdlib.h>
@@ -277,7 +277,8 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       if (mw == 0) MARLIN_STAMP(5);
     }
     if (p.cluster) {
-      // every thread of every CTA of the cluster takes part in the two barriers of the epilogue
+      // every thread of every CTA of the cluster takes part in the three barriers of the epilogue
+      cluster_sync_all();
       cluster_sync_all();
       cluster_sync_all();
     }
@@ -384,19 +385,20 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
     const bool shared_tile = last_w > first_w;
     if (p.cluster) {
       // The CTAs of this column tile form a thread-block cluster and finish side by side, so the partial
-      // tiles never leave the SMs: the batch rows are dealt out to the S CTAs in blocks of four, every CTA
-      // sends each block of its partial tile into the shared memory of the block's owner (the stage ring is
-      // free by now; these remote stores run at about 30 GB/s per SM, asynchronous ones counting on an mbarrier
-      // of the owner were slower still), and each owner adds the S partials of its rows in rank order and stores
-      // that part of C.
-      // Fixed order of the fp32 sum, no atomics, no workspace.
+      // tiles never leave the SMs.  Every CTA puts its partial tile into its own stage ring (free by now), a
+      // cluster barrier publishes them, and every CTA fetches, for its share of the batch rows (blocks of four
+      // rows are dealt out to the ranks), the S partials from the shared memory of the CTAs that hold them,
+      // adds them in rank order and stores that part of C.  Fixed order of the fp32 sum, no atomics, no
+      // workspace.  Distributed shared memory is slow here (20-30 GB/s per SM, loads and stores alike, and worse
+      // with many requests in flight), so this epilogue still costs microseconds at 128 rows; pushing the tiles
+      // with remote stores, with asynchronous remote stores, or exchanging them through the L2 under the same
+      // barriers were all slower.
       constexpr int R4 = MPAD / 4;              // blocks of four batch rows
       const int S = (int)p.split;
-      const int rmax = (R4 + S - 1) / S;        // blocks per owner, at most
       const int r = (int)cluster_ctarank();
       cluster_sync_all();                       // all CTAs of the tile are done with their stage rings
       if (warp == 0) MARLIN_STAMP(20);
-      const uint32_t recv = smem_u32(stage0);   // [source rank][block][256 columns] float4
+      const uint32_t mine_s = smem_u32(stage0); // [block of four rows][256 columns] float4
 #pragma unroll 1
       for (int cc = 0; cc < MPAD / 32; ++cc) {
         float part[32];
@@ -415,29 +417,26 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
           for (int e = 0; e < 32; ++e) part[e] *= sc_col;
         }
 #pragma unroll
-        for (int m4 = 0; m4 < 8; ++m4) {
-          const int blk = cc * 8 + m4;
-          const int owner = ((blk + 1) * S - 1) / R4;   // owner o holds blocks [o * R4 / S, (o + 1) * R4 / S)
-          const int li = blk - owner * R4 / S;
-          st_cluster_f32x4(recv + (uint32_t)(((r * rmax + li) * kTileN + n256) * 16), (uint32_t)owner, part[4 * m4],
-                           part[4 * m4 + 1], part[4 * m4 + 2], part[4 * m4 + 3]);
-        }
+        for (int m4 = 0; m4 < 8; ++m4)
+          *reinterpret_cast<float4*>(stage0 + (size_t)((cc * 8 + m4) * kTileN + n256) * 16) =
+              make_float4(part[4 * m4], part[4 * m4 + 1], part[4 * m4 + 2], part[4 * m4 + 3]);
       }
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(dempty);
       if (warp == 0) MARLIN_STAMP(21);
-      cluster_sync_all();                       // everybody's blocks have arrived
+      cluster_sync_all();                       // every CTA's partial tile is in its shared memory
       if (warp == 0) MARLIN_STAMP(22);
       const int b0 = r * R4 / S, b1 = (r + 1) * R4 / S;
-      // the sums go through a row-major fp16 tile behind the receive buffer, so that C is written with 16-byte
+      // the sums go through a row-major fp16 tile behind the partial tile, so that C is written with 16-byte
       // stores along its rows
-      uint16_t* out = reinterpret_cast<uint16_t*>(stage0 + (size_t)S * rmax * kTileN * 16);
+      uint16_t* out = reinterpret_cast<uint16_t*>(stage0 + (size_t)R4 * kTileN * 16);
       for (int blk = b0; blk < b1; ++blk) {
         const int li = blk - b0;
-        float4 sum = *reinterpret_cast<const float4*>(stage0 + (size_t)((0 * rmax + li) * kTileN + n256) * 16);
+        const uint32_t at = mine_s + (uint32_t)((blk * kTileN + n256) * 16);
+        float4 sum = ld_cluster_f32x4(at, 0u);
         for (int src = 1; src < S; ++src) {
-          const float4 v = *reinterpret_cast<const float4*>(stage0 + (size_t)((src * rmax + li) * kTileN + n256) * 16);
+          const float4 v = ld_cluster_f32x4(at, (uint32_t)src);
           sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
         }
         out[(4 * li + 0) * kTileN + n256] = __half_as_ushort(__float2half_rn(sum.x));
@@ -456,6 +455,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
                 *reinterpret_cast<const uint4*>(out + row * kTileN + c16 * 8);
         }
       }
+      cluster_sync_all();                       // nobody reads this CTA's shared memory any more
       u += len;
       if (warp == 0) MARLIN_STAMP(8);
       continue;
