@@ -1,7 +1,7 @@
 // Dense W4A16 layer for sm_100a, batch sizes 17..128 per launch: tcgen05 tensor cores with the WEIGHTS
 // as the A operand in tensor memory.
 //
-// The warp-level MMA (mma.sync) of the small-batch kernel runs at about a quarter of the tcgen05 rate on
+// The warp-level MMA (mma.sync) of the small-batch kernel runs at about a tenth of the tcgen05 rate on
 // this architecture and is out of steam above batch 16.  Here the product is computed transposed, as the
 // paper does for its sparse kernel (Section 4: C = (B^T A^T)^T): per 256-column tile of W and 128-row
 // k-block
