@@ -181,7 +181,7 @@ def run_reference(args):
 # GPU leg
 # ------------------------------------------------------------------------------------------------
 def extra_layers(marlin, dev, stream, l2, peaks, capture, time_graph):
-    """Per-layer numbers outside the timed step: Llama-2-7B shapes (dense) and the 8192^2 2:4 layer."""
+    """Per-layer numbers outside the timed step: Llama-2-7B and -70B shapes (dense) and the 8192^2 2:4 layer."""
     import torch
     out = []
     rng = np.random.default_rng(1234)
@@ -250,6 +250,14 @@ def extra_layers(marlin, dev, stream, l2, peaks, capture, time_graph):
         r = measure(8192, 8192, GROUP, M, True)
         r["layer"] = "2:4 sparse 8192x8192"
         out.append(r)
+    for name, K, N in inputs.LLAMA70B_LAYERS:
+        for M in (1, 16, 64):
+            r = measure(K, N, GROUP, M, False)
+            r["layer"] = "llama2-70b " + name
+            out.append(r)
+    r = measure(28672, 8192, 28672, 16, False)
+    r["layer"] = "llama2-70b down, one scale per column"
+    out.append(r)
     return out
 
 
