@@ -66,7 +66,7 @@ MARLIN_API size_t marlin_packed_scale_bytes(int K, int N, int group_size);
 MARLIN_API size_t marlin_packed_meta_bytes(int K, int N);
 /* Bytes of the workspace marlin_gemm* needs for any M <= max_M on this K x N layer.
  * The workspace holds a status word, per-column-tile arrival counters and the fp32 partial tiles
- * of the stripe fix-up (Section 3.4 "Striped Partitioning": the paper's "small extra lock buffer").
+ * of the stripe fix-up (the global reduction of Section 3.4 "Striped Partitioning").
  * The caller zeroes it ONCE after allocation (cudaMemset); every call leaves the counters zero.
  * One workspace must not be used by two calls that can run at the same time. */
 MARLIN_API size_t marlin_workspace_bytes(int max_M, int K, int N);
@@ -120,10 +120,14 @@ MARLIN_API int marlin_gemm(const void* A, const void* w_packed, const void* s_pa
  *
  * The first call on each device looks up the device address of that array (with that device
  * current) and remembers it; make this first call outside any stream capture.  Every call clears
- * the status word and the arrival counters of the array on `stream` before the kernels run, and
- * all calls on one device share the one array: two such calls that can overlap on the GPU (two
- * streams, or two host threads) race with each other and must be serialised by the caller.
- * Errors: as marlin_gemm; MARLIN_ERR_CUDA if the address lookup or the clearing fails. */
+ * the arrival counters of the array on `stream` before the kernels run (the array keeps whatever
+ * the previous call left), and all calls on one device share the one array: two such calls that
+ * can overlap on the GPU (two streams, or two host threads) race with each other and must be
+ * serialised by the caller.
+ * Errors: the argument checks of marlin_gemm, made before anything is queued; MARLIN_ERR_CUDA if
+ * the address lookup or the clearing fails.  The array's status word is private to the library:
+ * a bounded wait that expires inside a kernel of this entry point is NOT reported to the caller
+ * (use marlin_gemm with a workspace of your own and marlin_read_status where that matters). */
 #define MARLIN_STATIC_WS_MAX_M 16
 MARLIN_API int marlin_gemm_static_ws(const void* A, const void* w_packed, const void* s_packed, void* C,
                                      int M, int K, int N, int group_size, marlin_stream stream);

@@ -223,9 +223,16 @@ static __device__ __align__(256) unsigned char g_static_workspace[kStaticWsBytes
 
 int marlin_gemm_static_ws(const void* A, const void* w_packed, const void* s_packed, void* C, int M, int K, int N,
                           int group_size, marlin_stream stream) {
-  if (M < 1 || M > MARLIN_STATIC_WS_MAX_M) return MARLIN_ERR_SHAPE;
-  if (marlin_workspace_bytes(M, K, N) == 0) return MARLIN_ERR_SHAPE;
+  // the argument checks of marlin_gemm first: nothing is queued for a call that is going to be refused
+  if (!A || !w_packed || !s_packed || !C) return MARLIN_ERR_NULL;
+  if (M < 1 || M > MARLIN_STATIC_WS_MAX_M || !shape_ok(K, N)) return MARLIN_ERR_SHAPE;
+  if (!normalise_group(K, group_size)) return MARLIN_ERR_GROUP;
+  if (!aligned16(A) || !aligned16(w_packed) || !aligned16(s_packed) || !aligned16(C)) return MARLIN_ERR_ALIGN;
   if (marlin_workspace_bytes(M, K, N) > kStaticWsBytes) return MARLIN_ERR_WORKSPACE;
+  DeviceInfo info;
+  int st = device_info(&info);
+  if (st != MARLIN_OK) return st;
+  if (info.cc_major != 10) return MARLIN_ERR_ARCH;
   static void* device_address[64] = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MARLIN_ERR_CUDA;
@@ -235,9 +242,12 @@ int marlin_gemm_static_ws(const void* A, const void* w_packed, const void* s_pac
     if (cudaGetSymbolAddress(&ptr, g_static_workspace) != cudaSuccess || !ptr) return MARLIN_ERR_CUDA;
     device_address[dev] = ptr;
   }
-  void* ws = device_address[dev];
-  // the array keeps whatever the last call left: start from a clean status word and clean counters
-  if (cudaMemsetAsync(ws, 0, kWsPartialOff, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MARLIN_ERR_CUDA;
+  uint8_t* ws = static_cast<uint8_t*>(device_address[dev]);
+  // the array keeps whatever the last call left: the arrival counters must start at zero (the partial-tile
+  // slots behind them are written before they are read; the status word is left alone)
+  if (cudaMemsetAsync(ws + kWsCounterOff, 0, kWsPartialOff - kWsCounterOff, static_cast<cudaStream_t>(stream)) !=
+      cudaSuccess)
+    return MARLIN_ERR_CUDA;
   return marlin_gemm(A, w_packed, s_packed, C, M, K, N, group_size, ws, kStaticWsBytes, stream);
 }
 

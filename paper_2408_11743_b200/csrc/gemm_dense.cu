@@ -45,13 +45,6 @@
 namespace marlin_b200 {
 namespace {
 
-// Optional per-CTA cycle stamps for tuning (built only with -DMARLIN_TIMING; not part of the library).
-#ifdef MARLIN_TIMING
-__device__ long long g_timing[kMaxWorkers][16];
-#define MARLIN_STAMP(slot) do { if (lane == 0) g_timing[blockIdx.x][slot] = (long long)global_timer_ns(); } while (0)
-#else
-#define MARLIN_STAMP(slot) do { } while (0)
-#endif
 
 // ---------------------------------------------------------------------------------------------
 // shared memory map
@@ -127,7 +120,6 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
   const int nstages = p.stages;
 
   pdl_launch_dependents();
-  if (warp == 0) MARLIN_STAMP(10);
   if ((int)threadIdx.x < nstages) {
     mbar_init(&full[threadIdx.x], 1);
     mbar_init(&empty[threadIdx.x], NW);
@@ -139,7 +131,6 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
   }
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   __syncthreads();
-  if (warp == 0) MARLIN_STAMP(0);
 
   if (warp >= kConsumerWarps) {
     // ------------------------------- producers --------------------------------------------
@@ -186,7 +177,6 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
       }
     }
     __syncwarp();
-    MARLIN_STAMP(1 + (pw & 1));
     setmaxnreg_dec<kProducerRegs>();
     pdl_wait_prior_grids();
     u = u0 + pw;
@@ -216,7 +206,6 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
       s += kProducerWarps;
       if (s >= nstages) { s -= nstages; ph ^= 1u; }
     }
-    if (pw == 0) MARLIN_STAMP(3);
     if (*abort_flag) {
       // give copies that may still be in flight time to land before the CTA's shared memory goes away
       for (int x = 0; x < 1000; ++x) __nanosleep(1000);
@@ -234,7 +223,6 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
   // From here on this kernel writes C and the workspace, which the previous kernel of the stream
   // may still be using: wait until it has finished and its memory is visible.
   pdl_wait_prior_grids();
-  if (warp == 0) MARLIN_STAMP(11);
   const int grp = warp / NW;
   const int wn = warp % NW;
   const int g = lane >> 2, c = lane & 3;
@@ -326,7 +314,6 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
           cur_group = gi;
         }
       }
-      if (warp == 0 && x == off && it0 == 0) MARLIN_STAMP(4);
       const uint8_t* st = stage0 + (size_t)s * G::STAGE_BYTES;
       const uint32_t st_s = stage0_s + (uint32_t)s * G::STAGE_BYTES;  // the same as a shared-space address
       if constexpr (SP) {
@@ -436,8 +423,6 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
       if (s >= nstages) { s -= nstages; ph ^= 1u; }
     }
     if (cur_group >= 0) close_group();
-    if (warp == 0) MARLIN_STAMP(5);
-    if (warp == kConsumerWarps - 1) MARLIN_STAMP(6);
 
     // ---- reduce the SK groups of this CTA (the last step of Algorithm 1) ----
     // Every group but the first parks its tile in shared memory; after one barrier group 0 adds them to its
@@ -461,7 +446,6 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
     }
     named_bar_sync(1, kConsumerThreads);  // `red` may be written again
 
-    if (warp == 0) MARLIN_STAMP(7);
     // ---- stripe fix-up across CTAs and output ----
     const int first_w = p.split ? (int)(col * p.split) : (int)stripe_owner32(col * KB, U, P);
     const int last_w = p.split ? (int)(col * p.split + p.split - 1) : (int)stripe_owner32((col + 1) * KB - 1, U, P);
@@ -664,9 +648,7 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
 
     u += len;
     it0 += len;
-    if (warp == 0) MARLIN_STAMP(8);
   }
-  if (warp == 0) MARLIN_STAMP(9);
   if (*abort_flag) {
     // a wait gave up: copies may still be in flight towards this CTA's shared memory
     for (int x = 0; x < 1000; ++x) __nanosleep(1000);
@@ -770,11 +752,6 @@ void fill_geometry(DensePlan* plan) {
 
 }  // namespace
 
-#ifdef MARLIN_TIMING
-extern "C" __attribute__((visibility("default"))) int marlin_timing_read(void* host) {
-  return (int)cudaMemcpyFromSymbol(host, g_timing, sizeof(g_timing));
-}
-#endif
 
 #define MARLIN_DISPATCH(MBV, NWV, STMT)         \
   if (plan_mb == MBV && plan_nw == NWV) { STMT; }

@@ -44,12 +44,6 @@
 namespace marlin_b200 {
 namespace {
 
-#ifdef MARLIN_TIMING
-__device__ long long g_timing_tc[kMaxWorkers][24];
-#define MARLIN_STAMP(slot) do { if (lane == 0) g_timing_tc[blockIdx.x][slot] = (long long)global_timer_ns(); } while (0)
-#else
-#define MARLIN_STAMP(slot) do { } while (0)
-#endif
 
 // ---------------------------------------------------------------------------------------------
 // geometry
@@ -132,7 +126,6 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
   const uint32_t u1 = p.split ? split_begin32(worker + 1, KB, p.split) : stripe_begin32(worker + 1, U, P);
 
   pdl_launch_dependents();
-  if (warp == 0) MARLIN_STAMP(10);
   if (threadIdx.x == 0) {
     for (int s = 0; s < NSTAGES; ++s) {
       mbar_init(&full[s], 1);
@@ -155,7 +148,6 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_base_slot;
-  if (warp == 0) MARLIN_STAMP(0);
 
   if (warp >= kDequantWarps) {
     setmaxnreg_dec<kAuxRegs>();
@@ -188,9 +180,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         }
       }
       __syncwarp();
-      if (pw == 0) MARLIN_STAMP(1);
       pdl_wait_prior_grids();
-      if (pw == 0) MARLIN_STAMP(11);
       u = u0 + pw;
       s = pw;
       for (; u < u1 && s < NSTAGES; u += kTcProducerWarps, s += kTcProducerWarps) {
@@ -221,7 +211,6 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         s += kTcProducerWarps;
         if (s >= NSTAGES) { s -= NSTAGES; ph ^= 1u; }
       }
-      if (pw == 0) MARLIN_STAMP(3);
       if (*abort_flag) {
         for (int x = 0; x < 1000; ++x) __nanosleep(1000);
       }
@@ -247,11 +236,8 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         for (uint32_t x = 0; x < len; ++x, ++it) {
           const int s = (int)(it % NSTAGES);
           const int slot = (int)(it % NSLOTS);
-          if (it == 6 && mw == 0) MARLIN_STAMP(19);
           mbar_wait(&xfull[s], (it / NSTAGES) & 1u, abort_flag, p.status);
           mbar_wait(&afull[slot], (it / NSLOTS) & 1u, abort_flag, p.status);
-          if (it == 0 && mw == 0) MARLIN_STAMP(4);
-          if (it == 6 && mw == 0) MARLIN_STAMP(16);
           tc_fence_after_sync();
           if (lane == 0) {
             // descriptor of the first K = 16 step of the stage; the others differ in the address field only
@@ -263,18 +249,15 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
               const uint64_t bdesc = desc0 + (uint64_t)(((ks >> 2) * G::A_HALF_BYTES + (ks & 3) * 32) >> 4);
               tc_mma_ts(d_tmem, a_tmem + ks * 8, bdesc, idesc, (x == 0 && k2 == 0) ? 0u : 1u);
             }
-            if (it == 6 && mw == 0) MARLIN_STAMP(17);
             // one arrival when these MMAs are done: the A slot may be rewritten, the activation tile refilled
             tc_commit(&mdone[s]);
             if (x + 1 == len) tc_commit(dfull);
-            if (it == 6 && mw == 0) MARLIN_STAMP(18);
           }
           __syncwarp();
         }
         u += len;
         ++seg;
       }
-      if (mw == 0) MARLIN_STAMP(5);
     }
     if (p.cluster) {
       // every thread of every CTA of the cluster takes part in the three barriers of the epilogue
@@ -318,10 +301,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
     for (uint32_t x = 0; x < len; ++x, ++it) {
       const int s = (int)(it % NSTAGES);
       const int slot = (int)(it % NSLOTS);
-      const bool tr = (warp == 0 && it == 6);
-      if (tr) MARLIN_STAMP(12);
       mbar_wait(&full[s], (it / NSTAGES) & 1u, abort_flag, p.status);
-      if (tr) MARLIN_STAMP(13);
       if constexpr (GR) {
         // the scale row of the k-block came with the stage (a global read here would be a cold DRAM access)
         const uint32_t sv = lds16(smem_u32(sc_ring) + (uint32_t)s * G::SC_BYTES + (uint32_t)spos * 2);
@@ -340,7 +320,6 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         const uint32_t jt = it - NSLOTS;
         mbar_wait(&mdone[jt % NSTAGES], (jt / NSTAGES) & 1u, abort_flag, p.status);
       }
-      if (tr) MARLIN_STAMP(14);
       tc_fence_after_sync();
       const uint32_t a_col = tmem_lane + (uint32_t)(G::A_COL0 + (slot * 2 + tile) * 64);
 #pragma unroll
@@ -361,18 +340,14 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         }
         tc_st_x32(a_col + (uint32_t)(32 * hh), r);  // column = row / 2
       }
-      if (tr) MARLIN_STAMP(15);
       tc_wait_st();
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(&afull[slot]);
-      if (tr) MARLIN_STAMP(2);
     }
 
     // ---- segment end: read the accumulators, fix-up across CTAs, store C ----
-    if (warp == 0) MARLIN_STAMP(6);
     mbar_wait(dfull, seg & 1u, abort_flag, p.status);
-    if (warp == 0) MARLIN_STAMP(7);
     tc_fence_after_sync();
     ++seg;
     if (!waited_for_prior_grid) {
@@ -397,7 +372,6 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       const int S = (int)p.split;
       const int r = (int)cluster_ctarank();
       cluster_sync_all();                       // all CTAs of the tile are done with their stage rings
-      if (warp == 0) MARLIN_STAMP(20);
       const uint32_t mine_s = smem_u32(stage0); // [block of four rows][256 columns] float4
 #pragma unroll 1
       for (int cc = 0; cc < MPAD / 32; ++cc) {
@@ -424,9 +398,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(dempty);
-      if (warp == 0) MARLIN_STAMP(21);
       cluster_sync_all();                       // every CTA's partial tile is in its shared memory
-      if (warp == 0) MARLIN_STAMP(22);
       const int b0 = r * R4 / S, b1 = (r + 1) * R4 / S;
       // the sums go through a row-major fp16 tile behind the partial tile, so that C is written with 16-byte
       // stores along its rows
@@ -457,7 +429,6 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       }
       cluster_sync_all();                       // nobody reads this CTA's shared memory any more
       u += len;
-      if (warp == 0) MARLIN_STAMP(8);
       continue;
     }
     // The column tile may be shared by several CTAs.  With up to 128 rows a partial tile is large and
@@ -530,9 +501,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       named_bar_sync(1, kDequantThreads);  // last_flag may be rewritten by the next segment
     }
     u += len;
-    if (warp == 0) MARLIN_STAMP(8);
   }
-  if (warp == 0) MARLIN_STAMP(9);
   // everybody is done with tensor memory
   tc_fence_before_sync();
   named_bar_sync(2, kDequantThreads + 32);
@@ -591,11 +560,6 @@ cudaError_t launch_tc(const GemmParams& p, int workers, cudaStream_t stream) {
 
 }  // namespace
 
-#ifdef MARLIN_TIMING
-extern "C" __attribute__((visibility("default"))) int marlin_timing_read_tc(void* host) {
-  return (int)cudaMemcpyFromSymbol(host, g_timing_tc, sizeof(g_timing_tc));
-}
-#endif
 
 bool tc_path_supported(int m_slab, int K, int N) {
   return m_slab >= 1 && m_slab <= kTcMaxSlabM && N % kTileN == 0 && K % kTileK == 0;

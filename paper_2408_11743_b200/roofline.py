@@ -35,7 +35,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 
 def load_peaks(root: str):
-    """Measured peaks of this machine (generated file), else the stated fallback."""
+    """Measured peaks (HBM copy GB/s, bf16 GEMM TFLOP/s) from MEASURED_PEAKS.json beside the benchmark, else a stated fallback."""
     path = os.path.join(root, "MEASURED_PEAKS.json")
     try:
         with open(path) as f:

@@ -188,6 +188,59 @@ def test_one_hot_rows_probe_every_k_position(marlin, oracle_lib):
         assert np.array_equal(C, want)
 
 
+# Exact-answer tests on the large-batch kernels (17 rows and more per launch), in every partition and fix-up
+# those kernels have: the default, even stripes, and the reduction through the workspace instead of clusters.
+LARGE_BATCH_MODES = [{}, {"MARLIN_B200_TC_SPLIT": "0", "MARLIN_B200_SPLIT": "0"},
+                     {"MARLIN_B200_TC_CLUSTER": "0", "MARLIN_B200_CLUSTER": "0"}]
+
+
+@pytest.mark.parametrize("mode", range(len(LARGE_BATCH_MODES)))
+@pytest.mark.parametrize("M,K,N,G", [(33, 1024, 256, 128), (64, 2048, 512, 128), (128, 4096, 1024, -1),
+                                     (17, 1024, 512, 256), (48, 2048, 256, -1)])
+def test_integer_closed_form_is_bit_exact_on_the_large_batch_kernels(marlin, oracle_lib, monkeypatch, mode, M, K, N, G):
+    # powers of two as scales and small integers as activations: every product and every partial sum is an
+    # integer multiple of the scale below 2^24, so fp32 sums are exact in ANY order (also the arrival order of
+    # the reductions at the L2) and the result must equal the oracle bit for bit
+    for k, v in LARGE_BATCH_MODES[mode].items():
+        monkeypatch.setenv(k, v)
+    rng = np.random.default_rng(7 * M + K + N)
+    Q = rng.integers(0, 16, size=(K, N), dtype=np.uint8)
+    A = rng.integers(-3, 4, size=(M, K)).astype(np.float16)
+    Gn = K if G == -1 else G
+    S = np.ldexp(1.0, rng.integers(-4, 1, size=(K // Gn, N))).astype(np.float16)
+    q = inputs.kpack(Q)
+    C = DenseLayer(marlin, q, S, G, max_M=M)(A)
+    C_ref = oracle_lib.gemm(A, q, S, Gn)
+    assert np.array_equal(C.view(np.uint16), C_ref.view(np.uint16))
+
+
+@pytest.mark.parametrize("mode", range(len(LARGE_BATCH_MODES)))
+@pytest.mark.parametrize("N", [256, 512])
+def test_one_hot_rows_probe_every_k_position_on_the_large_batch_kernels(marlin, monkeypatch, mode, N):
+    # 128 unit vectors at a time: C[m, n] = (Q[k_m, n] - 8) * S[k_m // G, n] exactly, for every k of the layer;
+    # a wrong operand descriptor, k order or scale group shows as a wrong entry
+    for k, v in LARGE_BATCH_MODES[mode].items():
+        monkeypatch.setenv(k, v)
+    K, G = 1024, 128
+    rng = np.random.default_rng(11 + N)
+    Q = rng.integers(0, 16, size=(K, N), dtype=np.uint8)
+    expo = rng.integers(-5, 2, size=(K // G, N))
+    S = np.ldexp(1.0, expo).astype(np.float16)
+    layer = DenseLayer(marlin, inputs.kpack(Q), S, G, max_M=128)
+    for k0 in range(0, K, 128):
+        A = np.zeros((128, K), dtype=np.float16)
+        A[np.arange(128), k0 + np.arange(128)] = 1.0
+        C = layer(A).astype(np.float64)
+        want = (Q[k0:k0 + 128].astype(np.float64) - 8) * np.ldexp(1.0, expo[k0 // G])[None, :]
+        assert np.array_equal(C, want), f"k-block {k0 // 128}"
+    # the same with fewer rows (other instances of the kernels): rows = the first 40 / 64 unit vectors of a block
+    for M in (40, 64):
+        A = np.zeros((M, K), dtype=np.float16)
+        A[np.arange(M), 300 + np.arange(M)] = 1.0
+        want = np.stack([(Q[300 + i].astype(np.float64) - 8) * np.ldexp(1.0, expo[(300 + i) // G]) for i in range(M)])
+        assert np.array_equal(layer(A).astype(np.float64), want), f"M = {M}"
+
+
 def test_subnormal_scales_and_large_values(marlin, oracle_lib):
     K, N = 1024, 128
     case = inputs.make_dense(4, K, N, 128, seed=9)

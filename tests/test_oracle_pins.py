@@ -345,3 +345,31 @@ def test_generator_recipe_and_seeds():
     cases = list(inputs.iter_cases(4))
     assert len(cases) == 3 * 2 * 4 and len({c[-1] for c in cases}) == len(cases)
     assert list(inputs.iter_cases(1)) == [("single", 16, 4096, 4096, 128, 0)]
+
+
+def test_sparse24_literal_case_typed_out_by_hand(oracle_lib):
+    # Section 2.2 / Section 4: in every group of four consecutive rows of a column two values are kept, each with
+    # its 2-bit position inside the group; everything else is zero.  K = 16, N = 2, scale groups of 8 rows.
+    # Every number below was written out by hand from that definition (no formula of the oracle is re-used).
+    #
+    # kept values (code, position) in the order they are stored, four groups per column:
+    #   column 0: (15,1) (0,3) | (9,0) (6,2) | (8,0) (11,3) | (7,1) (8,2)
+    #   column 1: (8,0) (12,1) | (3,2) (10,3) | (15,1) (1,2) | (0,0) (9,3)
+    qc = np.array([[0x87B8690F, 0x901FA3C8]], dtype=np.uint32)   # nibble t of a word = code of kept value t
+    idx = np.array([[1, 0], [3, 1], [0, 2], [2, 3], [0, 1], [3, 2], [1, 0], [2, 3]], dtype=np.uint8)
+    # the dense codes this stands for (8 = the zero code at pruned positions)
+    Q = np.array([[8, 8], [15, 12], [8, 8], [0, 8],
+                  [9, 8], [8, 8], [6, 3], [8, 10],
+                  [8, 8], [8, 15], [8, 1], [11, 8],
+                  [8, 0], [7, 8], [8, 8], [8, 9]], dtype=np.uint8)
+    assert np.array_equal(oracle_lib.sparse24_expand(qc, idx), Q)
+    S = np.array([[0.5, 0.25], [2.0, 1.0]], dtype=np.float16)
+    A = np.array([[1, 2, 3, 4, 5, 6, 7, 8, 1, 1, 1, 1, 2, 2, 2, 2],
+                  [-1, 0, 0, 0.5, 0, 0, 0, -2, 0, 0, 3, 0, 0, -1, 0, 0.25]], dtype=np.float16)
+    # row 0, column 0: 0.5 * (2*7 + 4*(-8) + 5*1 + 7*(-2)) + 2 * (1*3 + 2*(-1)) = -13.5 + 2 = -11.5
+    # row 0, column 1: 0.25 * (2*4 + 7*(-5) + 8*2) + 1 * (7 - 7 + 2*(-8) + 2*1) = -2.75 - 14 = -16.75
+    # row 1, column 0: 0.5 * (0.5*(-8)) + 2 * ((-1)*(-1)) = -2 + 2 = 0
+    # row 1, column 1: 0.25 * ((-2)*2) + 1 * (3*(-7) + 0.25*1) = -1 - 20.75 = -21.75
+    want = np.array([[-11.5, -16.75], [0.0, -21.75]])
+    got = oracle_lib.gemm_sparse24(A, qc, idx, S, 8).astype(np.float64)
+    assert np.array_equal(got, want)
