@@ -61,6 +61,15 @@ int tc_min_m() {
   return v;
 }
 
+// The tcgen05 kernel with deferred scales and 128-column tiles (gemm_tcd.cu) takes the layers whose N is a
+// multiple of 128 but not of 256 at batch sizes above 16.  MARLIN_B200_TCD (tuning knob): 0 switches it off
+// (slabs of 16 rows through the warp-level kernel instead), 1 makes it take every batch size on every layer
+// whose N is a multiple of 128 (64 rows per launch).
+int tcd_mode() {
+  const char* e = getenv("MARLIN_B200_TCD");  // read at every call, like the other tuning knobs
+  return !e ? 2 : (atoi(e) == 0 ? 0 : 1);     // 0 off, 1 everywhere, 2 default
+}
+
 }  // namespace
 
 extern "C" {
@@ -99,9 +108,15 @@ size_t marlin_packed_meta_bytes(int K, int N) {
 // Workspace map: [status word, counters: 8192 bytes][partial-tile slots of the warp-MMA kernel]
 // ... [fp32 accumulation tiles of the tcgen05 kernel, placed at the END of the buffer].  Everything is
 // zero at rest; both kernels leave it that way.
-static size_t mma_slot_bytes(int /*max_M*/) {
-  // two slots per worker, each the widest partial tile of the small-batch kernels: 16 rows x 256 columns
-  return (size_t)2 * kMaxWorkers * kWsSlotCols * kMaxSlabM * sizeof(float);
+static size_t mma_slot_bytes(int max_M, int N) {
+  // two slots per worker, each the widest partial tile of the warp-level kernel: 16 rows x 256 columns
+  size_t b = (size_t)2 * kMaxWorkers * kWsSlotCols * kMaxSlabM * sizeof(float);
+  // the tcgen05 kernel with deferred scales: 128 columns x 16, 32 or 64 rows
+  if (tcd_mode() != 0 && N % 128 == 0) {
+    const size_t t = (size_t)2 * kMaxWorkers * tcd_slot_floats(max_M < kTcdMaxSlabM ? max_M : kTcdMaxSlabM) * sizeof(float);
+    if (t > b) b = t;
+  }
+  return b;
 }
 static size_t tc_tile_bytes(int max_M, int N) {
   if (max_M < tc_min_m() || N % 256) return 0;
@@ -110,7 +125,7 @@ static size_t tc_tile_bytes(int max_M, int N) {
 
 size_t marlin_workspace_bytes(int max_M, int K, int N) {
   if (max_M < 1 || !shape_ok(K, N)) return 0;
-  return kWsPartialOff + mma_slot_bytes(max_M) + tc_tile_bytes(max_M, N);
+  return kWsPartialOff + mma_slot_bytes(max_M, N) + tc_tile_bytes(max_M, N);
 }
 
 int marlin_pack(const uint32_t* q_kpacked, const void* scales, void* w_packed, void* s_packed, int K, int N,
@@ -164,8 +179,17 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
   int m0 = 0;
   while (m0 < M) {
     const int rem = M - m0;
-    const bool use_tc = !sparse24 && rem >= tc_min_m() && tc_path_supported(rem < kTcMaxSlabM ? rem : kTcMaxSlabM, K, N);
-    const int m_slab = use_tc ? (rem < kTcMaxSlabM ? rem : kTcMaxSlabM) : (rem < kMaxSlabM ? rem : kMaxSlabM);
+    // Which kernel takes the next rows.  Up to 16: the warp-level kernel.  Above: the tcgen05 kernel with
+    // in-loop scales (128 rows per launch, N a multiple of 256), or the one with deferred scales (64 rows per
+    // launch, N a multiple of 128).  What none of them serves (2:4 layers, other N) goes through the warp-level
+    // kernel in slabs of 16 rows.
+    const int tmode = tcd_mode();
+    const bool tc_ok = !sparse24 && tc_path_supported(1, K, N);
+    const bool use_tcd = !sparse24 && tcd_path_supported(1, K, N) &&
+                         (tmode == 1 || (tmode == 2 && rem >= tc_min_m() && !tc_ok));
+    const bool use_tc = !use_tcd && tc_ok && rem >= tc_min_m();
+    const int m_slab = use_tcd ? (rem < kTcdMaxSlabM ? rem : kTcdMaxSlabM)
+                               : use_tc ? (rem < kTcMaxSlabM ? rem : kTcMaxSlabM) : (rem < kMaxSlabM ? rem : kMaxSlabM);
     GemmParams p;
     p.A = static_cast<const uint16_t*>(A) + (size_t)m0 * K;
     p.wq = static_cast<const uint8_t*>(w_packed);
@@ -189,7 +213,9 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
     p.split = 0;
     p.cluster = 0;
     p.slot_floats = kWsSlotCols * kMaxSlabM;
-    if (use_tc) {
+    if (use_tcd) {
+      if (launch_gemm_tcd(p, info.sm_count, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MARLIN_ERR_CUDA;
+    } else if (use_tc) {
       if (launch_gemm_dense_tc(p, info.sm_count, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return MARLIN_ERR_CUDA;
     } else {

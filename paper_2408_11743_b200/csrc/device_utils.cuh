@@ -105,6 +105,15 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, i
       ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(pol)
       : "memory");
 }
+// One box of a 3-D tensor map -> shared memory
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, int x, int y, int z, uint64_t* bar,
+                                            uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%2, %3, %4}], [%5], %6;"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar)), "l"(pol)
+      : "memory");
+}
 __device__ __forceinline__ int atom_add_acq_rel_gpu(int* addr, int v) {
   int old;
   asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(addr), "r"(v) : "memory");
@@ -192,6 +201,14 @@ __device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4],
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+// four 8 x 8 matrices of 16-bit elements from shared memory: lanes 8i .. 8i + 7 give the row addresses of matrix i,
+// register i of every lane receives its two elements of matrix i (the m16n8k16 operand order)
+__device__ __forceinline__ void ldmatrix_x4(uint32_t saddr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(saddr));
+}
+
 // 2:4 sparse MMA: A = 16 x 32 with 16 stored values per row (the usual 16 x 16 A fragment), B = 32 x 8,
 // E = metadata word of the lanes the selector names (lane % 4 in {0, 1} for selector 0, {2, 3} for 1):
 // nibble x of that lane's word = positions (first | second << 2) of the two kept values of row
@@ -243,5 +260,8 @@ __device__ __forceinline__ float4 ld_cg_f4(const float4* p) { return __ldcg(p); 
 
 // tensor maps are built through the runtime's driver entry point (no link against libcuda)
 bool make_a_tensor_map(CUtensorMap* map, const void* A, int M, int K, int box_rows);
+// A[M][K] as a 3-D tensor (64 columns, M rows, K / 64 column blocks): one box of 64 x box_rows x 2 brings both
+// 64-wide halves of a 128-row k-block, each as a 128-byte-swizzled tile of box_rows rows, one after the other
+bool make_a_tensor_map_3d(CUtensorMap* map, const void* A, int M, int K, int box_rows);
 
 }  // namespace marlin_b200

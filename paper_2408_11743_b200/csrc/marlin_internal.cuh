@@ -26,7 +26,8 @@ constexpr int kProducerRegs = 40;
 constexpr int kMaxStages = 32;
 constexpr int kMaxWorkers = 160;      // grid size cap (a B200 has 148 SMs)
 constexpr int kMaxSlabM = 16;         // rows of A handled by one launch of the mma.sync kernel
-constexpr int kTcMaxSlabM = 128;      // rows of A handled by one launch of the tcgen05 kernel
+constexpr int kTcMaxSlabM = 128;      // rows of A handled by one launch of the tcgen05 kernel with in-loop scales
+constexpr int kTcdMaxSlabM = 64;      // rows of A handled by one launch of the tcgen05 kernel with deferred scales
 constexpr int kSmemBudget = 227 * 1024;
 
 // workspace layout (bytes)
@@ -88,6 +89,12 @@ bool tc_path_supported(int m_slab, int K, int N);
 int tc_mpad(int m_slab);  // rows of A padded to the MMA's N: 32, 64 or 128
 // fills the plan fields of `p` (ncols, units, workers) itself
 cudaError_t launch_gemm_dense_tc(GemmParams p, int sm_count, cudaStream_t stream);
+// tcgen05 kernel with deferred scales (gemm_tcd.cu): 128-column tiles, up to 64 rows of A per launch.
+bool tcd_path_supported(int m_slab, int K, int N);
+int tcd_mpad(int m_slab);            // rows of A padded to the MMA's N: 16, 32 or 64
+size_t tcd_slot_floats(int m_slab);  // floats of one partial-tile slot of the fix-up
+// fills the plan fields of `p` (ncols, units, workers, slot_floats) itself
+cudaError_t launch_gemm_tcd(GemmParams p, int sm_count, cudaStream_t stream);
 // inverse == false: (q, s) canonical inputs -> (wq, sq) packed outputs; inverse == true: the other way round.
 cudaError_t launch_pack_dense(uint32_t* q, uint16_t* s, uint32_t* wq, uint16_t* sq, int K, int N, int G, bool inverse,
                               cudaStream_t stream);
