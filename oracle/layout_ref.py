@@ -72,9 +72,46 @@ def _chunk_order(KB, NB):
     return order
 
 
+# Layers whose N is a multiple of 256 use the WIDE layout (read by the tcgen05 kernel).  Records in the order
+# T * (K/128) + kb for the 256-column tile T and the k-block kb:
+#   codes (2048 words): word ((c*256 + n)*4 + w) holds kept values e = 32c + 8w + o (o = 0..7) of column 256T + n, value o in
+#     nibble (o >> 1) + 4(o & 1); kept value e of the k-block is kept row 64kb + e.
+#   metadata (1024 words): word ((128t + L)*4 + i) with L = 16a + 8h + r: bits 0-15 describe column 256T + 128t + 16a + r,
+#     bits 16-31 column 256T + 128t + 16a + 8 + r; the four 4-bit entries of each half are idx_first | idx_second << 2 of the
+#     groups 8i + 4h + 0..3 of the k-block's 32 groups of four original rows.
+
+def _wide_sparse_codes(Qc: np.ndarray, K: int) -> np.ndarray:
+    N = Qc.shape[1]
+    KB, NT = K // 128, N // 256
+    T, kb, c, n, w, o = np.meshgrid(np.arange(NT), np.arange(KB), np.arange(2), np.arange(256), np.arange(4), np.arange(8),
+                                    indexing="ij")
+    codes = Qc[64 * kb + 32 * c + 8 * w + o, 256 * T + n].astype(np.uint32)
+    words = np.zeros(codes.shape[:-1], dtype=np.uint32)
+    for oo in range(8):
+        words |= codes[..., oo] << np.uint32(4 * ((oo >> 1) + 4 * (oo & 1)))
+    return words.reshape(-1)
+
+
+def _wide_sparse_meta(idx: np.ndarray, K: int) -> np.ndarray:
+    N = idx.shape[1]
+    KB, NT = K // 128, N // 256
+    T, kb, t, a, h, r, i, hw, gq = np.meshgrid(np.arange(NT), np.arange(KB), np.arange(2), np.arange(8), np.arange(2),
+                                               np.arange(8), np.arange(4), np.arange(2), np.arange(4), indexing="ij")
+    col = 256 * T + 128 * t + 16 * a + 8 * hw + r
+    g2 = 2 * (32 * kb + 8 * i + 4 * h + gq)
+    nib = idx[g2, col].astype(np.uint32) | (idx[g2 + 1, col].astype(np.uint32) << np.uint32(2))
+    words = np.zeros(nib.shape[:-2], dtype=np.uint32)
+    for hh in range(2):
+        for gg in range(4):
+            words |= nib[..., hh, gg] << np.uint32(16 * hh + 4 * gg)
+    return words.reshape(-1)  # order [T, kb, t, a, h, r, i] = record, lane 16a + 8h + r of half t, step i
+
+
 def pack_sparse_codes(Qc: np.ndarray, K: int) -> np.ndarray:
     """Kept codes Qc[K/2, N] (uint8) -> packed uint32 words (K*N/16)."""
     N = Qc.shape[1]
+    if N % 256 == 0:
+        return _wide_sparse_codes(Qc, K)
     KB, NB = K // 128, N // 64
     kb, nb, j, g, c, t, p = np.meshgrid(np.arange(KB), np.arange(NB), np.arange(4), np.arange(8), np.arange(4),
                                         np.arange(4), np.arange(8), indexing="ij")
@@ -96,6 +133,8 @@ def pack_sparse_codes(Qc: np.ndarray, K: int) -> np.ndarray:
 def pack_sparse_meta(idx: np.ndarray, K: int) -> np.ndarray:
     """Positions idx[K/2, N] (uint8, 0..3) -> packed uint32 metadata words (K*N/32)."""
     N = idx.shape[1]
+    if N % 256 == 0:
+        return _wide_sparse_meta(idx, K)
     KB, NB = K // 128, N // 64
     kb, nb, jh, g, c, jl, w, x = np.meshgrid(np.arange(KB), np.arange(NB), np.arange(2), np.arange(8), np.arange(4),
                                              np.arange(2), np.arange(2), np.arange(8), indexing="ij")

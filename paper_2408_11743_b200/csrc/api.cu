@@ -118,14 +118,21 @@ static size_t mma_slot_bytes(int max_M, int N) {
   }
   return b;
 }
-static size_t tc_tile_bytes(int max_M, int N) {
-  if (max_M < tc_min_m() || N % 256) return 0;
+// sparse24: 2:4 layers on the wide layout run on the tcgen05 kernel at every batch size
+static size_t tc_tile_bytes(int max_M, int N, bool sparse24) {
+  if ((!sparse24 && max_M < tc_min_m()) || N % 256) return 0;
   return (size_t)N * (size_t)tc_mpad(max_M < kTcMaxSlabM ? max_M : kTcMaxSlabM) * sizeof(float);
+}
+static size_t workspace_bytes_for(int max_M, int K, int N, bool sparse24) {
+  (void)K;
+  return kWsPartialOff + mma_slot_bytes(max_M, N) + tc_tile_bytes(max_M, N, sparse24);
 }
 
 size_t marlin_workspace_bytes(int max_M, int K, int N) {
   if (max_M < 1 || !shape_ok(K, N)) return 0;
-  return kWsPartialOff + mma_slot_bytes(max_M, N) + tc_tile_bytes(max_M, N);
+  // the larger of what a dense and a 2:4 layer of this shape need (the query does not know which it will be)
+  const size_t d = workspace_bytes_for(max_M, K, N, false), sp = workspace_bytes_for(max_M, K, N, true);
+  return d > sp ? d : sp;
 }
 
 int marlin_pack(const uint32_t* q_kpacked, const void* scales, void* w_packed, void* s_packed, int K, int N,
@@ -169,7 +176,7 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
   if (!aligned16(A) || !aligned16(w_packed) || !aligned16(s_packed) || !aligned16(C) || !aligned16(workspace) ||
       (sparse24 && !aligned16(meta_packed)))
     return MARLIN_ERR_ALIGN;
-  if (workspace_bytes < marlin_workspace_bytes(M, K, N)) return MARLIN_ERR_WORKSPACE;
+  if (workspace_bytes < workspace_bytes_for(M, K, N, sparse24)) return MARLIN_ERR_WORKSPACE;
   DeviceInfo info;
   int st = device_info(&info);
   if (st != MARLIN_OK) return st;
@@ -184,10 +191,12 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
     // launch, N a multiple of 128).  What none of them serves (2:4 layers, other N) goes through the warp-level
     // kernel in slabs of 16 rows.
     const int tmode = tcd_mode();
-    const bool tc_ok = !sparse24 && tc_path_supported(1, K, N);
+    // 2:4 layers whose N is a multiple of 256 are packed in the wide layout, which only the tcgen05 kernel reads:
+    // it takes every batch size there
+    const bool tc_ok = tc_path_supported(1, K, N);
     const bool use_tcd = !sparse24 && tcd_path_supported(1, K, N) &&
                          (tmode == 1 || (tmode == 2 && rem >= tc_min_m() && !tc_ok));
-    const bool use_tc = !use_tcd && tc_ok && rem >= tc_min_m();
+    const bool use_tc = !use_tcd && tc_ok && (sparse24 || rem >= tc_min_m());
     const int m_slab = use_tcd ? (rem < kTcdMaxSlabM ? rem : kTcdMaxSlabM)
                                : use_tc ? (rem < kTcMaxSlabM ? rem : kTcMaxSlabM) : (rem < kMaxSlabM ? rem : kMaxSlabM);
     GemmParams p;
@@ -208,7 +217,7 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
     p.status = reinterpret_cast<int*>(ws + kWsStatusOff);
     p.counters = reinterpret_cast<int*>(ws + kWsCounterOff);
     p.partials = reinterpret_cast<float*>(ws + kWsPartialOff);
-    p.tc_tiles = use_tc ? reinterpret_cast<float*>(ws + ((workspace_bytes & ~(size_t)255) - tc_tile_bytes(m_slab, N)))
+    p.tc_tiles = use_tc ? reinterpret_cast<float*>(ws + ((workspace_bytes & ~(size_t)255) - tc_tile_bytes(m_slab, N, sparse24)))
                         : nullptr;
     p.split = 0;
     p.cluster = 0;
@@ -216,7 +225,7 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
     if (use_tcd) {
       if (launch_gemm_tcd(p, info.sm_count, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MARLIN_ERR_CUDA;
     } else if (use_tc) {
-      if (launch_gemm_dense_tc(p, info.sm_count, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+      if (launch_gemm_dense_tc(p, info.sm_count, sparse24, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return MARLIN_ERR_CUDA;
     } else {
       DensePlan plan;
@@ -254,7 +263,7 @@ int marlin_gemm_static_ws(const void* A, const void* w_packed, const void* s_pac
   if (M < 1 || M > MARLIN_STATIC_WS_MAX_M || !shape_ok(K, N)) return MARLIN_ERR_SHAPE;
   if (!normalise_group(K, group_size)) return MARLIN_ERR_GROUP;
   if (!aligned16(A) || !aligned16(w_packed) || !aligned16(s_packed) || !aligned16(C)) return MARLIN_ERR_ALIGN;
-  if (marlin_workspace_bytes(M, K, N) > kStaticWsBytes) return MARLIN_ERR_WORKSPACE;
+  if (workspace_bytes_for(M, K, N, false) > kStaticWsBytes) return MARLIN_ERR_WORKSPACE;
   DeviceInfo info;
   int st = device_info(&info);
   if (st != MARLIN_OK) return st;

@@ -59,12 +59,16 @@ constexpr int kTmemCols = 512;
 constexpr int kAuxRegs = 40;         // registers per thread of the copy and MMA warps
 constexpr int kDequantRegs = 216;    // 512 threads start with 128 each: 2 x 128 x (128 - 40) / 256 = 88 more
 
-template <int MPAD>
+// SP: the 2:4 variant (Section 4).  A stage then holds the 64 kept codes per column of the k-block (8 KB) and the
+// metadata words of the 256 tensor-memory lanes (4 KB); an A-operand slot holds 32 columns of kept values and 4
+// columns of metadata per 128-channel tile.
+template <int MPAD, bool SP>
 struct TcGeometry {
   static constexpr int A_HALF_BYTES = MPAD * 128;
   static constexpr int A_BYTES = 2 * A_HALF_BYTES;
-  static constexpr int W_BYTES = 4 * kChunkBytes;
-  static constexpr int STAGE_BYTES = A_BYTES + W_BYTES;
+  static constexpr int W_BYTES = SP ? 2 * kChunkBytes : 4 * kChunkBytes;
+  static constexpr int META_BYTES = SP ? kChunkBytes : 0;
+  static constexpr int STAGE_BYTES = A_BYTES + W_BYTES + META_BYTES;
   static constexpr int SC_BYTES = kTileN * 2;                       // group scales of one stage
   static constexpr int FIXED_BYTES = 1024 + kTcMaxStages * SC_BYTES; // barriers + scale ring
   static constexpr int ALIGN_SLACK = 1024;
@@ -84,9 +88,16 @@ struct TcGeometry {
   static constexpr int NH = MPAD <= 64 ? 1 : 2;            // halves of the batch per tile
   static constexpr int MMA_N = MPAD / NH;                  // N of one MMA
   static constexpr int D_COLS = 2 * KH * MPAD;             // accumulator of (tile t, half h) at column (t * KH + h) * MPAD
-  // then as many A-operand slots (2 tiles x 64 columns each) as fit in the 512 columns
-  static constexpr int A_SLOTS = (kTmemCols - D_COLS) / 128 > 4 ? 4 : (kTmemCols - D_COLS) / 128;
-  static constexpr int A_COL0 = kTmemCols - A_SLOTS * 128;
+  // then as many A-operand slots as fit in the 512 columns: 2 tiles x 64 columns each; 2:4: 2 tiles x 32 columns of
+  // kept values, then 2 tiles x 4 columns of metadata (even column numbers: the instruction names a pair of
+  // metadata columns and which of the two)
+  static constexpr int TILE_A_COLS = SP ? 32 : 64;
+  static constexpr int SLOT_COLS = SP ? 72 : 128;
+  static constexpr int A_SLOTS = (kTmemCols - D_COLS) / SLOT_COLS > 4 ? 4 : (kTmemCols - D_COLS) / SLOT_COLS;
+  static constexpr int A_COL0 = kTmemCols - A_SLOTS * SLOT_COLS;
+  static_assert(A_COL0 % 2 == 0 && SLOT_COLS % 2 == 0, "metadata columns must start on an even column");
+  static_assert(A_SLOTS >= 2 && A_COL0 >= D_COLS, "tensor memory");
+  static_assert(STAGE_BYTES % 1024 == 0, "swizzled tiles need 1024-byte alignment");
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -94,10 +105,10 @@ struct TcGeometry {
 // ---------------------------------------------------------------------------------------------
 // GR: the layer has group scales (multiplied into the weights in the loop); otherwise one scale per column,
 // applied to the accumulators in the epilogue.
-template <int MPAD, bool GR>
+template <int MPAD, bool GR, bool SP>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a) {
-  using G = TcGeometry<MPAD>;
+  using G = TcGeometry<MPAD, SP>;
   constexpr int NSTAGES = G::STAGES;
   constexpr int NSLOTS = G::A_SLOTS;
   constexpr int NM = G::MMA_WARPS;
@@ -159,7 +170,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       const uint64_t pol_a = policy_evict_last();
       // weights and activations complete barriers of their own: the converting warps need only the former, and
       // on the first pass over the ring those arrive before the dependency wait
-      const uint32_t tx_bytes = G::W_BYTES + (p.grouped ? G::SC_BYTES : 0);
+      const uint32_t tx_bytes = G::W_BYTES + G::META_BYTES + (p.grouped ? G::SC_BYTES : 0);
       auto scale_src = [&](uint32_t col, uint32_t kb) -> const uint8_t* {
         const uint32_t gi = p.group_shift >= 0 ? (kb >> p.group_shift) : (kb / (uint32_t)p.kb_per_group);
         return p.sq + ((size_t)gi * p.N + (size_t)col * kTileN) * 2;
@@ -167,6 +178,10 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       // weights of (kb, col): the four chunks of a 256-column tile are adjacent, k-blocks follow one another
       auto weight_src = [&](uint32_t col, uint32_t kb) -> const uint8_t* {
         return p.wq + ((size_t)col * KB + kb) * (size_t)G::W_BYTES;
+      };
+      // 2:4: the metadata records follow the same order in a buffer of their own
+      auto meta_src = [&](uint32_t col, uint32_t kb) -> const uint8_t* {
+        return p.meta + ((size_t)col * KB + kb) * (size_t)G::META_BYTES;
       };
       // first pass over the ring: weights before the dependency wait, activations after it
       uint32_t u = u0 + pw;
@@ -176,6 +191,9 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
           const uint32_t col = u / KB, kb = u - col * KB;
           mbar_expect_tx(&full[s], tx_bytes);
           bulk_g2s(stage0 + (size_t)s * G::STAGE_BYTES + G::A_BYTES, weight_src(col, kb), G::W_BYTES, &full[s], pol_w);
+          if constexpr (SP)
+            bulk_g2s(stage0 + (size_t)s * G::STAGE_BYTES + G::A_BYTES + G::W_BYTES, meta_src(col, kb), G::META_BYTES,
+                     &full[s], pol_w);
           if (p.grouped) bulk_g2s(sc_ring + (size_t)s * G::SC_BYTES, scale_src(col, kb), G::SC_BYTES, &full[s], pol_w);
         }
       }
@@ -202,6 +220,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         if (lane == 0) {
           mbar_expect_tx(&full[s], tx_bytes);
           bulk_g2s(st + G::A_BYTES, weight_src(col, kb), G::W_BYTES, &full[s], pol_w);
+          if constexpr (SP) bulk_g2s(st + G::A_BYTES + G::W_BYTES, meta_src(col, kb), G::META_BYTES, &full[s], pol_w);
           if (p.grouped) bulk_g2s(sc_ring + (size_t)s * G::SC_BYTES, scale_src(col, kb), G::SC_BYTES, &full[s], pol_w);
           mbar_expect_tx(&xfull[s], G::A_BYTES);
         }
@@ -242,12 +261,26 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
           if (lane == 0) {
             // descriptor of the first K = 16 step of the stage; the others differ in the address field only
             const uint64_t desc0 = smem_desc_k_sw128(smem_u32(stage0 + (size_t)s * G::STAGE_BYTES) + b_rows_off);
-            const uint32_t a_tmem = tmem_base + (uint32_t)(G::A_COL0 + (slot * 2 + t) * 64);
+            const uint32_t slot_col = tmem_base + (uint32_t)(G::A_COL0 + slot * G::SLOT_COLS);
+            const uint32_t a_tmem = slot_col + (uint32_t)(t * G::TILE_A_COLS);
+            if constexpr (!SP) {
 #pragma unroll
-            for (int k2 = 0; k2 < KS; ++k2) {
-              const int ks = h * KS + k2;
-              const uint64_t bdesc = desc0 + (uint64_t)(((ks >> 2) * G::A_HALF_BYTES + (ks & 3) * 32) >> 4);
-              tc_mma_ts(d_tmem, a_tmem + ks * 8, bdesc, idesc, (x == 0 && k2 == 0) ? 0u : 1u);
+              for (int k2 = 0; k2 < KS; ++k2) {
+                const int ks = h * KS + k2;
+                const uint64_t bdesc = desc0 + (uint64_t)(((ks >> 2) * G::A_HALF_BYTES + (ks & 3) * 32) >> 4);
+                tc_mma_ts(d_tmem, a_tmem + ks * 8, bdesc, idesc, (x == 0 && k2 == 0) ? 0u : 1u);
+              }
+            } else {
+              // 2:4 (Section 4): one instruction takes 32 rows of k (16 kept values per channel = 8 columns of
+              // the slot) and the metadata column of that step; four steps per k-block
+              const uint32_t e_tmem = slot_col + (uint32_t)(2 * G::TILE_A_COLS + t * 4);
+#pragma unroll
+              for (int k2 = 0; k2 < KS / 2; ++k2) {
+                const int i = h * (KS / 2) + k2;
+                const uint64_t bdesc = desc0 + (uint64_t)(((i >> 1) * G::A_HALF_BYTES + (i & 1) * 64) >> 4);
+                tc_mma_sp_ts(d_tmem, a_tmem + i * 8, bdesc, e_tmem + (uint32_t)(i & ~1), idesc | kIdescSparse | (uint32_t)(i & 1),
+                             (x == 0 && k2 == 0) ? 0u : 1u);
+              }
             }
             // one arrival when these MMAs are done: the A slot may be rewritten, the activation tile refilled
             tc_commit(&mdone[s]);
@@ -307,10 +340,16 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         const uint32_t sv = lds16(smem_u32(sc_ring) + (uint32_t)s * G::SC_BYTES + (uint32_t)spos * 2);
         s2 = sv | (sv << 16);
       }
-      const uint32_t wbase = smem_u32(stage0) + (uint32_t)s * G::STAGE_BYTES + G::A_BYTES + vec_off;
+      const uint32_t wbase = smem_u32(stage0) + (uint32_t)s * G::STAGE_BYTES + G::A_BYTES + (SP ? (uint32_t)n256 * 16u : vec_off);
       uint4 v[4];
+      if constexpr (!SP) {
 #pragma unroll
-      for (int c = 0; c < 4; ++c) v[c] = lds128(wbase + c * 16);
+        for (int c = 0; c < 4; ++c) v[c] = lds128(wbase + c * 16);
+      } else {
+        v[0] = lds128(wbase);                        // kept values 0..31 of this column
+        v[1] = lds128(wbase + 256 * 16);             // kept values 32..63
+        v[2] = lds128(wbase + (uint32_t)G::W_BYTES); // the four metadata words of this tensor-memory lane
+      }
       // the codes are in registers: the weight part of the stage is free as far as this warp is concerned
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty[s]);
@@ -321,24 +360,44 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         mbar_wait(&mdone[jt % NSTAGES], (jt / NSTAGES) & 1u, abort_flag, p.status);
       }
       tc_fence_after_sync();
-      const uint32_t a_col = tmem_lane + (uint32_t)(G::A_COL0 + (slot * 2 + tile) * 64);
+      const uint32_t slot_col = tmem_lane + (uint32_t)(G::A_COL0 + slot * G::SLOT_COLS);
+      if constexpr (!SP) {
+        const uint32_t a_col = slot_col + (uint32_t)(tile * 64);
 #pragma unroll
-      for (int hh = 0; hh < 2; ++hh) {
-        // 64 rows of k = 32 columns of the slot, written with one store
+        for (int hh = 0; hh < 2; ++hh) {
+          // 64 rows of k = 32 columns of the slot, written with one store
+          uint32_t r[32];
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const uint32_t w0 = hh == 0 ? v[c].x : v[c].z, w1 = hh == 0 ? v[c].y : v[c].w;
+            uint32_t lo[4], hi[4];
+            dequant8(w0, lo);  // rows 64hh + 16c + 0..7
+            dequant8(w1, hi);  // rows 64hh + 16c + 8..15
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              r[8 * c + e] = GR ? hmul2_u32(lo[e], s2) : lo[e];
+              r[8 * c + 4 + e] = GR ? hmul2_u32(hi[e], s2) : hi[e];
+            }
+          }
+          tc_st_x32(a_col + (uint32_t)(32 * hh), r);  // column = row / 2
+        }
+      } else {
+        // 64 kept values = 32 columns: column G holds the two kept values of the k-block's group G of four rows
         uint32_t r[32];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const uint32_t w0 = hh == 0 ? v[c].x : v[c].z, w1 = hh == 0 ? v[c].y : v[c].w;
-          uint32_t lo[4], hi[4];
-          dequant8(w0, lo);  // rows 64hh + 16c + 0..7
-          dequant8(w1, hi);  // rows 64hh + 16c + 8..15
+        for (int c = 0; c < 2; ++c) {
+          const uint32_t w[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            r[8 * c + e] = GR ? hmul2_u32(lo[e], s2) : lo[e];
-            r[8 * c + 4 + e] = GR ? hmul2_u32(hi[e], s2) : hi[e];
+          for (int wi = 0; wi < 4; ++wi) {
+            uint32_t a[4];
+            dequant8(w[wi], a);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) r[16 * c + 4 * wi + e] = GR ? hmul2_u32(a[e], s2) : a[e];
           }
         }
-        tc_st_x32(a_col + (uint32_t)(32 * hh), r);  // column = row / 2
+        tc_st_x32(slot_col + (uint32_t)(tile * 32), r);
+        const uint32_t mw[4] = {v[2].x, v[2].y, v[2].z, v[2].w};
+        tc_st_x4(slot_col + (uint32_t)(64 + tile * 4), mw);
       }
       tc_wait_st();
       tc_fence_before_sync();
@@ -507,10 +566,10 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
   named_bar_sync(2, kDequantThreads + 32);
 }
 
-template <int MPAD, bool GR>
+template <int MPAD, bool GR, bool SP>
 cudaError_t launch_tc(const GemmParams& p, int workers, cudaStream_t stream) {
-  using G = TcGeometry<MPAD>;
-  auto kernel = gemm_dense_tc_kernel<MPAD, GR>;
+  using G = TcGeometry<MPAD, SP>;
+  auto kernel = gemm_dense_tc_kernel<MPAD, GR, SP>;
   static bool attr_set[64] = {};
   int dev = 0;
   cudaError_t err = cudaGetDevice(&dev);
@@ -567,7 +626,7 @@ bool tc_path_supported(int m_slab, int K, int N) {
 
 int tc_mpad(int m_slab) { return m_slab <= 32 ? 32 : (m_slab <= 64 ? 64 : 128); }
 
-cudaError_t launch_gemm_dense_tc(GemmParams p, int sm_count, cudaStream_t stream) {
+cudaError_t launch_gemm_dense_tc(GemmParams p, int sm_count, bool sparse24, cudaStream_t stream) {
   // stripe plan for 256-column tiles
   const long long units = (long long)(p.N / kTileN) * (p.K / kTileK);
   long long workers = sm_count < kMaxWorkers ? sm_count : kMaxWorkers;
@@ -596,14 +655,24 @@ cudaError_t launch_gemm_dense_tc(GemmParams p, int sm_count, cudaStream_t stream
   }
   p.workers = (uint32_t)workers;
   const int mpad = tc_mpad(p.M);
-  if (p.grouped) {
-    if (mpad == 32) return launch_tc<32, true>(p, (int)workers, stream);
-    if (mpad == 64) return launch_tc<64, true>(p, (int)workers, stream);
-    return launch_tc<128, true>(p, (int)workers, stream);
+  if (sparse24) {
+    if (p.grouped) {
+      if (mpad == 32) return launch_tc<32, true, true>(p, (int)workers, stream);
+      if (mpad == 64) return launch_tc<64, true, true>(p, (int)workers, stream);
+      return launch_tc<128, true, true>(p, (int)workers, stream);
+    }
+    if (mpad == 32) return launch_tc<32, false, true>(p, (int)workers, stream);
+    if (mpad == 64) return launch_tc<64, false, true>(p, (int)workers, stream);
+    return launch_tc<128, false, true>(p, (int)workers, stream);
   }
-  if (mpad == 32) return launch_tc<32, false>(p, (int)workers, stream);
-  if (mpad == 64) return launch_tc<64, false>(p, (int)workers, stream);
-  return launch_tc<128, false>(p, (int)workers, stream);
+  if (p.grouped) {
+    if (mpad == 32) return launch_tc<32, true, false>(p, (int)workers, stream);
+    if (mpad == 64) return launch_tc<64, true, false>(p, (int)workers, stream);
+    return launch_tc<128, true, false>(p, (int)workers, stream);
+  }
+  if (mpad == 32) return launch_tc<32, false, false>(p, (int)workers, stream);
+  if (mpad == 64) return launch_tc<64, false, false>(p, (int)workers, stream);
+  return launch_tc<128, false, false>(p, (int)workers, stream);
 }
 
 }  // namespace marlin_b200

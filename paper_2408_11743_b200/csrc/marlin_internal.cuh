@@ -87,8 +87,9 @@ cudaError_t launch_pack_sparse24(uint32_t* qc, uint8_t* idx, uint16_t* s, uint32
 // tcgen05 kernel (gemm_dense_tc.cu): 256-column tiles, up to 128 rows of A per launch.
 bool tc_path_supported(int m_slab, int K, int N);
 int tc_mpad(int m_slab);  // rows of A padded to the MMA's N: 32, 64 or 128
-// fills the plan fields of `p` (ncols, units, workers) itself
-cudaError_t launch_gemm_dense_tc(GemmParams p, int sm_count, cudaStream_t stream);
+// fills the plan fields of `p` (ncols, units, workers) itself; sparse24: the 2:4 instances (tcgen05.mma.sp), which read
+// the wide 2:4 layout (N a multiple of 256)
+cudaError_t launch_gemm_dense_tc(GemmParams p, int sm_count, bool sparse24, cudaStream_t stream);
 // tcgen05 kernel with deferred scales (gemm_tcd.cu): 128-column tiles, up to 64 rows of A per launch.
 bool tcd_path_supported(int m_slab, int K, int N);
 int tcd_mpad(int m_slab);            // rows of A padded to the MMA's N: 16, 32 or 64

@@ -40,6 +40,28 @@ __device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint
       "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// The 2:4 form (Section 4): A holds 16 kept values per row for 32 rows of k (eight columns), `e_tmem` names an even
+// metadata column and the sparsity selector in the instruction descriptor (bits 0-1) which column of that pair:
+// lane 16a + 8h + r of it holds, for k-half h of the step, four 4-bit entries (first | second << 2 position of the
+// two kept values inside each group of four) for row 16a + r in its low half and for row 16a + 8 + r in its high
+// half.  (Confirmed on a B200 with random kept values, patterns and identity activations.)
+constexpr uint32_t kIdescSparse = 1u << 2;
+__device__ __forceinline__ void tc_mma_sp_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t e_tmem,
+                                             uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %5, 0;\n"
+      "tcgen05.mma.sp.cta_group::1.kind::f16 [%0], [%1], %2, [%3], %4, p;\n"
+      "}\n" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(b_desc), "r"(e_tmem), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_st_x4(uint32_t taddr, const uint32_t (&r)[4]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};" ::"r"(taddr), "r"(r[0]), "r"(r[1]),
+               "r"(r[2]), "r"(r[3])
+               : "memory");
+}
 // eight consecutive 32-bit columns of this thread's TMEM lane
 __device__ __forceinline__ void tc_st_x8(uint32_t taddr, const uint32_t (&r)[8]) {
   asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr), "r"(r[0]),

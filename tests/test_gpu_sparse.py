@@ -69,15 +69,17 @@ def test_sparse_gemm_matches_oracle(marlin, oracle_lib, M, K, N, G):
 
 
 # the partition and the fix-up the planner did not pick for a shape, forced through the library's tuning switches
-SPARSE_MODES = [{"MARLIN_B200_SPLIT": "0"}, {"MARLIN_B200_CLUSTER": "0"}, {"MARLIN_B200_NW": "1"},
-                {"MARLIN_B200_NW": "2"}, {"MARLIN_B200_NW": "4", "MARLIN_B200_SPLIT": "0"}]
+SPARSE_MODES = [{"MARLIN_B200_SPLIT": "0", "MARLIN_B200_TC_SPLIT": "0"}, {"MARLIN_B200_CLUSTER": "0", "MARLIN_B200_TC_CLUSTER": "0"},
+                {"MARLIN_B200_NW": "1"}, {"MARLIN_B200_NW": "2"}, {"MARLIN_B200_NW": "4", "MARLIN_B200_SPLIT": "0"}]
 
 
 @pytest.mark.parametrize("mode", range(len(SPARSE_MODES)))
 def test_sparse_every_partition_and_fixup_path(marlin, oracle_lib, mode, monkeypatch):
     for k, v in SPARSE_MODES[mode].items():
         monkeypatch.setenv(k, v)
-    for M, K, N, G in [(1, 4096, 4096, 128), (8, 2048, 1536, 128), (16, 1024, 768, -1), (40, 4096, 1024, 128)]:
+    for M, K, N, G in [(1, 4096, 4096, 128), (8, 2048, 1536, 128), (16, 1024, 768, -1), (40, 4096, 1024, 128),
+                       (8, 2048, 1344, 128), (16, 1024, 704, -1), (40, 4096, 320, 128), (128, 2048, 2048, 128),
+                       (64, 8192, 1024, -1)]:
         case = inputs.make_sparse24(M, K, N, G, seed=17 * mode + M + K + N)
         C = SparseLayer(marlin, case, M)(case.A)
         C_ref = oracle_lib.gemm_sparse24(case.A, case.qc_kpacked, case.idx, case.S, case.G)
@@ -85,10 +87,18 @@ def test_sparse_every_partition_and_fixup_path(marlin, oracle_lib, mode, monkeyp
         assert bad == 0, f"{bad} elements out of tolerance, worst ratio {worst:.3f}, rms {rms:.3f}"
 
 
-@pytest.mark.parametrize("M,K,N", [(1, 4096, 4096), (16, 4096, 22016), (40, 2048, 1024)])
-def test_sparse_long_stream_of_overlapping_launches_is_stable(marlin, oracle_lib, M, K, N):
+@pytest.mark.parametrize("M,K,N,exact", [
+    (1, 4096, 4096, False),     # wide layout (N a multiple of 256): tcgen05.mma.sp kernel, partial tiles added at the L2
+    (16, 4096, 22016, False),
+    (64, 8192, 8192, True),     # tcgen05.mma.sp kernel, clusters: fixed order of the sum
+    (40, 2048, 1024, False),
+    (8, 4096, 1344, True),      # N = 64 mod 256: warp-level mma.sp kernel, fixed order of the sum
+    (40, 2048, 448, True),      # the same in slabs of 16 rows
+])
+def test_sparse_long_stream_of_overlapping_launches_is_stable(marlin, oracle_lib, M, K, N, exact):
     # 120 launches that overlap on the stream and share one workspace, two inputs and two outputs in turn:
-    # at the end each output holds exactly what a single launch gives (the sum order is fixed in this kernel)
+    # at the end each output holds what a single launch gives (bit for bit where the order of the sum is fixed;
+    # within a quarter of the allowance where partial tiles are added at the L2 in arrival order)
     import torch
     case = inputs.make_sparse24(M, K, N, 128, seed=9 + M)
     other = inputs.make_sparse24(M, K, N, 128, seed=10 + M)
@@ -104,7 +114,14 @@ def test_sparse_long_stream_of_overlapping_launches_is_stable(marlin, oracle_lib
         torch.cuda.synchronize()
         assert marlin.read_status(layer.ws) == 0
         for i in range(2):
-            assert np.array_equal(to_host(C[i]).view(np.uint16), want[i].view(np.uint16)), f"repetition {rep}, buffer {i}"
+            got = to_host(C[i])
+            if exact:
+                assert np.array_equal(got.view(np.uint16), want[i].view(np.uint16)), f"repetition {rep}, buffer {i}"
+            else:
+                bad, worst, _ = oracle_lib.check_tolerance(got, want[i])
+                assert bad == 0 and worst < 0.25, f"repetition {rep}, buffer {i}"
+    ws = to_host(layer.ws)
+    assert np.all(ws[256:8192] == 0)   # arrival counters left clean
 
 
 def test_sparse_equals_dense_kernel_on_the_expanded_matrix(marlin, oracle_lib):
@@ -121,9 +138,12 @@ def test_sparse_equals_dense_kernel_on_the_expanded_matrix(marlin, oracle_lib):
     assert bad == 0 and worst < 0.3
 
 
-def test_sparse_integer_closed_form_and_one_hot(marlin, oracle_lib):
+@pytest.mark.parametrize("M,N", [(8, 256), (8, 192), (40, 512), (128, 256), (64, 320)])
+def test_sparse_integer_closed_form_and_one_hot(marlin, oracle_lib, M, N):
+    # N = 256, 512: the wide layout and the tcgen05.mma.sp kernel (its metadata placement in tensor memory is what the
+    # one-hot rows probe); N = 192, 320: the warp-level mma.sp kernel
     rng = np.random.default_rng(8)
-    M, K, N, G = 8, 1024, 256, 128
+    K, G = 1024, 128
     case = inputs.make_sparse24(M, K, N, G, seed=9)
     case.A = rng.integers(-3, 4, size=(M, K)).astype(np.float16)
     case.S = np.ldexp(1.0, rng.integers(-4, 1, size=(K // G, N))).astype(np.float16)
