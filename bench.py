@@ -1,7 +1,9 @@
 #!/usr/bin/env python
 """Benchmark of the W4A16 layer on B200: the batch sweep on one large layer.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-extra]
+    python bench.py --sustain SECONDS          # the same step replayed for that long, rate per SM-clock bin
+    python bench.py --case M,K,N,G[,sparse]    # one layer shape a few times (for profiler captures)
 
 Workload (config 2 of this build): K = N = 8192, group size 128, M in {1,2,4,8,16,32,64,128};
 A ~ fp16 N(0,1), codes uniform 0..15 (zero point 8), scales uniform in [0.005, 0.02]; synthetic.
@@ -51,13 +53,14 @@ REFERENCE_SAMPLE_MS = (16,)   # one step of --impl reference
 
 
 def launches_for(M: int) -> int:
-    """Kernels one marlin_gemm call launches on this layer: the warp-MMA kernel up to 32 rows, the tcgen05
+    """Kernels one marlin_gemm call launches on this layer: the warp-MMA kernel up to 16 rows, the tcgen05
     kernel (up to 128 rows per launch) above."""
     return 1 if M <= 128 else (M + 127) // 128
 
 
-# DRAM bytes of one launch of the dominant kernel from the committed ncu capture
-# (profiles/gemm_dense_kernel_M16_K8192_N8192.md: dram__bytes_read.sum + dram__bytes_write.sum)
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel, the instance that
+# serves M <= 8, from the committed ncu capture of its M = 1 launch (profiles/gemm_dense_kernel_M1_K8192_N8192.md);
+# the algorithmic bytes of that launch are 34.64e6
 NCU_DRAM_BYTES_PER_LAUNCH = 34.69e6
 
 
@@ -180,15 +183,14 @@ def run_reference(args):
 # ------------------------------------------------------------------------------------------------
 # GPU leg
 # ------------------------------------------------------------------------------------------------
-def extra_layers(marlin, dev, stream, l2, peaks, capture, time_graph):
-    """Per-layer numbers outside the timed step: Llama-2-7B and -70B shapes (dense) and the 8192^2 2:4 layer."""
-    import torch
-    out = []
-    rng = np.random.default_rng(1234)
+class LayerBench:
+    """One packed layer resident on the GPU (several cold copies) and its cuBLAS fp16 counterpart, timed per batch size."""
 
-    def measure(K, N, G, M, sparse):
-        wb = roofline.weight_bytes(K, N, G, sparse24=sparse)
-        copies = max(2, int(np.ceil(2.0 * l2 / wb)) + 1)
+    def __init__(self, marlin, dev, stream, l2, K, N, G, sparse, rng, with_fp16=True):
+        import torch
+        self.m, self.dev, self.stream, self.K, self.N, self.G, self.sparse = marlin, dev, stream, K, N, G, sparse
+        self.wb = roofline.weight_bytes(K, N, G, sparse24=sparse)
+        self.copies = max(2, int(np.ceil(2.0 * l2 / self.wb)) + 1)
         S = torch.from_numpy(rng.uniform(0.005, 0.02, size=(K // G, N)).astype(np.float16)).to(dev)
         if sparse:
             qc = torch.from_numpy(rng.integers(-2**31, 2**31 - 1, size=(K // 16, N), dtype=np.int64).astype(np.int32)).to(dev)
@@ -199,16 +201,25 @@ def extra_layers(marlin, dev, stream, l2, peaks, capture, time_graph):
         else:
             q = torch.from_numpy(rng.integers(-2**31, 2**31 - 1, size=(K // 8, N), dtype=np.int64).astype(np.int32)).to(dev)
             packed0 = marlin.pack(q, S, G)
-        packed = [tuple(t.clone() for t in packed0) for _ in range(copies)]
-        A = torch.from_numpy(rng.standard_normal((M, K), dtype=np.float32).astype(np.float16)).to(dev)
+        self.packed = [tuple(t.clone() for t in packed0) for _ in range(self.copies)]
+        self.W16 = None
+        if with_fp16:
+            n16 = max(2, int(np.ceil(2.0 * l2 / (2 * K * N))) + 1)
+            self.W16 = [torch.randn((K, N), dtype=torch.float16, device=dev) * 0.05 for _ in range(n16)]
+        self.rng = rng
+
+    def time(self, M, capture, time_graph, peaks, reps_min=16):
+        import torch
+        marlin, dev, stream, K, N, G = self.m, self.dev, self.stream, self.K, self.N, self.G
+        A = torch.from_numpy(self.rng.standard_normal((M, K), dtype=np.float32).astype(np.float16)).to(dev)
         C = torch.empty((M, N), dtype=torch.float16, device=dev)
         ws = marlin.new_workspace(M, K, N, device=dev)
         rot = [0]
 
         def call():
-            pk = packed[rot[0] % copies]
+            pk = self.packed[rot[0] % self.copies]
             rot[0] += 1
-            if sparse:
+            if self.sparse:
                 marlin.gemm_sparse24(A, pk[0], pk[1], pk[2], K, N, G, ws, out=C, stream=stream)
             else:
                 marlin.gemm(A, pk[0], pk[1], K, N, G, ws, out=C, stream=stream)
@@ -216,49 +227,95 @@ def extra_layers(marlin, dev, stream, l2, peaks, capture, time_graph):
             for _ in range(3):
                 call()
         torch.cuda.synchronize(dev)
-        reps = max(16, 2 * copies)
+        reps = max(reps_min, 2 * self.copies)
         g = capture(call, reps)
         time_graph(g)
         t = min(time_graph(g) for _ in range(5)) / reps
-        W16 = [torch.randn((K, N), dtype=torch.float16, device=dev) * 0.05
-               for _ in range(max(2, int(np.ceil(2.0 * l2 / (2 * K * N))) + 1))]
-        o16 = torch.empty((M, N), dtype=torch.float16, device=dev)
-        r16 = [0]
+        troof = roofline.roofline_seconds(M, K, N, G, peaks, sparse24=self.sparse)
+        if marlin.read_status(ws, stream=stream) != 0:
+            raise RuntimeError("device-side wait expired")
+        r = {"K": K, "N": N, "G": G, "M": M, "sparse24": self.sparse, "us": round(t * 1e6, 3),
+             "weight_gbs": round(self.wb / t / 1e9, 1), "tflops": round(roofline.flops(M, K, N) / t / 1e12, 2),
+             "roofline_frac": round(troof / t, 4)}
+        if self.W16 is not None:
+            o16 = torch.empty((M, N), dtype=torch.float16, device=dev)
+            r16 = [0]
 
-        def fp16():
-            torch.matmul(A, W16[r16[0] % len(W16)], out=o16)
-            r16[0] += 1
-        with torch.cuda.stream(stream):
-            for _ in range(3):
-                fp16()
-        torch.cuda.synchronize(dev)
-        g16 = capture(fp16, 2 * len(W16))
-        time_graph(g16)
-        t16 = min(time_graph(g16) for _ in range(5)) / (2 * len(W16))
-        troof = roofline.roofline_seconds(M, K, N, G, peaks, sparse24=sparse)
-        assert marlin.read_status(ws, stream=stream) == 0
-        return {"K": K, "N": N, "M": M, "sparse24": sparse, "us": round(t * 1e6, 3),
-                "weight_gbs": round(wb / t / 1e9, 1), "roofline_frac": round(troof / t, 4),
-                "cublas_fp16_us": round(t16 * 1e6, 3), "speedup_vs_fp16": round(t16 / t, 3)}
+            def fp16():
+                torch.matmul(A, self.W16[r16[0] % len(self.W16)], out=o16)
+                r16[0] += 1
+            with torch.cuda.stream(stream):
+                for _ in range(3):
+                    fp16()
+            torch.cuda.synchronize(dev)
+            g16 = capture(fp16, 2 * len(self.W16))
+            time_graph(g16)
+            t16 = min(time_graph(g16) for _ in range(5)) / (2 * len(self.W16))
+            r["cublas_fp16_us"] = round(t16 * 1e6, 3)
+            r["speedup_vs_fp16"] = round(t16 / t, 3)
+        return r
+
+
+def extra_layers(marlin, dev, stream, l2, peaks, capture, time_graph):
+    """Per-layer numbers outside the timed step: every layer and batch size of configs 3 (Llama-2-7B shapes), 4
+    (Llama-2-70B shapes, group 128 and one scale per column) and 5 (the 2:4 layer, with the dense layer beside it)."""
+    import torch
+    out = []
+    rng = np.random.default_rng(1234)
+
+    def sweep(K, N, G, sparse, Ms, label, config):
+        layer = LayerBench(marlin, dev, stream, l2, K, N, G, sparse, rng)
+        for M in Ms:
+            r = layer.time(M, capture, time_graph, peaks)
+            r["layer"], r["config"] = label, config
+            out.append(r)
+        del layer
+        torch.cuda.empty_cache()
 
     for name, K, N in inputs.LLAMA7B_LAYERS:
-        for M in (1, 16, 32):
-            r = measure(K, N, GROUP, M, False)
-            r["layer"] = "llama2-7b " + name
-            out.append(r)
-    for M in (16, 32, 64, 128):
-        r = measure(8192, 8192, GROUP, M, True)
-        r["layer"] = "2:4 sparse 8192x8192"
-        out.append(r)
+        sweep(K, N, GROUP, False, (1, 16, 32, 64, 128), "llama2-7b " + name, 3)
+    sweep(8192, 8192, GROUP, True, (16, 32, 64, 128), "2:4 sparse 8192x8192", 5)
     for name, K, N in inputs.LLAMA70B_LAYERS:
-        for M in (1, 16, 64):
-            r = measure(K, N, GROUP, M, False)
-            r["layer"] = "llama2-70b " + name
-            out.append(r)
-    r = measure(28672, 8192, 28672, 16, False)
-    r["layer"] = "llama2-70b down, one scale per column"
-    out.append(r)
+        for G in (GROUP, K):
+            sweep(K, N, G, False, (1, 16, 64, 128),
+                  "llama2-70b " + name + (" g128" if G == GROUP else " per-column scales"), 4)
     return out
+
+
+def run_case(args):
+    """One layer shape, a few launches: the small, self-contained command the profiler captures are made with."""
+    import torch
+    import paper_2408_11743_b200 as marlin
+    parts = args.case.split(",")
+    M, K, N, G = (int(x) for x in parts[:4])
+    sparse = len(parts) > 4 and parts[4].startswith("sparse")
+    if G <= 0:
+        G = K
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    stream = torch.cuda.Stream(device=dev)
+    peaks = roofline.load_peaks(ROOT)
+    l2 = args.copies_bytes
+    layer = LayerBench(marlin, dev, stream, l2, K, N, G, sparse, np.random.default_rng(1), with_fp16=False)
+
+    def capture(fn, reps):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for _ in range(reps):
+                fn()
+        return g
+
+    def time_graph(g):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            e0.record(stream)
+            g.replay()
+            e1.record(stream)
+        e1.synchronize()
+        return e0.elapsed_time(e1) * 1e-3
+    r = layer.time(M, capture, time_graph, peaks, reps_min=args.iters)
+    r["copies"] = layer.copies
+    print(json.dumps(r), flush=True)
 
 
 def run_ours(args):
@@ -359,6 +416,52 @@ def run_ours(args):
     value = replicas.job_throughput(step_wbytes, world, step_s) / 1e9
     step_alg_bytes = sum(roofline.algorithmic_bytes(M, K_DIM, N_DIM, GROUP) for M in SWEEP)
     launches_per_step = sum(launches_for(M) for M in SWEEP)
+
+    # ---- sustained mode (Section 5.1 "Sustained performance"): the same graph replayed for seconds; the SM clock is
+    # sampled beside it (read-only) and the rate is reported per clock bin and as time x clock ----
+    sustained = None
+    if args.sustain > 0:
+        s2 = ClockSampler(local_rank)
+        s2.start()
+        time.sleep(0.3)
+        barrier()
+        batches = []
+        t_end = time.time() + args.sustain
+        while time.time() < t_end:
+            w0 = time.time()
+            dt = time_graph(g_steps, replays=10)
+            batches.append((w0, time.time(), dt / (10 * args.steps)))
+        barrier()
+        s2.stop()
+        if rank == 0 and batches:
+            samples = []
+            for t, row in s2.rows:
+                parts = [x.strip() for x in row.split(",")]
+                try:
+                    samples.append((t, float(parts[0])))
+                except (ValueError, IndexError):
+                    pass
+            bins = {}
+            prods = []
+            for w0, w1, step_t in batches:
+                near = [mhz for t, mhz in samples if w0 - 0.06 <= t <= w1 + 0.06]
+                if not near:
+                    continue
+                mhz = statistics.median(near)
+                bins.setdefault(int(round(mhz / 50.0)) * 50, []).append(step_t)
+                prods.append(step_t * mhz)
+            all_t = [b[2] for b in batches]
+            summ = s2.summary(batches[0][0], batches[-1][1])
+            sustained = {
+                "seconds": round(batches[-1][1] - batches[0][0], 2), "steps": len(batches) * 10 * args.steps,
+                "ms_per_step": round(1e3 * statistics.median(all_t), 5),
+                "value": round(world * step_wbytes / statistics.median(all_t) / 1e9, 2), "unit": UNIT,
+                "sm_mhz_median": summ["sm_mhz"], "reasons": summ["reasons"],
+                "us_per_step_x_ghz": round(1e3 * statistics.median(prods), 3) if prods else None,
+                "by_clock": [{"sm_mhz": k, "batches": len(v), "ms_per_step": round(1e3 * statistics.median(v), 5),
+                              "value": round(world * step_wbytes / statistics.median(v) / 1e9, 2)}
+                             for k, v in sorted(bins.items())],
+            }
 
     line = None
     if rank == 0:
@@ -507,6 +610,8 @@ def run_ours(args):
             "gpu_launches": launches_per_step * args.steps,
             "clocks": clocks,
         }
+        if sustained is not None:
+            line["sustained"] = sustained
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
@@ -521,8 +626,17 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extra", action="store_true", help="skip the Llama-shaped and 2:4 context measurements")
+    ap.add_argument("--sustain", type=float, default=0.0, metavar="SECONDS",
+                    help="replay the step for this long and report the rate per sampled SM clock (Section 5.1, "
+                         "sustained performance); clocks are only read, never set")
+    ap.add_argument("--case", default=None, metavar="M,K,N,G[,sparse]", help="time one layer shape and exit")
+    ap.add_argument("--iters", type=int, default=8, help="--case: launches per timed graph")
+    ap.add_argument("--copies-bytes", type=int, default=126 * 1024 * 1024,
+                    help="--case: the cold copies of the packed layer exceed twice this many bytes")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.case:
+        run_case(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
