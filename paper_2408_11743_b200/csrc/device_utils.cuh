@@ -48,7 +48,14 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 // are set; from then on every wait of the CTA returns at once, so all warps run to the end of the
 // kernel through their normal control flow (no barrier is left unattended) and the host sees
 // MARLIN_ERR_DEVICE_TIMEOUT instead of a hang.
-constexpr uint64_t kWaitLimitNs = 2000000000ull;
+#ifndef MARLIN_WAIT_LIMIT_NS
+#define MARLIN_WAIT_LIMIT_NS 2000000000ull  // a test build of the library shortens this to milliseconds
+#endif
+constexpr uint64_t kWaitLimitNs = MARLIN_WAIT_LIMIT_NS;
+// Test builds only (-DMARLIN_TEST_HOOKS): when word 7 of the workspace's status area holds this value, worker 0
+// leaves out the copies of its second pipeline stage, so that the waits on that stage run into their limit and
+// the time-out path can be exercised without any fault.  The product library is built without the hooks.
+constexpr int kTestWithholdMagic = 0x57495448;
 // BACKOFF_NS > 0: sleep between polls.  The copy-issuing warps use it: their waits are long and not urgent,
 // and a warp that polls flat out takes issue slots from the compute warps of its scheduler.
 template <int BACKOFF_NS = 0>

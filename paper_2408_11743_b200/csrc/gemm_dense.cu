@@ -82,6 +82,15 @@ struct Geometry {
   static constexpr int STAGES_FIT = (kSmemBudget - ALIGN_SLACK - SC_OFF - 1023) / (STAGE_BYTES + SC_BYTES);
   static constexpr int STAGES = STAGES_FIT > kMaxStages ? kMaxStages : STAGES_FIT;
   static constexpr int FIXED_BYTES = ((SC_OFF + STAGES * SC_BYTES + 1023) / 1024) * 1024;
+  // what the kernel relies on
+  static_assert(CW % NW == 0 && SK >= 1, "warp groups");
+  static_assert(STAGE_BYTES % 1024 == 0, "swizzled activation tiles need 1024-byte alignment");
+  static_assert(FIXED_BYTES + ALIGN_SLACK + STAGES * STAGE_BYTES <= kSmemBudget, "shared memory");
+  static_assert(STAGES >= SK && STAGES >= kProducerWarps, "the ring must hold one stage per group and per producer warp");
+  static_assert(2 * kMaxStages * 8 <= 512 && kBarBytes >= 512 + 16, "barrier area: full[] at 0, empty[] at 256, flags at 512");
+  static_assert(MPAD * NT * 4 == TILE_F4 * 16, "a partial tile is MPAD x NT floats");
+  static_assert(TILE_F4 * 4 <= kWsSlotCols * kMaxSlabM, "a partial tile must fit a workspace slot");
+  static_assert(CST_BYTES >= MPAD * NT * 2, "output staging tile");
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -165,9 +174,15 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
     // kernel boundary; the A tiles follow once the previous kernel's memory is visible.
     uint32_t u = u0 + pw;
     int s = pw;
+#ifdef MARLIN_TEST_HOOKS
+    const bool withhold = worker == 0 && pw == 1 && p.status[7] == kTestWithholdMagic;  // stage 1 belongs to producer 1
+#else
+    constexpr bool withhold = false;
+#endif
     if (lane == 0) {
       for (; u < u1 && s < nstages; u += kProducerWarps, s += kProducerWarps) {
         const uint32_t col = u / KB, kb = u - col * KB;
+        if (withhold && s == 1) continue;
         mbar_expect_tx(&full[s], tx_bytes);
         bulk_g2s(stage0 + (size_t)s * G::STAGE_BYTES + G::A_BYTES, weight_src(col, kb), G::W_BYTES, &full[s], pol_w);
         if constexpr (SP)
@@ -183,6 +198,7 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
     s = pw;
     for (; u < u1 && s < nstages; u += kProducerWarps, s += kProducerWarps) {
       const uint32_t col = u / KB, kb = u - col * KB;
+      if (withhold && s == 1) continue;
       if (lane < 2)
         tma_load_2d(stage0 + (size_t)s * G::STAGE_BYTES + lane * G::A_HALF_BYTES, &tmap_a,
                     (int)(kb * kTileK + lane * 64), 0, &full[s], pol_a);
@@ -758,6 +774,16 @@ void fill_geometry(DensePlan* plan) {
   plan->stage_bytes = G::STAGE_BYTES;
   int stages = G::STAGES;
   if (const char* e = getenv("MARLIN_B200_STAGES")) { int v = atoi(e); if (v >= 2 && v < stages) stages = v; }
+  // The ring length is a multiple of the number of warp groups and of the number of producer warps, so that a
+  // stage is always consumed by the same group and refilled by the same producer warp.  Every thread then waits
+  // on a given barrier for consecutive fillings in its own program order.  Without this, stage s would pass from
+  // group to group between ring passes, and a group running more than a ring pass ahead of another (group 0 alone
+  // finishes segments in the middle of a stripe) could ask for the filling after next of a barrier: a parity wait
+  // cannot tell that from the last completed one and falls through, after which the stage's transaction counts
+  // no longer add up.
+  constexpr int kRingUnit = G::SK > kProducerWarps ? G::SK : kProducerWarps;
+  static_assert(kRingUnit % G::SK == 0 && kRingUnit % kProducerWarps == 0, "ring unit must be a common multiple");
+  stages -= stages % kRingUnit;
   plan->stages = stages;
   plan->smem_bytes = G::FIXED_BYTES + G::ALIGN_SLACK + stages * G::STAGE_BYTES;
 }

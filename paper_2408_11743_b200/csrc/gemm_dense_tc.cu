@@ -186,9 +186,15 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       // first pass over the ring: weights before the dependency wait, activations after it
       uint32_t u = u0 + pw;
       int s = pw;
+#ifdef MARLIN_TEST_HOOKS
+      const bool withhold = worker == 0 && pw == 1 && p.status[7] == kTestWithholdMagic;  // stage 1 belongs to producer 1
+#else
+      constexpr bool withhold = false;
+#endif
       if (lane == 0) {
         for (; u < u1 && s < NSTAGES; u += kTcProducerWarps, s += kTcProducerWarps) {
           const uint32_t col = u / KB, kb = u - col * KB;
+          if (withhold && s == 1) continue;
           mbar_expect_tx(&full[s], tx_bytes);
           bulk_g2s(stage0 + (size_t)s * G::STAGE_BYTES + G::A_BYTES, weight_src(col, kb), G::W_BYTES, &full[s], pol_w);
           if constexpr (SP)

@@ -253,6 +253,44 @@ def test_subnormal_scales_and_large_values(marlin, oracle_lib):
     _assert_close(oracle_lib, C, oracle_lib.gemm(A, case.q_kpacked, S, 128))
 
 
+@pytest.mark.parametrize("M,G", [(1, 128), (8, 128), (8, -1), (16, 128), (32, 128)])
+def test_activations_with_offset_and_outliers(marlin, oracle_lib, M, G):
+    # The small-batch kernels carry the offsets of the exponent trick (1024 + q, 64 + q) through the product and take
+    # them off per scale group: activations with a non-zero mean and a few outliers of 1e2..1e3 among small values make
+    # those offset sums large against the result.  The bound must still hold, also on the columns whose reference
+    # is small (their allowance is 5e-3 * rms alone).
+    K, N = 4096, 512
+    rng = np.random.default_rng(100 + M)
+    A = (0.5 + 0.25 * rng.standard_normal((M, K))).astype(np.float32)
+    for m in range(M):
+        ks = rng.choice(K, size=6, replace=False)
+        A[m, ks] = rng.choice([-1.0, 1.0], size=6) * rng.uniform(1e2, 1e3, size=6)
+    A = A.astype(np.float16)
+    case = inputs.make_dense(M, K, N, G, seed=200 + M)
+    C = DenseLayer(marlin, case.q_kpacked, case.S, G, max_M=M)(A)
+    C_ref = oracle_lib.gemm(A, case.q_kpacked, case.S, case.G)
+    bad, worst, rms = oracle_lib.check_tolerance(C, C_ref)
+    assert bad == 0, f"{bad} elements out of tolerance, worst ratio {worst:.3f}, rms {rms:.3f}"
+    small = np.abs(C_ref.astype(np.float64)) < 0.05 * rms
+    assert small.any()
+    err = np.abs(C.astype(np.float64) - C_ref.astype(np.float64))
+    assert err[small].max() <= 5e-3 * (0.05 * rms + rms)
+
+
+@pytest.mark.parametrize("M", [4, 32, 128])
+def test_scales_near_and_below_the_smallest_normal_half(marlin, oracle_lib, M):
+    # scales around 2^-14 (the smallest normal fp16) and below: the large-batch kernel multiplies (q - 8) * s in fp16
+    # before the MMA, where such products are subnormal; the result must still be within the bound of the exact one
+    K, N = 2048, 512
+    case = inputs.make_dense(M, K, N, 128, seed=300 + M)
+    rng = np.random.default_rng(M)
+    S = (2.0 ** -14 * rng.uniform(0.25, 2.0, size=(K // 128, N))).astype(np.float16)
+    A = (case.A.astype(np.float32) * 16).astype(np.float16)
+    C = DenseLayer(marlin, case.q_kpacked, S, 128, max_M=M)(A)
+    bad, worst, rms = oracle_lib.check_tolerance(C, oracle_lib.gemm(A, case.q_kpacked, S, 128))
+    assert bad == 0, f"{bad} elements out of tolerance, worst ratio {worst:.3f}, rms {rms:.3g}"
+
+
 def test_full_size_layers_on_sampled_outputs(marlin, oracle_lib):
     # the largest layers of the workload list, checked on outputs the oracle computes one by one
     rng = np.random.default_rng(2)
