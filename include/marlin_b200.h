@@ -19,7 +19,8 @@
  *     capability 10.x the calls return MARLIN_ERR_ARCH.
  *   - Shapes: K % 128 == 0, K <= 2^20, N % 64 == 0, N <= 65536, M >= 1 (any number of rows: a call splits
  *     them over as many launches as it needs).  group_size is a multiple of 128 that divides K, or K itself
- *     (also written -1): one scale per column.
+ *     (also written -1): one scale per column; on layers whose N is a multiple of 256 also 64 or 32 (Section 2.3,
+ *     group quantization with smaller groups; other values return MARLIN_ERR_GROUP).
  *   - The packed device layout is opaque (the design notes of this repository describe it); only marlin_pack* writes it and
  *     only marlin_unpack* / marlin_gemm* read it.
  */
@@ -95,13 +96,18 @@ MARLIN_API int marlin_unpack(const void* w_packed, const void* s_packed, uint32_
  *   w_packed, s_packed   device, from marlin_pack with the same K, N, group_size
  *   C          device, out, fp16 [M][N] row-major, every element written
  *   workspace  device, at least marlin_workspace_bytes(M, K, N) bytes, zeroed once by the caller
- * Accumulation is fp32 (also across stripes); the result is rounded once to fp16 (nearest even).
+ * Accumulation is fp32 (also across stripes) and the result is rounded to fp16 once (nearest even).  The
+ * weights reach the tensor cores as exact integers q - 8 (warp-level kernel, up to 16 rows: scales applied to
+ * the fp32 sums per group) or as fp16((q - 8) * s) (tcgen05 kernel with in-loop scales, from 17 rows: one more
+ * rounding of 2^-11 per weight, as in the paper's kernel).
  * Up to 16 rows the warp-level kernel runs and the same inputs give the same bits on every call.
- * From 17 rows the tcgen05 kernel takes over (128 rows per launch, N a multiple of 256; otherwise the
- * warp-level kernel runs on slabs of 16 rows).  Where it adds the partial sums of a column tile shared
- * by several CTAs through the L2 (up to 32 rows, or shapes whose CTAs do not fit as one wave of
- * thread-block clusters) the fp32 additions happen in arrival order, so the last bit of an fp16 result
- * can differ between two calls; otherwise the order is fixed there too.
+ * From 17 rows a tcgen05 kernel takes over: 128 rows per launch where N is a multiple of 256, 64 rows per
+ * launch where N is a multiple of 128 only; any other N goes through the warp-level kernel in slabs of 16
+ * rows.  Groups of 64 or 32 rows run on the tcgen05 kernel at every batch size.  Where the 256-column
+ * tcgen05 kernel adds the partial sums of a column tile shared by several CTAs through the L2 (up to 32
+ * rows, or shapes whose CTAs do not fit as one wave of thread-block clusters) the fp32 additions happen in
+ * arrival order, so the last bit of an fp16 result can differ between two calls; everywhere else the order
+ * is fixed.
  * Errors: argument checks return before anything is queued.  A kernel whose bounded waits expire
  * sets the workspace status word; read it with marlin_read_status. */
 MARLIN_API int marlin_gemm(const void* A, const void* w_packed, const void* s_packed, void* C,
@@ -148,7 +154,9 @@ MARLIN_API int marlin_unpack_sparse24(const void* w_packed, const void* meta_pac
                            uint32_t* qc_kpacked, uint8_t* idx, void* scales,
                            int K, int N, int group_size, marlin_stream stream);
 
-/* C = A . dequant(expand(W)) with the pruned positions contributing zero. */
+/* C = A . dequant(expand(W)) with the pruned positions contributing zero.  Layers whose N is a multiple of 256
+ * run on the sparse tcgen05 instruction (tcgen05.mma.sp) at every batch size, 128 rows per launch, reading the
+ * compressed weights once per launch; other N on the warp-level sparse MMA in slabs of 16 rows. */
 MARLIN_API int marlin_gemm_sparse24(const void* A, const void* w_packed, const void* meta_packed,
                          const void* s_packed, void* C, int M, int K, int N, int group_size,
                          void* workspace, size_t workspace_bytes, marlin_stream stream);

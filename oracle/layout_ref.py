@@ -11,7 +11,8 @@ Inside a chunk, 16-byte vector v = (2*j + b)*32 + lane (lane = 4*g + c) holds 32
     n = 64*nb + 16*j + 8*b + g;
 its word w = 2*h + u holds rows k = 128*kb + 64*h + 16*c + 8*u + o (o = 0..7), row offset o sitting in
 nibble (o >> 1) + 4*(o & 1) (bits 4p..4p+3 for nibble p).
-Scales: inside every run of 64 columns, packed position 8*g + 2*j + b holds column 16*j + 8*b + g.
+Scales: inside every run of 64 columns, packed position 8*g + 2*j + b holds column 16*j + 8*b + g; groups of 64 or
+32 rows are regrouped per k-block and 256-column tile (see pack_scales).
 """
 from __future__ import annotations
 
@@ -43,14 +44,23 @@ def pack_dense_weights(Q: np.ndarray) -> np.ndarray:
     return out.reshape(-1)
 
 
-def pack_scales(S: np.ndarray) -> np.ndarray:
-    """Scales S[K/G, N] fp16 -> packed order (same shape)."""
+def pack_scales(S: np.ndarray, sub: int = 1) -> np.ndarray:
+    """Scales S[K/G, N] fp16 -> packed order (same number of elements).
+
+    sub = 1 (groups of 128 rows and more): rows stay in place, inside every run of 64 columns packed position
+    8g + 2j + b holds column 16j + 8b + g.  sub = 2, 4 (groups of 64, 32 rows; N a multiple of 256): the same
+    permutation inside the runs, and the rows regrouped per k-block and 256-column tile: [K/128][N/256][sub][256].
+    """
     R, N = S.shape
     assert N % 64 == 0
     pos = np.arange(64)
     g, j, b = pos >> 3, (pos >> 1) & 3, pos & 1
     src = 16 * j + 8 * b + g
-    return S.reshape(R, N // 64, 64)[:, :, src].reshape(R, N)
+    P = S.reshape(R, N // 64, 64)[:, :, src].reshape(R, N)
+    if sub == 1:
+        return P
+    assert N % 256 == 0 and R % sub == 0
+    return P.reshape(R // sub, sub, N // 256, 256).transpose(0, 2, 1, 3).reshape(R, N)
 
 
 # ---- 2:4 variant ---------------------------------------------------------------------------------------

@@ -9,10 +9,12 @@ namespace {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// group_size -> normalised G, or 0 if unsupported.
-int normalise_group(int K, int group_size) {
+// group_size -> normalised G, or 0 if unsupported: K itself (one scale per column, also written -1), a multiple of
+// 128 that divides K, or 64 / 32 on layers whose N is a multiple of 256 (those run on the tcgen05 kernel alone).
+int normalise_group(int K, int N, int group_size) {
   if (K <= 0) return 0;
   if (group_size == -1 || group_size == K) return K;
+  if (group_size == 64 || group_size == 32) return (N % 256 == 0) ? group_size : 0;
   if (group_size <= 0 || group_size % kTileK || K % group_size) return 0;
   return group_size;
 }
@@ -95,7 +97,7 @@ size_t marlin_packed_weight_bytes(int K, int N, int sparse24) {
 }
 
 size_t marlin_packed_scale_bytes(int K, int N, int group_size) {
-  int G = normalise_group(K, group_size);
+  int G = normalise_group(K, N, group_size);
   if (!shape_ok(K, N) || !G) return 0;
   return (size_t)2 * (K / G) * N;
 }
@@ -139,7 +141,7 @@ int marlin_pack(const uint32_t* q_kpacked, const void* scales, void* w_packed, v
                 int group_size, marlin_stream stream) {
   if (!q_kpacked || !scales || !w_packed || !s_packed) return MARLIN_ERR_NULL;
   if (!shape_ok(K, N)) return MARLIN_ERR_SHAPE;
-  int G = normalise_group(K, group_size);
+  int G = normalise_group(K, N, group_size);
   if (!G) return MARLIN_ERR_GROUP;
   if (!aligned16(q_kpacked) || !aligned16(scales) || !aligned16(w_packed) || !aligned16(s_packed))
     return MARLIN_ERR_ALIGN;
@@ -154,7 +156,7 @@ int marlin_unpack(const void* w_packed, const void* s_packed, uint32_t* q_kpacke
                   int group_size, marlin_stream stream) {
   if (!q_kpacked || !scales || !w_packed || !s_packed) return MARLIN_ERR_NULL;
   if (!shape_ok(K, N)) return MARLIN_ERR_SHAPE;
-  int G = normalise_group(K, group_size);
+  int G = normalise_group(K, N, group_size);
   if (!G) return MARLIN_ERR_GROUP;
   if (!aligned16(q_kpacked) || !aligned16(scales) || !aligned16(w_packed) || !aligned16(s_packed))
     return MARLIN_ERR_ALIGN;
@@ -171,12 +173,12 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
                        bool sparse24) {
   if (!A || !w_packed || !s_packed || !C || !workspace || (sparse24 && !meta_packed)) return MARLIN_ERR_NULL;
   if (M < 1 || !shape_ok(K, N)) return MARLIN_ERR_SHAPE;
-  int G = normalise_group(K, group_size);
+  int G = normalise_group(K, N, group_size);
   if (!G) return MARLIN_ERR_GROUP;
   if (!aligned16(A) || !aligned16(w_packed) || !aligned16(s_packed) || !aligned16(C) || !aligned16(workspace) ||
       (sparse24 && !aligned16(meta_packed)))
     return MARLIN_ERR_ALIGN;
-  if (workspace_bytes < workspace_bytes_for(M, K, N, sparse24)) return MARLIN_ERR_WORKSPACE;
+  if (workspace_bytes < workspace_bytes_for(M, K, N, sparse24 || G < kTileK)) return MARLIN_ERR_WORKSPACE;
   DeviceInfo info;
   int st = device_info(&info);
   if (st != MARLIN_OK) return st;
@@ -194,9 +196,11 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
     // 2:4 layers whose N is a multiple of 256 are packed in the wide layout, which only the tcgen05 kernel reads:
     // it takes every batch size there
     const bool tc_ok = tc_path_supported(1, K, N);
-    const bool use_tcd = !sparse24 && tcd_path_supported(1, K, N) &&
+    // groups of 64 or 32 rows likewise (accepted only where N is a multiple of 256)
+    const bool small_groups = G < kTileK;
+    const bool use_tcd = !sparse24 && !small_groups && tcd_path_supported(1, K, N) &&
                          (tmode == 1 || (tmode == 2 && rem >= tc_min_m() && !tc_ok));
-    const bool use_tc = !use_tcd && tc_ok && (sparse24 || rem >= tc_min_m());
+    const bool use_tc = !use_tcd && tc_ok && (sparse24 || small_groups || rem >= tc_min_m());
     const int m_slab = use_tcd ? (rem < kTcdMaxSlabM ? rem : kTcdMaxSlabM)
                                : use_tc ? (rem < kTcMaxSlabM ? rem : kTcMaxSlabM) : (rem < kMaxSlabM ? rem : kMaxSlabM);
     GemmParams p;
@@ -209,7 +213,8 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
     p.K = K;
     p.N = N;
     p.kb = (uint32_t)(K / kTileK);
-    p.kb_per_group = G / kTileK;
+    p.kb_per_group = G >= kTileK ? G / kTileK : 1;
+    p.sub_groups = G >= kTileK ? 1 : kTileK / G;
     p.group_shift = -1;
     for (int sh = 0; sh < 31; ++sh)
       if ((1 << sh) == p.kb_per_group) p.group_shift = sh;
@@ -217,7 +222,7 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
     p.status = reinterpret_cast<int*>(ws + kWsStatusOff);
     p.counters = reinterpret_cast<int*>(ws + kWsCounterOff);
     p.partials = reinterpret_cast<float*>(ws + kWsPartialOff);
-    p.tc_tiles = use_tc ? reinterpret_cast<float*>(ws + ((workspace_bytes & ~(size_t)255) - tc_tile_bytes(m_slab, N, sparse24)))
+    p.tc_tiles = use_tc ? reinterpret_cast<float*>(ws + ((workspace_bytes & ~(size_t)255) - tc_tile_bytes(m_slab, N, sparse24 || small_groups)))
                         : nullptr;
     p.split = 0;
     p.cluster = 0;
@@ -261,7 +266,8 @@ int marlin_gemm_static_ws(const void* A, const void* w_packed, const void* s_pac
   // the argument checks of marlin_gemm first: nothing is queued for a call that is going to be refused
   if (!A || !w_packed || !s_packed || !C) return MARLIN_ERR_NULL;
   if (M < 1 || M > MARLIN_STATIC_WS_MAX_M || !shape_ok(K, N)) return MARLIN_ERR_SHAPE;
-  if (!normalise_group(K, group_size)) return MARLIN_ERR_GROUP;
+  const int Gs = normalise_group(K, N, group_size);
+  if (!Gs || Gs < kTileK) return MARLIN_ERR_GROUP;  // groups of 64 / 32 rows need the tcgen05 kernel's share of a workspace
   if (!aligned16(A) || !aligned16(w_packed) || !aligned16(s_packed) || !aligned16(C)) return MARLIN_ERR_ALIGN;
   if (workspace_bytes_for(M, K, N, false) > kStaticWsBytes) return MARLIN_ERR_WORKSPACE;
   DeviceInfo info;
@@ -290,7 +296,7 @@ int marlin_pack_sparse24(const uint32_t* qc_kpacked, const uint8_t* idx, const v
                          void* meta_packed, void* s_packed, int K, int N, int group_size, marlin_stream stream) {
   if (!qc_kpacked || !idx || !scales || !w_packed || !meta_packed || !s_packed) return MARLIN_ERR_NULL;
   if (!shape_ok(K, N)) return MARLIN_ERR_SHAPE;
-  int G = normalise_group(K, group_size);
+  int G = normalise_group(K, N, group_size);
   if (!G) return MARLIN_ERR_GROUP;
   if (!aligned16(qc_kpacked) || !aligned16(idx) || !aligned16(scales) || !aligned16(w_packed) ||
       !aligned16(meta_packed) || !aligned16(s_packed))
@@ -306,7 +312,7 @@ int marlin_unpack_sparse24(const void* w_packed, const void* meta_packed, const 
                            uint8_t* idx, void* scales, int K, int N, int group_size, marlin_stream stream) {
   if (!qc_kpacked || !idx || !scales || !w_packed || !meta_packed || !s_packed) return MARLIN_ERR_NULL;
   if (!shape_ok(K, N)) return MARLIN_ERR_SHAPE;
-  int G = normalise_group(K, group_size);
+  int G = normalise_group(K, N, group_size);
   if (!G) return MARLIN_ERR_GROUP;
   if (!aligned16(qc_kpacked) || !aligned16(idx) || !aligned16(scales) || !aligned16(w_packed) ||
       !aligned16(meta_packed) || !aligned16(s_packed))

@@ -69,7 +69,8 @@ struct TcGeometry {
   static constexpr int W_BYTES = SP ? 2 * kChunkBytes : 4 * kChunkBytes;
   static constexpr int META_BYTES = SP ? kChunkBytes : 0;
   static constexpr int STAGE_BYTES = A_BYTES + W_BYTES + META_BYTES;
-  static constexpr int SC_BYTES = kTileN * 2;                       // group scales of one stage
+  static constexpr int SC_ROW_BYTES = kTileN * 2;                   // one row of the tile's group scales
+  static constexpr int SC_BYTES = 4 * SC_ROW_BYTES;                 // scales of one stage: up to four rows (groups of 32)
   static constexpr int FIXED_BYTES = 1024 + kTcMaxStages * SC_BYTES; // barriers + scale ring
   static constexpr int ALIGN_SLACK = 1024;
   static constexpr int STAGES =
@@ -170,8 +171,12 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       const uint64_t pol_a = policy_evict_last();
       // weights and activations complete barriers of their own: the converting warps need only the former, and
       // on the first pass over the ring those arrive before the dependency wait
-      const uint32_t tx_bytes = G::W_BYTES + G::META_BYTES + (p.grouped ? G::SC_BYTES : 0);
+      // groups of 128 rows and more: one scale row per k-block; groups of 64 or 32 rows: two or four, which the
+      // packed layout keeps together per (k-block, column tile)
+      const uint32_t sc_copy = (uint32_t)p.sub_groups * G::SC_ROW_BYTES;
+      const uint32_t tx_bytes = G::W_BYTES + G::META_BYTES + (p.grouped ? sc_copy : 0);
       auto scale_src = [&](uint32_t col, uint32_t kb) -> const uint8_t* {
+        if (p.sub_groups > 1) return p.sq + ((size_t)kb * (p.N / kTileN) + col) * sc_copy;
         const uint32_t gi = p.group_shift >= 0 ? (kb >> p.group_shift) : (kb / (uint32_t)p.kb_per_group);
         return p.sq + ((size_t)gi * p.N + (size_t)col * kTileN) * 2;
       };
@@ -200,7 +205,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
           if constexpr (SP)
             bulk_g2s(stage0 + (size_t)s * G::STAGE_BYTES + G::A_BYTES + G::W_BYTES, meta_src(col, kb), G::META_BYTES,
                      &full[s], pol_w);
-          if (p.grouped) bulk_g2s(sc_ring + (size_t)s * G::SC_BYTES, scale_src(col, kb), G::SC_BYTES, &full[s], pol_w);
+          if (p.grouped) bulk_g2s(sc_ring + (size_t)s * G::SC_BYTES, scale_src(col, kb), sc_copy, &full[s], pol_w);
         }
       }
       __syncwarp();
@@ -227,7 +232,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
           mbar_expect_tx(&full[s], tx_bytes);
           bulk_g2s(st + G::A_BYTES, weight_src(col, kb), G::W_BYTES, &full[s], pol_w);
           if constexpr (SP) bulk_g2s(st + G::A_BYTES + G::W_BYTES, meta_src(col, kb), G::META_BYTES, &full[s], pol_w);
-          if (p.grouped) bulk_g2s(sc_ring + (size_t)s * G::SC_BYTES, scale_src(col, kb), G::SC_BYTES, &full[s], pol_w);
+          if (p.grouped) bulk_g2s(sc_ring + (size_t)s * G::SC_BYTES, scale_src(col, kb), sc_copy, &full[s], pol_w);
           mbar_expect_tx(&xfull[s], G::A_BYTES);
         }
         __syncwarp();
@@ -334,7 +339,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
     const uint32_t len = min(KB - kb0, u1 - u);
     const uint16_t* sptr = reinterpret_cast<const uint16_t*>(p.sq) + (size_t)col * kTileN + spos;
 
-    uint32_t s2 = 0;    // {scale, scale} of this thread's column for the current k-block
+    uint32_t sv4[4] = {0, 0, 0, 0};  // {scale, scale} of this thread's column for the four 32-row quarters of the k-block
     float sc_col = 1.f;  // the column's single scale
     if constexpr (!GR) sc_col = __half2float(__ushort_as_half(__ldg(sptr)));
     for (uint32_t x = 0; x < len; ++x, ++it) {
@@ -343,8 +348,13 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       mbar_wait(&full[s], (it / NSTAGES) & 1u, abort_flag, p.status);
       if constexpr (GR) {
         // the scale row of the k-block came with the stage (a global read here would be a cold DRAM access)
-        const uint32_t sv = lds16(smem_u32(sc_ring) + (uint32_t)s * G::SC_BYTES + (uint32_t)spos * 2);
-        s2 = sv | (sv << 16);
+        const uint32_t sbase = smem_u32(sc_ring) + (uint32_t)s * G::SC_BYTES + (uint32_t)spos * 2;
+#pragma unroll
+        for (int qd = 0; qd < 4; ++qd) {
+          // quarter qd lies in scale row qd * sub_groups / 4 of the stage (row 0 for groups of 128 rows and more)
+          const uint32_t sv = lds16(sbase + (uint32_t)((qd * p.sub_groups) >> 2) * G::SC_ROW_BYTES);
+          sv4[qd] = sv | (sv << 16);
+        }
       }
       const uint32_t wbase = smem_u32(stage0) + (uint32_t)s * G::STAGE_BYTES + G::A_BYTES + (SP ? (uint32_t)n256 * 16u : vec_off);
       uint4 v[4];
@@ -381,8 +391,9 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
             dequant8(w1, hi);  // rows 64hh + 16c + 8..15
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              r[8 * c + e] = GR ? hmul2_u32(lo[e], s2) : lo[e];
-              r[8 * c + 4 + e] = GR ? hmul2_u32(hi[e], s2) : hi[e];
+              // rows 64hh + 16c ..: quarter 2hh + c / 2 of the k-block
+              r[8 * c + e] = GR ? hmul2_u32(lo[e], sv4[2 * hh + (c >> 1)]) : lo[e];
+              r[8 * c + 4 + e] = GR ? hmul2_u32(hi[e], sv4[2 * hh + (c >> 1)]) : hi[e];
             }
           }
           tc_st_x32(a_col + (uint32_t)(32 * hh), r);  // column = row / 2
@@ -398,7 +409,8 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
             uint32_t a[4];
             dequant8(w[wi], a);
 #pragma unroll
-            for (int e = 0; e < 4; ++e) r[16 * c + 4 * wi + e] = GR ? hmul2_u32(a[e], s2) : a[e];
+            // kept pair 16c + 4wi + e = group of four original rows: quarter 2c + wi / 2 of the k-block
+            for (int e = 0; e < 4; ++e) r[16 * c + 4 * wi + e] = GR ? hmul2_u32(a[e], sv4[2 * c + (wi >> 1)]) : a[e];
           }
         }
         tc_st_x32(slot_col + (uint32_t)(tile * 32), r);

@@ -62,7 +62,8 @@ struct GemmParams {
   uint16_t* C;
   int M, K, N;
   uint32_t kb;       // K / 128
-  int kb_per_group;  // group_size / 128
+  int kb_per_group;  // group_size / 128 (1 for groups of 64 or 32 rows)
+  int sub_groups;    // scale groups per 128-row k-block: 1, or 2 / 4 for groups of 64 / 32 rows (tcgen05 kernel only)
   int group_shift;   // log2(kb_per_group) if it is a power of two, else -1
   int grouped;       // 0: one scale per column (group_size == K)
   int ncols;
@@ -99,6 +100,8 @@ cudaError_t launch_gemm_tcd(GemmParams p, int sm_count, cudaStream_t stream);
 // inverse == false: (q, s) canonical inputs -> (wq, sq) packed outputs; inverse == true: the other way round.
 cudaError_t launch_pack_dense(uint32_t* q, uint16_t* s, uint32_t* wq, uint16_t* sq, int K, int N, int G, bool inverse,
                               cudaStream_t stream);
+// canonical scales [K/G][N] <-> packed order (shared by the dense and the 2:4 pack)
+cudaError_t launch_permute_scales(uint16_t* s, uint16_t* sq, int K, int N, int G, bool inverse, cudaStream_t stream);
 
 // ---- the stripe partition (host and device use the same two formulas) ------------------------
 // worker w of P owns units [w*U/P, (w+1)*U/P); the owner of unit x is floor(((x+1)*P - 1) / U).

@@ -24,7 +24,9 @@
 //     - the tcgen05 kernel: a thread owns one column and reads its four vectors (c = 0..3), i.e. all
 //       128 rows of the k-block, dequantises and stores them to tensor memory in row order.
 //   scales: inside every run of 64 columns, position 8*g + 2*j + b holds column 16*j + 8*b + g,
-//   so that the 8 scales a thread needs are one 16-byte load.
+//   so that the 8 scales a thread needs are one 16-byte load.  Groups of 128 rows and more keep the row order
+//   [K/G][N].  Groups of 64 or 32 rows (N a multiple of 256) are stored per k-block and 256-column tile,
+//   [K/128][N/256][128/G][256], so that the two or four rows a k-block needs are one contiguous copy.
 #include "marlin_internal.cuh"
 
 namespace marlin_b200 {
@@ -103,13 +105,25 @@ __global__ void unpack_weights_kernel(const uint32_t* __restrict__ wq, uint32_t*
 }
 
 __global__ void permute_scales_kernel(const uint16_t* __restrict__ in, uint16_t* __restrict__ out, long long total,
-                                      bool inverse) {
+                                      int N, int sub, bool inverse) {
   for (long long x = blockIdx.x * (long long)blockDim.x + threadIdx.x; x < total;
        x += (long long)gridDim.x * blockDim.x) {
-    long long base = x & ~63LL;
-    int pos = (int)(x & 63);  // packed position inside the run of 64
-    int g = pos >> 3, j = (pos >> 1) & 3, b = pos & 1;
-    long long canon = base + 16 * j + 8 * b + g;
+    // x = packed position
+    const int pos = (int)(x & 63);  // packed position inside the run of 64
+    const int g = pos >> 3, j = (pos >> 1) & 3, b = pos & 1;
+    const int c64 = 16 * j + 8 * b + g;  // column inside the run
+    long long canon;
+    if (sub == 1) {
+      canon = (x & ~63LL) + c64;
+    } else {
+      // packed [kb][tile][r][256]  <->  canonical row kb * sub + r, column 256 * tile + ...
+      const long long rec = x >> 8;  // (kb * NT + tile) * sub + r
+      const int r = (int)(rec % sub);
+      const long long kt = rec / sub;
+      const int NT = N / 256;
+      const long long kb = kt / NT, tile = kt % NT;
+      canon = (kb * sub + r) * (long long)N + tile * 256 + (x & 192) + c64;
+    }
     if (inverse)
       out[canon] = in[x];
     else
@@ -131,13 +145,19 @@ cudaError_t launch_pack_dense(uint32_t* q, uint16_t* s, uint32_t* wq, uint16_t* 
     unpack_weights_kernel<<<blocks, threads, 0, stream>>>(wq, q, K, N);
   cudaError_t err = cudaGetLastError();
   if (err != cudaSuccess) return err;
-  long long ns = (long long)(K / G) * N;
+  return launch_permute_scales(s, sq, K, N, G, inverse, stream);
+}
+
+cudaError_t launch_permute_scales(uint16_t* s, uint16_t* sq, int K, int N, int G, bool inverse, cudaStream_t stream) {
+  const int threads = 256;
+  const long long ns = (long long)(K / G) * N;
+  const int sub = G < kTileK ? kTileK / G : 1;
   int sblocks = (int)((ns + threads - 1) / threads);
   if (sblocks > 148 * 16) sblocks = 148 * 16;
   if (!inverse)
-    permute_scales_kernel<<<sblocks, threads, 0, stream>>>(s, sq, ns, false);
+    permute_scales_kernel<<<sblocks, threads, 0, stream>>>(s, sq, ns, N, sub, false);
   else
-    permute_scales_kernel<<<sblocks, threads, 0, stream>>>(sq, s, ns, true);
+    permute_scales_kernel<<<sblocks, threads, 0, stream>>>(sq, s, ns, N, sub, true);
   return cudaGetLastError();
 }
 

@@ -146,21 +146,6 @@ __global__ void unpack_sparse_meta_kernel(const uint32_t* __restrict__ meta, uin
   }
 }
 
-__global__ void permute_scales_sp_kernel(const uint16_t* __restrict__ in, uint16_t* __restrict__ out, long long total,
-                                         bool inverse) {
-  for (long long x = blockIdx.x * (long long)blockDim.x + threadIdx.x; x < total;
-       x += (long long)gridDim.x * blockDim.x) {
-    const long long base = x & ~63LL;
-    const int pos = (int)(x & 63);
-    const int g = pos >> 3, j = (pos >> 1) & 3, b = pos & 1;
-    const long long canon = base + 16 * j + 8 * b + g;
-    if (inverse)
-      out[canon] = in[x];
-    else
-      out[x] = in[canon];
-  }
-}
-
 // ---- the wide layout (N % 256 == 0) ----------------------------------------------------------------
 __device__ __forceinline__ uint32_t permute_nibbles(uint32_t x, bool inverse) {
   // forward: value o (nibble o of x) goes to nibble (o >> 1) + 4(o & 1); inverse: the other way round
@@ -253,28 +238,27 @@ cudaError_t launch_pack_sparse24(uint32_t* qc, uint8_t* idx, uint16_t* s, uint32
                                  int N, int G, bool inverse, cudaStream_t stream) {
   const int threads = 256;
   const long long code_words = (long long)K * N / 16, meta_words = (long long)K * N / 32;
-  const long long ns = (long long)(K / G) * N;
   if (N % 256 == 0) {
     // the wide layout of the tcgen05 kernel
     if (!inverse) {
       wide_sparse_codes_kernel<<<grid_for(code_words, threads), threads, 0, stream>>>(qc, wq, K, N, false);
       wide_sparse_meta_pack_kernel<<<grid_for(meta_words, threads), threads, 0, stream>>>(idx, meta, K, N);
-      permute_scales_sp_kernel<<<grid_for(ns, threads), threads, 0, stream>>>(s, sq, ns, false);
+      if (launch_permute_scales(s, sq, K, N, G, false, stream) != cudaSuccess) return cudaGetLastError();
     } else {
       wide_sparse_codes_kernel<<<grid_for(code_words, threads), threads, 0, stream>>>(wq, qc, K, N, true);
       wide_sparse_meta_unpack_kernel<<<grid_for((long long)(K / 4) * N, threads), threads, 0, stream>>>(meta, idx, K, N);
-      permute_scales_sp_kernel<<<grid_for(ns, threads), threads, 0, stream>>>(sq, s, ns, true);
+      if (launch_permute_scales(s, sq, K, N, G, true, stream) != cudaSuccess) return cudaGetLastError();
     }
     return cudaGetLastError();
   }
   if (!inverse) {
     pack_sparse_codes_kernel<<<grid_for(code_words, threads), threads, 0, stream>>>(qc, wq, K, N);
     pack_sparse_meta_kernel<<<grid_for(meta_words, threads), threads, 0, stream>>>(idx, meta, K, N);
-    permute_scales_sp_kernel<<<grid_for(ns, threads), threads, 0, stream>>>(s, sq, ns, false);
+    if (launch_permute_scales(s, sq, K, N, G, false, stream) != cudaSuccess) return cudaGetLastError();
   } else {
     unpack_sparse_codes_kernel<<<grid_for(code_words, threads), threads, 0, stream>>>(wq, qc, K, N);
     unpack_sparse_meta_kernel<<<grid_for((long long)(K / 4) * N, threads), threads, 0, stream>>>(meta, idx, K, N);
-    permute_scales_sp_kernel<<<grid_for(ns, threads), threads, 0, stream>>>(sq, s, ns, true);
+    if (launch_permute_scales(s, sq, K, N, G, true, stream) != cudaSuccess) return cudaGetLastError();
   }
   return cudaGetLastError();
 }

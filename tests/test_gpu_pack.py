@@ -19,7 +19,8 @@ def marlin():
 
 
 @pytest.mark.parametrize("K,N,G", [(128, 64, 128), (256, 192, 128), (512, 320, 256), (1024, 1024, 1024),
-                                   (4096, 4096, 128), (11008, 4096, 128), (4096, 22016, -1)])
+                                   (4096, 4096, 128), (11008, 4096, 128), (4096, 22016, -1),
+                                   (256, 256, 64), (1024, 768, 32), (4096, 4096, 64)])
 def test_pack_matches_layout_reference_and_round_trips(marlin, oracle_lib, K, N, G):
     from oracle import layout_ref
     case = inputs.make_dense(1, K, N, G, seed=K + N)
@@ -27,7 +28,7 @@ def test_pack_matches_layout_reference_and_round_trips(marlin, oracle_lib, K, N,
     w, s = marlin.pack(to_dev(case.q_kpacked), to_dev(case.S), G)
     Q = oracle_lib.unpack_q(case.q_kpacked)
     want_w = layout_ref.pack_dense_weights(Q)
-    want_s = layout_ref.pack_scales(case.S)
+    want_s = layout_ref.pack_scales(case.S, sub=max(1, 128 // Gn))
     assert np.array_equal(to_host(w).view(np.uint32), want_w)
     assert np.array_equal(to_host(s).view(np.uint16), want_s.view(np.uint16).reshape(-1))
     q2, s2 = marlin.unpack(w, s, K, N, G)
@@ -59,5 +60,11 @@ def test_pack_rejects_bad_arguments(marlin):
     q = torch.zeros((32, 128), dtype=torch.int32, device="cuda")  # K = 256
     s = torch.ones((4, 128), dtype=torch.float16, device="cuda")
     with pytest.raises(marlin.MarlinError) as e:
-        marlin.pack(q, s, 64)  # group size must be a multiple of 128
+        marlin.pack(q, s, 64)  # groups of 64 rows need N to be a multiple of 256
     assert e.value.status == 3
+    q = torch.zeros((32, 256), dtype=torch.int32, device="cuda")
+    for bad_g in (16, 48, 96, 100):  # neither 32, 64, a multiple of 128 nor K
+        s = torch.ones((max(1, 256 // bad_g), 256), dtype=torch.float16, device="cuda")
+        with pytest.raises(marlin.MarlinError) as e:
+            marlin.pack(q, s, bad_g)
+        assert e.value.status == 3

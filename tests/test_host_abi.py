@@ -45,7 +45,11 @@ def test_size_queries(marlin):
     assert L.marlin_packed_scale_bytes(4096, 4096, 128) == 2 * 32 * 4096
     assert L.marlin_packed_scale_bytes(4096, 4096, -1) == 2 * 4096
     assert L.marlin_packed_scale_bytes(4096, 4096, 4096) == 2 * 4096
-    assert L.marlin_packed_scale_bytes(4096, 4096, 100) == 0     # not a multiple of 128
+    assert L.marlin_packed_scale_bytes(4096, 4096, 100) == 0     # not 32, 64, a multiple of 128 or K
+    assert L.marlin_packed_scale_bytes(4096, 4096, 64) == 2 * 64 * 4096
+    assert L.marlin_packed_scale_bytes(4096, 4096, 32) == 2 * 128 * 4096
+    assert L.marlin_packed_scale_bytes(4096, 4160, 64) == 0      # groups of 64 rows need N % 256 == 0
+    assert L.marlin_packed_scale_bytes(4096, 4096, 16) == 0
     assert L.marlin_packed_scale_bytes(4096, 4096, 384) == 0     # does not divide K
     assert L.marlin_packed_weight_bytes(4000, 4096, 0) == 0      # K % 128
     assert L.marlin_packed_weight_bytes(4096, 4000, 0) == 0      # N % 64
