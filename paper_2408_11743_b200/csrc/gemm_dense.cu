@@ -119,7 +119,9 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
   uint8_t* stage0 = smem + G::FIXED_BYTES;
   const uint32_t stage0_s = smem_u32(stage0);
 
-  const int warp = threadIdx.x >> 5;
+  // the warp index, broadcast from lane 0 so that the compiler knows it is the same in all lanes (every role branch
+  // and loop bound below depends on it: otherwise each warp-wide instruction gets a divergence check)
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
   const int lane = threadIdx.x & 31;
   const uint32_t worker = blockIdx.x;
   const uint32_t U = p.units, P = p.workers, KB = p.kb;
@@ -147,6 +149,8 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
     // take the stages round-robin: issuing a bulk or tensor copy occupies a warp for a few hundred
     // cycles whatever the size of the copy, so several warps issue in parallel.
     const int pw = warp - kConsumerWarps;
+    // give the registers away first: the consumers' setmaxnreg.inc retries until they are in the pool
+    setmaxnreg_dec<kProducerRegs>();
     if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
     const uint64_t pol_w = policy_evict_first();
     const uint64_t pol_a = policy_evict_last();
@@ -192,7 +196,6 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
       }
     }
     __syncwarp();
-    setmaxnreg_dec<kProducerRegs>();
     pdl_wait_prior_grids();
     u = u0 + pw;
     s = pw;

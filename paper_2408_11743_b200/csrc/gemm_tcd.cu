@@ -137,7 +137,9 @@ gemm_tcd_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a) 
   uint8_t* stage0 = smem + G::FIXED_BYTES;
   const uint32_t stage0_s = smem_u32(stage0);
 
-  const int warp = threadIdx.x >> 5;
+  // the warp index, broadcast from lane 0 so that the compiler knows it is the same in all lanes (every role branch
+  // and loop bound below depends on it: otherwise each warp-wide instruction gets a divergence check)
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
   const int lane = threadIdx.x & 31;
   const uint32_t worker = blockIdx.x;
   const uint32_t U = p.units, P = p.workers, KB = p.kb;
