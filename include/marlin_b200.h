@@ -67,7 +67,9 @@ MARLIN_API size_t marlin_packed_scale_bytes(int K, int N, int group_size);
 MARLIN_API size_t marlin_packed_meta_bytes(int K, int N);
 /* Bytes of the workspace marlin_gemm* needs for any M <= max_M on this K x N layer.
  * The workspace holds a status word, per-column-tile arrival counters and the fp32 partial tiles
- * of the stripe fix-up (the global reduction of Section 3.4 "Striped Partitioning").
+ * of the stripe fix-up (the global reduction of Section 3.4 "Striped Partitioning"); it grows with max_M up
+ * to 128 rows and, above, with the number of (column tile, 128-row slab) pairs up to the number of CTAs
+ * (at most 20 MB).
  * The caller zeroes it ONCE after allocation (cudaMemset); every call leaves the counters zero.
  * One workspace must not be used by two calls that can run at the same time. */
 MARLIN_API size_t marlin_workspace_bytes(int max_M, int K, int N);
@@ -101,13 +103,15 @@ MARLIN_API int marlin_unpack(const void* w_packed, const void* s_packed, uint32_
  * the fp32 sums per group) or as fp16((q - 8) * s) (tcgen05 kernel with in-loop scales, from 17 rows: one more
  * rounding of 2^-11 per weight, as in the paper's kernel).
  * Up to 16 rows the warp-level kernel runs and the same inputs give the same bits on every call.
- * From 17 rows a tcgen05 kernel takes over: 128 rows per launch where N is a multiple of 256, 64 rows per
- * launch where N is a multiple of 128 only; any other N goes through the warp-level kernel in slabs of 16
- * rows.  Groups of 64 or 32 rows run on the tcgen05 kernel at every batch size.  Where the 256-column
- * tcgen05 kernel adds the partial sums of a column tile shared by several CTAs through the L2 (up to 32
- * rows, or shapes whose CTAs do not fit as one wave of thread-block clusters) the fp32 additions happen in
- * arrival order, so the last bit of an fp16 result can differ between two calls; everywhere else the order
- * is fixed.
+ * From 17 rows a tcgen05 kernel takes over.  Where N is a multiple of 256 one launch takes all rows: above
+ * 128 rows the layer is replicated in the numbering of the work units, once per slab of 128 rows (Section 3.4,
+ * last paragraph), and the stripes of the CTAs run over (column tile, slab, k-block), so the weights come from
+ * DRAM once and from the L2 after that.  Where N is a multiple of 128 only, 64 rows per launch; any other N goes
+ * through the warp-level kernel in slabs of 16 rows.  Groups of 64 or 32 rows run on the tcgen05 kernel at
+ * every batch size.  Where the 256-column tcgen05 kernel adds the partial sums of a column tile shared by
+ * several CTAs through the L2 (up to 32 rows, above 128 rows, or shapes whose CTAs do not fit as one wave of
+ * thread-block clusters) the fp32 additions happen in arrival order, so the last bit of an fp16 result can
+ * differ between two calls; everywhere else the order is fixed.
  * Errors: argument checks return before anything is queued.  A kernel whose bounded waits expire
  * sets the workspace status word; read it with marlin_read_status. */
 MARLIN_API int marlin_gemm(const void* A, const void* w_packed, const void* s_packed, void* C,
@@ -155,8 +159,9 @@ MARLIN_API int marlin_unpack_sparse24(const void* w_packed, const void* meta_pac
                            int K, int N, int group_size, marlin_stream stream);
 
 /* C = A . dequant(expand(W)) with the pruned positions contributing zero.  Layers whose N is a multiple of 256
- * run on the sparse tcgen05 instruction (tcgen05.mma.sp) at every batch size, 128 rows per launch, reading the
- * compressed weights once per launch; other N on the warp-level sparse MMA in slabs of 16 rows. */
+ * run on the sparse tcgen05 instruction (tcgen05.mma.sp) at every batch size, all rows in one launch (slabs of
+ * 128 rows as in marlin_gemm), reading the compressed weights from DRAM once; other N on the warp-level sparse
+ * MMA in slabs of 16 rows. */
 MARLIN_API int marlin_gemm_sparse24(const void* A, const void* w_packed, const void* meta_packed,
                          const void* s_packed, void* C, int M, int K, int N, int group_size,
                          void* workspace, size_t workspace_bytes, marlin_stream stream);

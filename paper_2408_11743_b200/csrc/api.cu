@@ -123,7 +123,9 @@ static size_t mma_slot_bytes(int max_M, int N) {
 // sparse24: 2:4 layers on the wide layout run on the tcgen05 kernel at every batch size
 static size_t tc_tile_bytes(int max_M, int N, bool sparse24) {
   if ((!sparse24 && max_M < tc_min_m()) || N % 256) return 0;
-  return (size_t)N * (size_t)tc_mpad(max_M < kTcMaxSlabM ? max_M : kTcMaxSlabM) * sizeof(float);
+  // one tile of 256 columns x padded rows per column tile; above 128 rows per worker at most (one launch takes all rows)
+  return tc_fixup_tiles(max_M, N, kMaxWorkers) * 256 * (size_t)tc_mpad(max_M < kTcMaxSlabM ? max_M : kTcMaxSlabM) *
+         sizeof(float);
 }
 static size_t workspace_bytes_for(int max_M, int K, int N, bool sparse24) {
   (void)K;
@@ -189,8 +191,8 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
   while (m0 < M) {
     const int rem = M - m0;
     // Which kernel takes the next rows.  Up to 16: the warp-level kernel.  Above: the tcgen05 kernel with
-    // in-loop scales (128 rows per launch, N a multiple of 256), or the one with deferred scales (64 rows per
-    // launch, N a multiple of 128).  What none of them serves (2:4 layers, other N) goes through the warp-level
+    // in-loop scales (N a multiple of 256; all rows in one launch, slabs of 128 rows sharing its stripes), or the
+    // one with deferred scales (64 rows per launch, N a multiple of 128).  What none of them serves (2:4 layers, other N) goes through the warp-level
     // kernel in slabs of 16 rows.
     const int tmode = tcd_mode();
     // 2:4 layers whose N is a multiple of 256 are packed in the wide layout, which only the tcgen05 kernel reads:
@@ -202,7 +204,8 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
                          (tmode == 1 || (tmode == 2 && rem >= tc_min_m() && !tc_ok));
     const bool use_tc = !use_tcd && tc_ok && (sparse24 || small_groups || rem >= tc_min_m());
     const int m_slab = use_tcd ? (rem < kTcdMaxSlabM ? rem : kTcdMaxSlabM)
-                               : use_tc ? (rem < kTcMaxSlabM ? rem : kTcMaxSlabM) : (rem < kMaxSlabM ? rem : kMaxSlabM);
+                               : use_tc ? (rem < tc_max_rows(K, N, info.sm_count) ? rem : tc_max_rows(K, N, info.sm_count))
+                                        : (rem < kMaxSlabM ? rem : kMaxSlabM);
     GemmParams p;
     p.A = static_cast<const uint16_t*>(A) + (size_t)m0 * K;
     p.wq = static_cast<const uint8_t*>(w_packed);
@@ -225,6 +228,8 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
     p.tc_tiles = use_tc ? reinterpret_cast<float*>(ws + ((workspace_bytes & ~(size_t)255) - tc_tile_bytes(m_slab, N, sparse24 || small_groups)))
                         : nullptr;
     p.split = 0;
+    p.whole = 0;
+    p.slabs = 1;
     p.cluster = 0;
     p.slot_floats = kWsSlotCols * kMaxSlabM;
     if (use_tcd) {

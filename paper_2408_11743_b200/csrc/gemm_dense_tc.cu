@@ -1,5 +1,5 @@
-// Dense W4A16 layer for sm_100a, batch sizes 17..128 per launch: tcgen05 tensor cores with the WEIGHTS
-// as the A operand in tensor memory.
+// Dense W4A16 layer for sm_100a, batch sizes from 17 rows: tcgen05 tensor cores with the WEIGHTS as the A operand in
+// tensor memory, 128 batch rows per accumulator tile; larger batches are slabs of 128 rows inside one launch.
 //
 // The warp-level MMA (mma.sync) of the small-batch kernel runs at about a tenth of the tcgen05 rate on
 // this architecture and is out of steam above batch 16.  Here the product is computed transposed, as the
@@ -136,8 +136,13 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
   const uint32_t worker = blockIdx.x;
   const uint32_t U = p.units, P = p.workers, KB = p.kb;
   // split > 0: one k-range of one column tile per CTA (the last range of a tile ends where the next tile begins)
-  const uint32_t u0 = p.split ? split_begin32(worker, KB, p.split) : stripe_begin32(worker, U, P);
-  const uint32_t u1 = p.split ? split_begin32(worker + 1, KB, p.split) : stripe_begin32(worker + 1, U, P);
+  // whole: the stripes are cut at tile boundaries (many more tiles than workers: nothing is shared, no fix-up)
+  const uint32_t u0 = p.split   ? split_begin32(worker, KB, p.split)
+                      : p.whole ? stripe_begin32(worker, (uint32_t)p.ncols, P) * KB
+                                : stripe_begin32(worker, U, P);
+  const uint32_t u1 = p.split   ? split_begin32(worker + 1, KB, p.split)
+                      : p.whole ? stripe_begin32(worker + 1, (uint32_t)p.ncols, P) * KB
+                                : stripe_begin32(worker + 1, U, P);
 
   pdl_launch_dependents();
   if (threadIdx.x == 0) {
@@ -169,7 +174,8 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       // ------------------------------- producers --------------------------------------------
       const int pw = warp - kDequantWarps;
       if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
-      const uint64_t pol_w = policy_evict_first();
+      // one slab: every weight byte is read once; several slabs read the layer once each, from the L2 after the first
+      const uint64_t pol_w = p.slabs > 1 ? policy_evict_last() : policy_evict_first();
       const uint64_t pol_a = policy_evict_last();
       // weights and activations complete barriers of their own: the converting warps need only the former, and
       // on the first pass over the ring those arrive before the dependency wait
@@ -200,7 +206,8 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
 #endif
       if (lane == 0) {
         for (; u < u1 && s < NSTAGES; u += kTcProducerWarps, s += kTcProducerWarps) {
-          const uint32_t col = u / KB, kb = u - col * KB;
+          const uint32_t vcol = u / KB, kb = u - vcol * KB;
+          const uint32_t col = vcol / p.slabs;
           if (withhold && s == 1) continue;
           mbar_expect_tx(&full[s], tx_bytes);
           bulk_g2s(stage0 + (size_t)s * G::STAGE_BYTES + G::A_BYTES, weight_src(col, kb), G::W_BYTES, &full[s], pol_w);
@@ -215,17 +222,19 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       u = u0 + pw;
       s = pw;
       for (; u < u1 && s < NSTAGES; u += kTcProducerWarps, s += kTcProducerWarps) {
-        const uint32_t col = u / KB, kb = u - col * KB;
+        const uint32_t vcol = u / KB, kb = u - vcol * KB;
+        const uint32_t slab = vcol % p.slabs;
         if (lane == 0) mbar_expect_tx(&xfull[s], G::A_BYTES);
         __syncwarp();
         if (lane < 2)
           tma_load_2d(stage0 + (size_t)s * G::STAGE_BYTES + lane * G::A_HALF_BYTES, &tmap_a,
-                      (int)(kb * kTileK + lane * 64), 0, &xfull[s], pol_a);
+                      (int)(kb * kTileK + lane * 64), (int)(slab * MPAD), &xfull[s], pol_a);
       }
       uint32_t ph = 1;
       s -= NSTAGES;
       for (; u < u1; u += kTcProducerWarps) {
-        const uint32_t col = u / KB, kb = u - col * KB;
+        const uint32_t vcol = u / KB, kb = u - vcol * KB;
+        const uint32_t col = vcol / p.slabs, slab = vcol - col * p.slabs;
         // the stage is free when its codes are in registers and the MMAs that read its activations are done
         mbar_wait<200>(&empty[s], ph ^ 1u, abort_flag, p.status);
         mbar_wait<200>(&mdone[s], ph ^ 1u, abort_flag, p.status);
@@ -239,7 +248,8 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         }
         __syncwarp();
         if (lane < 2)
-          tma_load_2d(st + lane * G::A_HALF_BYTES, &tmap_a, (int)(kb * kTileK + lane * 64), 0, &xfull[s], pol_a);
+          tma_load_2d(st + lane * G::A_HALF_BYTES, &tmap_a, (int)(kb * kTileK + lane * 64), (int)(slab * MPAD), &xfull[s],
+                      pol_a);
         s += kTcProducerWarps;
         if (s >= NSTAGES) { s -= NSTAGES; ph ^= 1u; }
       }
@@ -336,7 +346,11 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
   uint32_t u = u0;
   bool waited_for_prior_grid = false;
   while (u < u1) {
-    const uint32_t col = u / KB;
+    // virtual column tile = (column tile of W, slab of MPAD batch rows): batches above 128 rows replicate the
+    // layer in the unit numbering (Section 3.4, last paragraph), slab after slab of one column tile
+    const uint32_t vcol = u / KB;
+    const uint32_t col = vcol / p.slabs, slab = vcol - col * p.slabs;
+    const int m_lim = p.M - (int)slab * MPAD;   // rows of this slab that exist
     const uint32_t kb0 = u % KB;
     const uint32_t len = min(KB - kb0, u1 - u);
     const uint16_t* sptr = reinterpret_cast<const uint16_t*>(p.sq) + (size_t)col * kTileN + spos;
@@ -434,9 +448,9 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       pdl_wait_prior_grids();
       waited_for_prior_grid = true;
     }
-    const int first_w = p.split ? (int)(col * p.split) : (int)stripe_owner32(col * KB, U, P);
-    const int last_w = p.split ? (int)(col * p.split + p.split - 1) : (int)stripe_owner32((col + 1) * KB - 1, U, P);
-    const bool shared_tile = last_w > first_w;
+    const int first_w = p.split ? (int)(vcol * p.split) : (int)stripe_owner32(vcol * KB, U, P);
+    const int last_w = p.split ? (int)(vcol * p.split + p.split - 1) : (int)stripe_owner32((vcol + 1) * KB - 1, U, P);
+    const bool shared_tile = !p.whole && last_w > first_w;
     if (p.cluster) {
       // The CTAs of this column tile form a thread-block cluster and finish side by side, so the partial
       // tiles never leave the SMs.  Every CTA puts its partial tile into its own stage ring (free by now), a
@@ -501,8 +515,8 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         for (int vec = ctid; vec < rows_here * (kTileN / 8); vec += kDequantThreads) {
           const int row = vec / (kTileN / 8), c16 = vec % (kTileN / 8);
           const int m = 4 * b0 + row;
-          if (m < p.M)
-            *reinterpret_cast<uint4*>(p.C + (size_t)m * p.N + (size_t)col * kTileN + c16 * 8) =
+          if (m < m_lim)
+            *reinterpret_cast<uint4*>(p.C + ((size_t)slab * MPAD + m) * p.N + (size_t)col * kTileN + c16 * 8) =
                 *reinterpret_cast<const uint4*>(out + row * kTileN + c16 * 8);
         }
       }
@@ -516,48 +530,50 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
     // (float4 index = (m / 4) * 256 + column: coalesced over columns), the last arriver reads the
     // total, clears the buffer for the next call and stores C.  (The order of these fp32 additions
     // is not fixed, so the last bits of a shared tile can differ from run to run.)
-    float4* mine = reinterpret_cast<float4*>(p.tc_tiles + (size_t)col * (kTileN * MPAD)) + n256;
-    uint16_t* cptr = p.C + (size_t)col * kTileN + n256;
-    // 32 batch rows at a time: accumulators out of tensor memory, then either to the L2 or straight to C
-#pragma unroll 1
+    // One accumulation tile and one counter per virtual column tile; where there are more of those than workers,
+    // per tile that can be shared, numbered by the first worker on it (at most one tile runs over the end of a
+    // worker's stripe).
+    const uint32_t fix = (uint32_t)p.ncols <= P ? vcol : (uint32_t)first_w;
+    float4* mine = reinterpret_cast<float4*>(p.tc_tiles + (size_t)fix * (kTileN * MPAD)) + n256;
+    uint16_t* cptr = p.C + (size_t)slab * MPAD * p.N + (size_t)col * kTileN + n256;
+    // All accumulators of this thread's channel out of tensor memory first: the MMAs of the next segment may then
+    // start while the partial tile goes to the L2 or C is stored.
+    float acc[MPAD];
+#pragma unroll
     for (int cc = 0; cc < MPAD / 32; ++cc) {
-      float part[32];
-      tc_ld_x32(tmem_lane + (uint32_t)(tile * KH * MPAD + cc * 32), part);
+      tc_ld_x32(tmem_lane + (uint32_t)(tile * KH * MPAD + cc * 32), reinterpret_cast<float(&)[32]>(acc[32 * cc]));
       if constexpr (KH == 2) {
         float part2[32];
         tc_ld_x32(tmem_lane + (uint32_t)((tile * KH + 1) * MPAD + cc * 32), part2);
         tc_wait_ld();
 #pragma unroll
-        for (int e = 0; e < 32; ++e) part[e] += part2[e];
-      } else {
-        tc_wait_ld();
-      }
-      if constexpr (!GR) {
-#pragma unroll
-        for (int e = 0; e < 32; ++e) part[e] *= sc_col;
-      }
-      if (shared_tile) {
-#pragma unroll
-        for (int m4 = 0; m4 < 8; ++m4)
-          red_add_f32x4(mine + (cc * 8 + m4) * kTileN, part[4 * m4], part[4 * m4 + 1], part[4 * m4 + 2], part[4 * m4 + 3]);
-      } else {
-#pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const int m = cc * 32 + e;
-          if (m < p.M) cptr[(size_t)m * p.N] = __half_as_ushort(__float2half_rn(part[e]));
-        }
+        for (int e = 0; e < 32; ++e) acc[32 * cc + e] += part2[e];
       }
     }
+    tc_wait_ld();
     tc_fence_before_sync();
     __syncwarp();
     if (lane == 0) mbar_arrive(dempty);
+    if constexpr (!GR) {
+#pragma unroll
+      for (int e = 0; e < MPAD; ++e) acc[e] *= sc_col;
+    }
+    if (shared_tile) {
+#pragma unroll
+      for (int m4 = 0; m4 < MPAD / 4; ++m4)
+        red_add_f32x4(mine + m4 * kTileN, acc[4 * m4], acc[4 * m4 + 1], acc[4 * m4 + 2], acc[4 * m4 + 3]);
+    } else {
+#pragma unroll
+      for (int m = 0; m < MPAD; ++m)
+        if (m < m_lim) cptr[(size_t)m * p.N] = __half_as_ushort(__float2half_rn(acc[m]));
+    }
 
     if (shared_tile) {
       named_bar_sync(1, kDequantThreads);
       if (ctid == 0) {
-        const int old = atom_add_acq_rel_gpu(&p.counters[col], 1);
+        const int old = atom_add_acq_rel_gpu(&p.counters[fix], 1);
         const int is_last = (old == last_w - first_w) ? 1 : 0;
-        if (is_last) p.counters[col] = 0;
+        if (is_last) p.counters[fix] = 0;
         *last_flag = is_last;
       }
       named_bar_sync(1, kDequantThreads);
@@ -571,10 +587,10 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
 #pragma unroll
         for (int m4 = 0; m4 < MPAD / 4; ++m4) {
           const int m = 4 * m4;
-          if (m < p.M) cptr[(size_t)m * p.N] = __half_as_ushort(__float2half_rn(t4[m4].x));
-          if (m + 1 < p.M) cptr[(size_t)(m + 1) * p.N] = __half_as_ushort(__float2half_rn(t4[m4].y));
-          if (m + 2 < p.M) cptr[(size_t)(m + 2) * p.N] = __half_as_ushort(__float2half_rn(t4[m4].z));
-          if (m + 3 < p.M) cptr[(size_t)(m + 3) * p.N] = __half_as_ushort(__float2half_rn(t4[m4].w));
+          if (m < m_lim) cptr[(size_t)m * p.N] = __half_as_ushort(__float2half_rn(t4[m4].x));
+          if (m + 1 < m_lim) cptr[(size_t)(m + 1) * p.N] = __half_as_ushort(__float2half_rn(t4[m4].y));
+          if (m + 2 < m_lim) cptr[(size_t)(m + 2) * p.N] = __half_as_ushort(__float2half_rn(t4[m4].z));
+          if (m + 3 < m_lim) cptr[(size_t)(m + 3) * p.N] = __half_as_ushort(__float2half_rn(t4[m4].w));
         }
       }
       named_bar_sync(1, kDequantThreads);  // last_flag may be rewritten by the next segment
@@ -641,17 +657,37 @@ cudaError_t launch_tc(const GemmParams& p, int workers, cudaStream_t stream) {
 
 
 bool tc_path_supported(int m_slab, int K, int N) {
-  return m_slab >= 1 && m_slab <= kTcMaxSlabM && N % kTileN == 0 && K % kTileK == 0;
+  return m_slab >= 1 && N % kTileN == 0 && K % kTileK == 0;
+}
+
+int tc_max_rows(int K, int N, int sm_count) {
+  // the device's 32-bit stripe arithmetic: slabs * tiles * k-blocks * workers stays below 2^31
+  const long long per_slab = (long long)(N / kTileN) * (K / kTileK) * (sm_count < kMaxWorkers ? sm_count : kMaxWorkers);
+  long long slabs = ((1ll << 31) - 1) / per_slab;
+  if (slabs < 1) slabs = 1;
+  if (slabs > (1 << 16)) slabs = 1 << 16;
+  return (int)slabs * kTcMaxSlabM;
+}
+
+size_t tc_fixup_tiles(int M, int N, int workers) {
+  // accumulation tiles of the fix-up: one per column tile up to 128 rows; above, one per (column tile, slab) or, if
+  // those outnumber the workers, one per worker
+  if (M <= kTcMaxSlabM) return (size_t)(N / kTileN);
+  const long long vcols = (long long)(N / kTileN) * ((M + kTcMaxSlabM - 1) / kTcMaxSlabM);
+  return (size_t)(vcols < workers ? vcols : workers);
 }
 
 int tc_mpad(int m_slab) { return m_slab <= 32 ? 32 : (m_slab <= 64 ? 64 : 128); }
 
 cudaError_t launch_gemm_dense_tc(GemmParams p, int sm_count, bool sparse24, cudaStream_t stream) {
   // stripe plan for 256-column tiles
-  const long long units = (long long)(p.N / kTileN) * (p.K / kTileK);
+  // above 128 rows the layer is replicated in the unit numbering, once per slab of 128 rows (Section 3.4, last
+  // paragraph): one launch, its stripes running over (column tile, slab, k-block)
+  p.slabs = (uint32_t)((p.M + kTcMaxSlabM - 1) / kTcMaxSlabM);
+  p.ncols = (p.N / kTileN) * (int)p.slabs;
+  const long long units = (long long)p.ncols * (p.K / kTileK);
   long long workers = sm_count < kMaxWorkers ? sm_count : kMaxWorkers;
   if (workers > units) workers = units;
-  p.ncols = p.N / kTileN;
   p.units = (uint32_t)units;
   // With up to 128 rows the epilogue of a segment (accumulators out of tensor memory, L2 reductions, arrival
   // count) takes microseconds during which the CTA converts nothing, and under even stripes most CTAs run it
@@ -673,8 +709,15 @@ cudaError_t launch_gemm_dense_tc(GemmParams p, int sm_count, bool sparse24, cuda
     // from 33 rows up: below that the partial tiles are small and the L2 path is as fast
     p.cluster = (p.split >= 2 && p.M > 32 && !(e && atoi(e) == 0)) ? 1u : 0u;
   }
+  // Many more (column tile, slab) pairs than workers: stripes cut at tile boundaries leave little imbalance and need
+  // no fix-up at all.
+  p.whole = 0;
+  if (p.split == 0 && p.ncols >= workers) {
+    const long long per = (p.ncols + workers - 1) / workers;
+    if (per * workers * 100 <= (long long)p.ncols * 106) p.whole = 1;
+  }
   p.workers = (uint32_t)workers;
-  const int mpad = tc_mpad(p.M);
+  const int mpad = tc_mpad(p.M < kTcMaxSlabM ? p.M : kTcMaxSlabM);
   if (sparse24) {
     if (p.grouped) {
       if (mpad == 32) return launch_tc<32, true, true>(p, (int)workers, stream);

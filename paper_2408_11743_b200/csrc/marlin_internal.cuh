@@ -77,6 +77,9 @@ struct GemmParams {
   float* tc_tiles;   // tcgen05 kernel: one fp32 accumulation tile per 256-column tile
   int slot_floats;   // floats per partial-tile slot
   uint32_t cluster;  // tcgen05 kernel: 1 = launched as thread-block clusters of `split` CTAs (the CTAs of one column tile)
+  uint32_t slabs;    // tcgen05 kernel: slabs of 128 batch rows in this launch (1 up to 128 rows); virtual column tile
+                     // v = column tile v / slabs of W, batch rows 128 * (v % slabs) ..
+  uint32_t whole;    // tcgen05 kernel: 1 = worker w owns the virtual column tiles [w * ncols / P, (w + 1) * ncols / P) whole
   uint32_t split;    // tcgen05 kernel: 0 = even stripes over all units; S > 0 = every column tile is cut into S
                      // k-ranges and worker w owns range w % S of tile w / S (one segment per CTA)
 };
@@ -88,6 +91,8 @@ cudaError_t launch_pack_sparse24(uint32_t* qc, uint8_t* idx, uint16_t* s, uint32
 // tcgen05 kernel (gemm_dense_tc.cu): 256-column tiles, up to 128 rows of A per launch.
 bool tc_path_supported(int m_slab, int K, int N);
 int tc_mpad(int m_slab);  // rows of A padded to the MMA's N: 32, 64 or 128
+int tc_max_rows(int K, int N, int sm_count);      // most rows one launch takes (a multiple of 128)
+size_t tc_fixup_tiles(int M, int N, int workers); // fp32 accumulation tiles (256 columns x padded rows) the fix-up needs
 // fills the plan fields of `p` (ncols, units, workers) itself; sparse24: the 2:4 instances (tcgen05.mma.sp), which read
 // the wide 2:4 layout (N a multiple of 256)
 cudaError_t launch_gemm_dense_tc(GemmParams p, int sm_count, bool sparse24, cudaStream_t stream);

@@ -31,3 +31,19 @@ class DenseLayer:
         torch.cuda.synchronize()
         assert self.m.read_status(self.ws) == 0
         return to_host(out)
+
+
+class SparseLayer:
+    """A packed 2:4 layer resident on the GPU, built through marlin_pack_sparse24 from a generated case."""
+
+    def __init__(self, marlin, case, max_M):
+        self.m, self.K, self.N, self.G = marlin, case.K, case.N, case.G
+        self.w, self.meta, self.s = marlin.pack_sparse24(to_dev(case.qc_kpacked), to_dev(case.idx), to_dev(case.S), case.G)
+        self.ws = marlin.new_workspace(max_M, self.K, self.N)
+
+    def __call__(self, A):
+        import torch
+        out = self.m.gemm_sparse24(to_dev(A), self.w, self.meta, self.s, self.K, self.N, self.G, self.ws)
+        torch.cuda.synchronize()
+        assert self.m.read_status(self.ws) == 0
+        return to_host(out)

@@ -3,7 +3,7 @@ import numpy as np
 import pytest
 
 from paper_2408_11743_b200 import inputs
-from gpu_util import DenseLayer, to_dev, to_host
+from gpu_util import DenseLayer, SparseLayer, to_dev, to_host
 
 pytestmark = pytest.mark.gpu
 
@@ -15,20 +15,6 @@ def marlin():
     import paper_2408_11743_b200 as m
     m.lib()
     return m
-
-
-class SparseLayer:
-    def __init__(self, marlin, case, max_M):
-        self.m, self.K, self.N, self.G = marlin, case.K, case.N, case.G
-        self.w, self.meta, self.s = marlin.pack_sparse24(to_dev(case.qc_kpacked), to_dev(case.idx), to_dev(case.S), case.G)
-        self.ws = marlin.new_workspace(max_M, self.K, self.N)
-
-    def __call__(self, A):
-        import torch
-        out = self.m.gemm_sparse24(to_dev(A), self.w, self.meta, self.s, self.K, self.N, self.G, self.ws)
-        torch.cuda.synchronize()
-        assert self.m.read_status(self.ws) == 0
-        return to_host(out)
 
 
 def _codes(qk):
