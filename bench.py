@@ -258,7 +258,8 @@ class LayerBench:
 
 def extra_layers(marlin, dev, stream, l2, peaks, capture, time_graph):
     """Per-layer numbers outside the timed step: every layer and batch size of configs 3 (Llama-2-7B shapes), 4
-    (Llama-2-70B shapes, group 128 and one scale per column) and 5 (the 2:4 layer, with the dense layer beside it)."""
+    (Llama-2-70B shapes, group 128 and one scale per column) and 5 (the 2:4 layer, with the dense layer beside it),
+    and batches of 256 to 4096 rows on two layers."""
     import torch
     out = []
     rng = np.random.default_rng(1234)
@@ -275,6 +276,23 @@ def extra_layers(marlin, dev, stream, l2, peaks, capture, time_graph):
     for name, K, N in inputs.LLAMA7B_LAYERS:
         sweep(K, N, GROUP, False, (1, 16, 32, 64, 128), "llama2-7b " + name, 3)
     sweep(8192, 8192, GROUP, True, (16, 32, 64, 128), "2:4 sparse 8192x8192", 5)
+    # batches above 128 rows (Section 5.1 "Large batch performance"): one launch, tensor-bound; roofline_frac is taken
+    # against the measured dense bf16 GEMM peak there, cublas_fp16_us is the uncompressed layer through torch.matmul
+    sweep(8192, 8192, GROUP, False, (256, 512, 1024, 2048, 4096), "large batch 8192x8192", 2)
+    sweep(4096, 22016, GROUP, False, (256, 1024, 4096), "large batch llama2-7b gate_up", 3)
+    # the offline quantiser in front of the pack (Section 3.5 (a)): fp16 weights -> codes and scales, 10 clipping
+    # candidates per group; bounded by the arithmetic of the search (the algorithmic bytes are 2.5 per weight)
+    for nc in (1, 10):
+        Wq = torch.randn((8192, 8192), device=dev, dtype=torch.float32).mul_(0.02).half()
+        with torch.cuda.stream(stream):
+            marlin.quantize_rtn(Wq, GROUP, 20, nc, stream=stream)
+        torch.cuda.synchronize(dev)
+        g = capture(lambda: marlin.quantize_rtn(Wq, GROUP, 20, nc, stream=stream), 2)
+        tq = min(time_graph(g) for _ in range(3)) / 2
+        out.append({"layer": "quantize_rtn 8192x8192", "config": "front end", "G": GROUP, "n_grid": 20, "n_candidates": nc,
+                    "us": round(tq * 1e6, 1), "gweights_per_s": round(8192 * 8192 / tq / 1e9, 1),
+                    "algorithmic_gbs": round((8192 * 8192 * 2.5 + 2 * 64 * 8192) / tq / 1e9, 1)})
+        del Wq
     for name, K, N in inputs.LLAMA70B_LAYERS:
         for G in (GROUP, K):
             sweep(K, N, G, False, (1, 16, 64, 128),

@@ -74,6 +74,23 @@ MARLIN_API size_t marlin_packed_meta_bytes(int K, int N);
  * One workspace must not be used by two calls that can run at the same time. */
 MARLIN_API size_t marlin_workspace_bytes(int max_M, int K, int N);
 
+/* ---- offline quantiser (Section 3.5 (a): group scales picked by a search over group-wise clipping
+ *      thresholds; here without calibration data: round to nearest, least squared weight error) ------ */
+
+/* fp16 weights -> canonical 4-bit codes and fp16 group scales, the inputs of marlin_pack.
+ *   W             device, fp16 [K][N] row-major, finite values
+ *   q_kpacked     device, out, uint32 [K/8][N]: nibble j of word (kb, n) = code of row 8*kb + j, codes 0..15 = q
+ *   scales        device, out, fp16 [K/G][N]
+ *   n_grid, n_candidates   1 <= n_candidates <= n_grid: candidate t = 0 .. n_candidates-1 clips the group's range
+ *                 to r_t = 1 - t / n_grid of its largest magnitude a (n_candidates = 1: plain round to nearest)
+ * Per group of G rows of a column: s_t = fp16(2 a r_t / 15) (never zero: at least the smallest positive fp16),
+ * q_i = clamp(round_half_even(w_i / s_t), -8, 7) + 8, and the candidate with the least sum of squared errors
+ * (w_i - (q_i - 8) s_t)^2 wins, the first one on ties.  All of it in fp32 with a fixed order of operations (see
+ * csrc/quantize.cu), so the outputs are reproducible bit for bit.  Shapes and group sizes as for marlin_pack;
+ * pointers 16-byte aligned; errors are returned before anything is queued. */
+MARLIN_API int marlin_quantize_rtn(const void* W, uint32_t* q_kpacked, void* scales, int K, int N, int group_size,
+                        int n_grid, int n_candidates, marlin_stream stream);
+
 /* ---- offline re-layout (Section 3.4 "Maximizing Loading Bandwidth", "Dequantization and Tensor
  *      Cores": weights are static, so they are reshuffled once into the order the kernel streams) -- */
 

@@ -15,6 +15,7 @@ from .binding import (  # noqa: F401
     pack,
     pack_sparse24,
     plan_stripes,
+    quantize_rtn,
     read_status,
     unpack,
     unpack_sparse24,

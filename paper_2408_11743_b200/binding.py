@@ -17,7 +17,7 @@ EXPORTS = [
     "marlin_status_string", "marlin_packed_weight_bytes", "marlin_packed_scale_bytes", "marlin_packed_meta_bytes",
     "marlin_workspace_bytes", "marlin_pack", "marlin_unpack", "marlin_gemm", "marlin_pack_sparse24",
     "marlin_unpack_sparse24", "marlin_gemm_sparse24", "marlin_read_status", "marlin_plan_stripes",
-    "marlin_gemm_static_ws",
+    "marlin_gemm_static_ws", "marlin_quantize_rtn",
 ]
 STATIC_WS_MAX_M = 16  # MARLIN_STATIC_WS_MAX_M of the header
 
@@ -57,6 +57,7 @@ def lib():
     L.marlin_workspace_bytes.argtypes = [i, i, i]
     L.marlin_pack.argtypes = [vp, vp, vp, vp, i, i, i, vp]
     L.marlin_unpack.argtypes = [vp, vp, vp, vp, i, i, i, vp]
+    L.marlin_quantize_rtn.argtypes = [vp, vp, vp, i, i, i, i, i, vp]
     L.marlin_gemm.argtypes = [vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
     L.marlin_gemm_static_ws.argtypes = [vp, vp, vp, vp, i, i, i, i, vp]
     L.marlin_pack_sparse24.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, vp]
@@ -64,7 +65,7 @@ def lib():
     L.marlin_gemm_sparse24.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
     L.marlin_read_status.argtypes = [vp, vp]
     L.marlin_plan_stripes.argtypes = [i, i, i, i, vp, vp, vp, i]
-    for name in ("marlin_gemm_static_ws", "marlin_pack", "marlin_unpack", "marlin_gemm", "marlin_pack_sparse24", "marlin_unpack_sparse24",
+    for name in ("marlin_quantize_rtn", "marlin_gemm_static_ws", "marlin_pack", "marlin_unpack", "marlin_gemm", "marlin_pack_sparse24", "marlin_unpack_sparse24",
                  "marlin_gemm_sparse24", "marlin_read_status", "marlin_plan_stripes"):
         getattr(L, name).restype = i
     _lib = L
@@ -109,6 +110,28 @@ def new_workspace(max_M: int, K: int, N: int, device="cuda"):
     """Allocates the workspace with torch and zeroes it once, as the C ABI requires."""
     torch = _torch()
     return torch.zeros(workspace_bytes(max_M, K, N), dtype=torch.uint8, device=device)
+
+
+def quantize_rtn(W, group_size: int, n_grid: int = 20, n_candidates: int = 10, stream=None):
+    """marlin_quantize_rtn: fp16 weights [K, N] -> (q_kpacked int32 [K/8, N], scales fp16 [K/G, N]), the inputs of pack.
+
+    Round to nearest with a per-group search over n_candidates clipping thresholds 1 - t / n_grid."""
+    torch = _torch()
+    W = _dev(W, torch.float16, "W")
+    if W.dim() != 2:
+        raise ValueError("W must be [K, N]")
+    K, N = W.shape
+    L = lib()
+    sb = L.marlin_packed_scale_bytes(K, N, group_size)
+    if L.marlin_packed_weight_bytes(K, N, 0) == 0:
+        raise MarlinError(2, "marlin_quantize_rtn")
+    if sb == 0:
+        raise MarlinError(3, "marlin_quantize_rtn")
+    q = torch.empty((K // 8, N), dtype=torch.int32, device=W.device)
+    s = torch.empty((sb // (2 * N), N), dtype=torch.float16, device=W.device)
+    _check(L.marlin_quantize_rtn(W.data_ptr(), q.data_ptr(), s.data_ptr(), K, N, group_size, n_grid, n_candidates,
+                                 _stream_ptr(stream)), "marlin_quantize_rtn")
+    return q, s
 
 
 def pack(q_kpacked, scales, group_size: int, stream=None):

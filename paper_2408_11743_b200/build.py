@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libmarlin_b200.so")
-SOURCES = ["api.cu", "pack.cu", "pack_sparse.cu", "gemm_dense.cu", "gemm_dense_tc.cu", "gemm_tcd.cu"]
+SOURCES = ["api.cu", "pack.cu", "pack_sparse.cu", "quantize.cu", "gemm_dense.cu", "gemm_dense_tc.cu", "gemm_tcd.cu"]
 HEADERS = [os.path.join(CSRC, "marlin_internal.cuh"), os.path.join(CSRC, "device_utils.cuh"), os.path.join(CSRC, "tc_utils.cuh"), os.path.join(_ROOT, "include", "marlin_b200.h")]
 
 NVCC_FLAGS = [

@@ -154,6 +154,20 @@ int marlin_pack(const uint32_t* q_kpacked, const void* scales, void* w_packed, v
   return err == cudaSuccess ? MARLIN_OK : MARLIN_ERR_CUDA;
 }
 
+int marlin_quantize_rtn(const void* W, uint32_t* q_kpacked, void* scales, int K, int N, int group_size, int n_grid,
+                        int n_candidates, marlin_stream stream) {
+  if (!W || !q_kpacked || !scales) return MARLIN_ERR_NULL;
+  if (!shape_ok(K, N)) return MARLIN_ERR_SHAPE;
+  int G = normalise_group(K, N, group_size);
+  if (!G) return MARLIN_ERR_GROUP;
+  if (n_grid < 1 || n_candidates < 1 || n_candidates > n_grid) return MARLIN_ERR_SHAPE;
+  if (!aligned16(W) || !aligned16(q_kpacked) || !aligned16(scales)) return MARLIN_ERR_ALIGN;
+  if ((long long)(K / G) > 65535) return MARLIN_ERR_SHAPE;  // one grid row per group
+  cudaError_t err = launch_quantize_rtn(static_cast<const uint16_t*>(W), q_kpacked, static_cast<uint16_t*>(scales), K, N, G,
+                                        n_grid, n_candidates, static_cast<cudaStream_t>(stream));
+  return err == cudaSuccess ? MARLIN_OK : MARLIN_ERR_CUDA;
+}
+
 int marlin_unpack(const void* w_packed, const void* s_packed, uint32_t* q_kpacked, void* scales, int K, int N,
                   int group_size, marlin_stream stream) {
   if (!q_kpacked || !scales || !w_packed || !s_packed) return MARLIN_ERR_NULL;

@@ -105,6 +105,9 @@ cudaError_t launch_gemm_tcd(GemmParams p, int sm_count, cudaStream_t stream);
 // inverse == false: (q, s) canonical inputs -> (wq, sq) packed outputs; inverse == true: the other way round.
 cudaError_t launch_pack_dense(uint32_t* q, uint16_t* s, uint32_t* wq, uint16_t* sq, int K, int N, int G, bool inverse,
                               cudaStream_t stream);
+// round-to-nearest quantiser with clipping search (quantize.cu): W fp16 [K][N] -> canonical codes and scales
+cudaError_t launch_quantize_rtn(const uint16_t* W, uint32_t* q_kpacked, uint16_t* scales, int K, int N, int G, int n_grid,
+                                int n_candidates, cudaStream_t stream);
 // canonical scales [K/G][N] <-> packed order (shared by the dense and the 2:4 pack)
 cudaError_t launch_permute_scales(uint16_t* s, uint16_t* sq, int K, int N, int G, bool inverse, cudaStream_t stream);
 
