@@ -107,6 +107,15 @@ MARLIN_API int marlin_pack(const uint32_t* q_kpacked, const void* scales, void* 
 MARLIN_API int marlin_unpack(const void* w_packed, const void* s_packed, uint32_t* q_kpacked, void* scales,
                   int K, int N, int group_size, marlin_stream stream);
 
+/* Zero points for layers quantised asymmetrically, W = (q - z) * s with one integer z in 0..15 per scale group
+ * (Section 2.3 "uniform quantization": a zero point and a scale per group; the integer form is the one of the
+ * activation-aware format the paper names in Section 6).  Codes and scales go through marlin_pack as usual.
+ *   zeros      device, uint8 [K/G][N] row-major, values 0..15
+ *   z_packed   device, out, marlin_packed_scale_bytes(K, N, G) bytes (fp16 values in the order of the packed scales)
+ * Layers with zero points need N % 256 == 0 (they run on the tcgen05 kernel at every batch size). */
+MARLIN_API int marlin_pack_zeros(const uint8_t* zeros, void* z_packed, int K, int N, int group_size, marlin_stream stream);
+MARLIN_API int marlin_unpack_zeros(const void* z_packed, uint8_t* zeros, int K, int N, int group_size, marlin_stream stream);
+
 /* ---- the layer (Section 3.4, all paragraphs: weight streaming, dequantisation, tensor-core
  *      product, striped partition with global reduction) ----------------------------------------- */
 
@@ -134,6 +143,16 @@ MARLIN_API int marlin_unpack(const void* w_packed, const void* s_packed, uint32_
 MARLIN_API int marlin_gemm(const void* A, const void* w_packed, const void* s_packed, void* C,
                 int M, int K, int N, int group_size,
                 void* workspace, size_t workspace_bytes, marlin_stream stream);
+
+
+/* The layer with zero points: C = A . W, W[k][n] = (q[k][n] - z[k/G][n]) * s[k/G][n].  Arguments as marlin_gemm, plus
+ * z_packed from marlin_pack_zeros.  N % 256 == 0 (else MARLIN_ERR_SHAPE); every batch size runs on the tcgen05
+ * kernel, where the zero point replaces the constant 8 inside the conversion (the subtrahend of the exponent
+ * trick of Section 3.4 "Dequantization and Tensor Cores" becomes 1024 + z): no extra instruction per weight.
+ * workspace: marlin_workspace_bytes(M, K, N). */
+MARLIN_API int marlin_gemm_zp(const void* A, const void* w_packed, const void* s_packed, const void* z_packed, void* C,
+                   int M, int K, int N, int group_size, void* workspace, size_t workspace_bytes,
+                   marlin_stream stream);
 
 /* The same layer for callers that cannot allocate device memory or carry a workspace pointer
  * around: for example a plug-in that runs inside another framework's pre-captured execution plan,

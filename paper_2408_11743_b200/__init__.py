@@ -9,15 +9,18 @@ from .binding import (  # noqa: F401
     gemm,
     gemm_sparse24,
     gemm_static_ws,
+    gemm_zp,
     lib,
     library_path,
     new_workspace,
     pack,
     pack_sparse24,
+    pack_zeros,
     plan_stripes,
     quantize_rtn,
     read_status,
     unpack,
     unpack_sparse24,
+    unpack_zeros,
     workspace_bytes,
 )

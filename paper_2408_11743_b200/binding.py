@@ -17,7 +17,7 @@ EXPORTS = [
     "marlin_status_string", "marlin_packed_weight_bytes", "marlin_packed_scale_bytes", "marlin_packed_meta_bytes",
     "marlin_workspace_bytes", "marlin_pack", "marlin_unpack", "marlin_gemm", "marlin_pack_sparse24",
     "marlin_unpack_sparse24", "marlin_gemm_sparse24", "marlin_read_status", "marlin_plan_stripes",
-    "marlin_gemm_static_ws", "marlin_quantize_rtn",
+    "marlin_gemm_static_ws", "marlin_quantize_rtn", "marlin_pack_zeros", "marlin_unpack_zeros", "marlin_gemm_zp",
 ]
 STATIC_WS_MAX_M = 16  # MARLIN_STATIC_WS_MAX_M of the header
 
@@ -58,6 +58,9 @@ def lib():
     L.marlin_pack.argtypes = [vp, vp, vp, vp, i, i, i, vp]
     L.marlin_unpack.argtypes = [vp, vp, vp, vp, i, i, i, vp]
     L.marlin_quantize_rtn.argtypes = [vp, vp, vp, i, i, i, i, i, vp]
+    L.marlin_pack_zeros.argtypes = [vp, vp, i, i, i, vp]
+    L.marlin_unpack_zeros.argtypes = [vp, vp, i, i, i, vp]
+    L.marlin_gemm_zp.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
     L.marlin_gemm.argtypes = [vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
     L.marlin_gemm_static_ws.argtypes = [vp, vp, vp, vp, i, i, i, i, vp]
     L.marlin_pack_sparse24.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, vp]
@@ -65,7 +68,7 @@ def lib():
     L.marlin_gemm_sparse24.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
     L.marlin_read_status.argtypes = [vp, vp]
     L.marlin_plan_stripes.argtypes = [i, i, i, i, vp, vp, vp, i]
-    for name in ("marlin_quantize_rtn", "marlin_gemm_static_ws", "marlin_pack", "marlin_unpack", "marlin_gemm", "marlin_pack_sparse24", "marlin_unpack_sparse24",
+    for name in ("marlin_pack_zeros", "marlin_unpack_zeros", "marlin_gemm_zp", "marlin_quantize_rtn", "marlin_gemm_static_ws", "marlin_pack", "marlin_unpack", "marlin_gemm", "marlin_pack_sparse24", "marlin_unpack_sparse24",
                  "marlin_gemm_sparse24", "marlin_read_status", "marlin_plan_stripes"):
         getattr(L, name).restype = i
     _lib = L
@@ -192,6 +195,58 @@ def gemm(A, w_packed, s_packed, K: int, N: int, group_size: int, workspace, out=
             raise ValueError("out must be [M, N]")
     _check(L.marlin_gemm(A.data_ptr(), w.data_ptr(), s.data_ptr(), out.data_ptr(), M, K, N, group_size,
                          ws.data_ptr(), ws.numel(), _stream_ptr(stream)), "marlin_gemm")
+    return out
+
+
+def pack_zeros(zeros, K: int, N: int, group_size: int, stream=None):
+    """marlin_pack_zeros: zero points uint8 [K/G, N] (0..15) -> z_packed for gemm_zp."""
+    torch = _torch()
+    z = _dev(zeros, torch.uint8, "zeros")
+    L = lib()
+    sb = L.marlin_packed_scale_bytes(K, N, group_size)
+    if sb == 0 or z.numel() * 2 != sb:
+        raise ValueError("zeros must be [K/G, N] for a supported K, N, group_size")
+    z_packed = torch.empty(sb, dtype=torch.uint8, device=z.device)
+    _check(L.marlin_pack_zeros(z.data_ptr(), z_packed.data_ptr(), K, N, group_size, _stream_ptr(stream)), "marlin_pack_zeros")
+    return z_packed
+
+
+def unpack_zeros(z_packed, K: int, N: int, group_size: int, stream=None):
+    """marlin_unpack_zeros: the inverse of pack_zeros; returns uint8 [K/G, N]."""
+    torch = _torch()
+    zq = _dev(z_packed, torch.uint8, "z_packed")
+    L = lib()
+    sb = L.marlin_packed_scale_bytes(K, N, group_size)
+    if sb == 0 or zq.numel() != sb:
+        raise ValueError("z_packed does not match K, N, group_size")
+    z = torch.empty((sb // (2 * N), N), dtype=torch.uint8, device=zq.device)
+    _check(L.marlin_unpack_zeros(zq.data_ptr(), z.data_ptr(), K, N, group_size, _stream_ptr(stream)), "marlin_unpack_zeros")
+    return z
+
+
+def gemm_zp(A, w_packed, s_packed, z_packed, K: int, N: int, group_size: int, workspace, out=None, stream=None):
+    """marlin_gemm_zp: C = A . ((q - z) * s) with per-group zero points; N % 256 == 0."""
+    torch = _torch()
+    A = _dev(A, torch.float16, "A")
+    if A.dim() != 2 or A.shape[1] != K:
+        raise ValueError("A must be [M, K]")
+    M = A.shape[0]
+    w = _dev(w_packed, torch.uint8, "w_packed")
+    s = _dev(s_packed, torch.uint8, "s_packed")
+    z = _dev(z_packed, torch.uint8, "z_packed")
+    ws = _dev(workspace, torch.uint8, "workspace")
+    L = lib()
+    sb = L.marlin_packed_scale_bytes(K, N, group_size)
+    if w.numel() != L.marlin_packed_weight_bytes(K, N, 0) or s.numel() != sb or z.numel() != sb:
+        raise ValueError("packed buffer sizes do not match K, N, group_size")
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float16, device=A.device)
+    else:
+        _dev(out, torch.float16, "out")
+        if tuple(out.shape) != (M, N):
+            raise ValueError("out must be [M, N]")
+    _check(L.marlin_gemm_zp(A.data_ptr(), w.data_ptr(), s.data_ptr(), z.data_ptr(), out.data_ptr(), M, K, N, group_size,
+                            ws.data_ptr(), ws.numel(), _stream_ptr(stream)), "marlin_gemm_zp")
     return out
 
 

@@ -168,6 +168,28 @@ int marlin_quantize_rtn(const void* W, uint32_t* q_kpacked, void* scales, int K,
   return err == cudaSuccess ? MARLIN_OK : MARLIN_ERR_CUDA;
 }
 
+int marlin_pack_zeros(const uint8_t* zeros, void* z_packed, int K, int N, int group_size, marlin_stream stream) {
+  if (!zeros || !z_packed) return MARLIN_ERR_NULL;
+  if (!shape_ok(K, N) || N % 256) return MARLIN_ERR_SHAPE;
+  int G = normalise_group(K, N, group_size);
+  if (!G) return MARLIN_ERR_GROUP;
+  if (!aligned16(zeros) || !aligned16(z_packed)) return MARLIN_ERR_ALIGN;
+  cudaError_t err = launch_permute_zeros(const_cast<uint8_t*>(zeros), static_cast<uint16_t*>(z_packed), K, N, G, false,
+                                         static_cast<cudaStream_t>(stream));
+  return err == cudaSuccess ? MARLIN_OK : MARLIN_ERR_CUDA;
+}
+
+int marlin_unpack_zeros(const void* z_packed, uint8_t* zeros, int K, int N, int group_size, marlin_stream stream) {
+  if (!zeros || !z_packed) return MARLIN_ERR_NULL;
+  if (!shape_ok(K, N) || N % 256) return MARLIN_ERR_SHAPE;
+  int G = normalise_group(K, N, group_size);
+  if (!G) return MARLIN_ERR_GROUP;
+  if (!aligned16(zeros) || !aligned16(z_packed)) return MARLIN_ERR_ALIGN;
+  cudaError_t err = launch_permute_zeros(zeros, static_cast<uint16_t*>(const_cast<void*>(z_packed)), K, N, G, true,
+                                         static_cast<cudaStream_t>(stream));
+  return err == cudaSuccess ? MARLIN_OK : MARLIN_ERR_CUDA;
+}
+
 int marlin_unpack(const void* w_packed, const void* s_packed, uint32_t* q_kpacked, void* scales, int K, int N,
                   int group_size, marlin_stream stream) {
   if (!q_kpacked || !scales || !w_packed || !s_packed) return MARLIN_ERR_NULL;
@@ -186,15 +208,18 @@ int marlin_unpack(const void* w_packed, const void* s_packed, uint32_t* q_kpacke
 // Shared body of marlin_gemm and marlin_gemm_sparse24 (meta_packed == nullptr: dense).
 static int gemm_common(const void* A, const void* w_packed, const void* meta_packed, const void* s_packed, void* C, int M,
                        int K, int N, int group_size, void* workspace, size_t workspace_bytes, marlin_stream stream,
-                       bool sparse24) {
+                       bool sparse24, const void* z_packed = nullptr) {
   if (!A || !w_packed || !s_packed || !C || !workspace || (sparse24 && !meta_packed)) return MARLIN_ERR_NULL;
+  // layers with zero points run on the tcgen05 kernel alone (N a multiple of 256), at every batch size
+  const bool zero_points = z_packed != nullptr;
+  if (zero_points && (N % 256 || !aligned16(z_packed))) return N % 256 ? MARLIN_ERR_SHAPE : MARLIN_ERR_ALIGN;
   if (M < 1 || !shape_ok(K, N)) return MARLIN_ERR_SHAPE;
   int G = normalise_group(K, N, group_size);
   if (!G) return MARLIN_ERR_GROUP;
   if (!aligned16(A) || !aligned16(w_packed) || !aligned16(s_packed) || !aligned16(C) || !aligned16(workspace) ||
       (sparse24 && !aligned16(meta_packed)))
     return MARLIN_ERR_ALIGN;
-  if (workspace_bytes < workspace_bytes_for(M, K, N, sparse24 || G < kTileK)) return MARLIN_ERR_WORKSPACE;
+  if (workspace_bytes < workspace_bytes_for(M, K, N, sparse24 || G < kTileK || zero_points)) return MARLIN_ERR_WORKSPACE;
   DeviceInfo info;
   int st = device_info(&info);
   if (st != MARLIN_OK) return st;
@@ -213,7 +238,7 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
     // it takes every batch size there
     const bool tc_ok = tc_path_supported(1, K, N);
     // groups of 64 or 32 rows likewise (accepted only where N is a multiple of 256)
-    const bool small_groups = G < kTileK;
+    const bool small_groups = G < kTileK || zero_points;
     const bool use_tcd = !sparse24 && !small_groups && tcd_path_supported(1, K, N) &&
                          (tmode == 1 || (tmode == 2 && rem >= tc_min_m() && !tc_ok));
     const bool use_tc = !use_tcd && tc_ok && (sparse24 || small_groups || rem >= tc_min_m());
@@ -225,6 +250,7 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
     p.wq = static_cast<const uint8_t*>(w_packed);
     p.sq = static_cast<const uint8_t*>(s_packed);
     p.meta = static_cast<const uint8_t*>(meta_packed);
+    p.zq = static_cast<const uint8_t*>(z_packed);
     p.C = static_cast<uint16_t*>(C) + (size_t)m0 * N;
     p.M = m_slab;
     p.K = K;
@@ -235,7 +261,7 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
     p.group_shift = -1;
     for (int sh = 0; sh < 31; ++sh)
       if ((1 << sh) == p.kb_per_group) p.group_shift = sh;
-    p.grouped = (G != K) ? 1 : 0;
+    p.grouped = (G != K || zero_points) ? 1 : 0;  // zero points travel with the scale rows of the in-loop path
     p.status = reinterpret_cast<int*>(ws + kWsStatusOff);
     p.counters = reinterpret_cast<int*>(ws + kWsCounterOff);
     p.partials = reinterpret_cast<float*>(ws + kWsPartialOff);
@@ -270,6 +296,13 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
 int marlin_gemm(const void* A, const void* w_packed, const void* s_packed, void* C, int M, int K, int N,
                 int group_size, void* workspace, size_t workspace_bytes, marlin_stream stream) {
   return gemm_common(A, w_packed, nullptr, s_packed, C, M, K, N, group_size, workspace, workspace_bytes, stream, false);
+}
+
+int marlin_gemm_zp(const void* A, const void* w_packed, const void* s_packed, const void* z_packed, void* C, int M, int K,
+                   int N, int group_size, void* workspace, size_t workspace_bytes, marlin_stream stream) {
+  if (!z_packed) return MARLIN_ERR_NULL;
+  return gemm_common(A, w_packed, nullptr, s_packed, C, M, K, N, group_size, workspace, workspace_bytes, stream, false,
+                     z_packed);
 }
 
 // ---- the variant with a built-in workspace ------------------------------------------------------

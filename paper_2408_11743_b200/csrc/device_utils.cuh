@@ -164,6 +164,11 @@ __device__ __forceinline__ uint32_t hsub2_u32(uint32_t a, uint32_t b) {
   asm("sub.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
   return r;
 }
+__device__ __forceinline__ uint32_t hadd2_u32(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("add.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
 __device__ __forceinline__ uint32_t hfma2_u32(uint32_t a, uint32_t b, uint32_t c) {
   uint32_t r;
   asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
@@ -184,6 +189,18 @@ __device__ __forceinline__ void dequant8(uint32_t w, uint32_t (&a)[4]) {
   a[1] = hfma2_u32(lop3<0xea>(w, HI, EX), MUL, ADD);
   a[2] = hsub2_u32(lop3<0xea>(w2, LO, EX), SUB);
   a[3] = hfma2_u32(lop3<0xea>(w2, HI, EX), MUL, ADD);
+}
+
+// The same with a per-group zero point z in place of 8 (W = (q - z) * s): the subtrahends become registers,
+// sub_lo = {1024 + z, 1024 + z} and add_hi = {-(64 + z), -(64 + z)}; the instruction count is unchanged.
+__device__ __forceinline__ void dequant8_zp(uint32_t w, uint32_t (&a)[4], uint32_t sub_lo, uint32_t add_hi) {
+  constexpr uint32_t LO = 0x000f000fu, HI = 0x00f000f0u, EX = 0x64006400u;
+  constexpr uint32_t MUL = 0x2c002c00u;  // {1/16, 1/16}
+  uint32_t w2 = w >> 8;
+  a[0] = hsub2_u32(lop3<0xea>(w, LO, EX), sub_lo);
+  a[1] = hfma2_u32(lop3<0xea>(w, HI, EX), MUL, add_hi);
+  a[2] = hsub2_u32(lop3<0xea>(w2, LO, EX), sub_lo);
+  a[3] = hfma2_u32(lop3<0xea>(w2, HI, EX), MUL, add_hi);
 }
 
 // The same eight codes WITHOUT the subtraction: a[0], a[2] = 1024 + q (lower nibbles under 0x6400), a[1],

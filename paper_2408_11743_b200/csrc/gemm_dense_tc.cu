@@ -70,7 +70,8 @@ struct TcGeometry {
   static constexpr int META_BYTES = SP ? kChunkBytes : 0;
   static constexpr int STAGE_BYTES = A_BYTES + W_BYTES + META_BYTES;
   static constexpr int SC_ROW_BYTES = kTileN * 2;                   // one row of the tile's group scales
-  static constexpr int SC_BYTES = 4 * SC_ROW_BYTES;                 // scales of one stage: up to four rows (groups of 32)
+  static constexpr int SC_ZP_OFF = 4 * SC_ROW_BYTES;                // the zero points of those groups, if the layer has any
+  static constexpr int SC_BYTES = 8 * SC_ROW_BYTES;                 // scales of one stage: up to four rows (groups of 32), then zero points
   static constexpr int FIXED_BYTES = 1024 + kTcMaxStages * SC_BYTES; // barriers + scale ring
   static constexpr int ALIGN_SLACK = 1024;
   static constexpr int STAGES =
@@ -182,12 +183,14 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       // groups of 128 rows and more: one scale row per k-block; groups of 64 or 32 rows: two or four, which the
       // packed layout keeps together per (k-block, column tile)
       const uint32_t sc_copy = (uint32_t)p.sub_groups * G::SC_ROW_BYTES;
-      const uint32_t tx_bytes = G::W_BYTES + G::META_BYTES + (p.grouped ? sc_copy : 0);
-      auto scale_src = [&](uint32_t col, uint32_t kb) -> const uint8_t* {
-        if (p.sub_groups > 1) return p.sq + ((size_t)kb * (p.N / kTileN) + col) * sc_copy;
+      const bool zp = p.zq != nullptr;  // zero points: rows of the same shape and order as the scales, copied beside them
+      const uint32_t tx_bytes = G::W_BYTES + G::META_BYTES + (p.grouped ? sc_copy : 0) + (zp ? sc_copy : 0);
+      auto scale_off = [&](uint32_t col, uint32_t kb) -> size_t {
+        if (p.sub_groups > 1) return ((size_t)kb * (p.N / kTileN) + col) * sc_copy;
         const uint32_t gi = p.group_shift >= 0 ? (kb >> p.group_shift) : (kb / (uint32_t)p.kb_per_group);
-        return p.sq + ((size_t)gi * p.N + (size_t)col * kTileN) * 2;
+        return ((size_t)gi * p.N + (size_t)col * kTileN) * 2;
       };
+      auto scale_src = [&](uint32_t col, uint32_t kb) -> const uint8_t* { return p.sq + scale_off(col, kb); };
       // weights of (kb, col): the four chunks of a 256-column tile are adjacent, k-blocks follow one another
       auto weight_src = [&](uint32_t col, uint32_t kb) -> const uint8_t* {
         return p.wq + ((size_t)col * KB + kb) * (size_t)G::W_BYTES;
@@ -215,6 +218,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
             bulk_g2s(stage0 + (size_t)s * G::STAGE_BYTES + G::A_BYTES + G::W_BYTES, meta_src(col, kb), G::META_BYTES,
                      &full[s], pol_w);
           if (p.grouped) bulk_g2s(sc_ring + (size_t)s * G::SC_BYTES, scale_src(col, kb), sc_copy, &full[s], pol_w);
+          if (zp) bulk_g2s(sc_ring + (size_t)s * G::SC_BYTES + G::SC_ZP_OFF, p.zq + scale_off(col, kb), sc_copy, &full[s], pol_w);
         }
       }
       __syncwarp();
@@ -244,6 +248,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
           bulk_g2s(st + G::A_BYTES, weight_src(col, kb), G::W_BYTES, &full[s], pol_w);
           if constexpr (SP) bulk_g2s(st + G::A_BYTES + G::W_BYTES, meta_src(col, kb), G::META_BYTES, &full[s], pol_w);
           if (p.grouped) bulk_g2s(sc_ring + (size_t)s * G::SC_BYTES, scale_src(col, kb), sc_copy, &full[s], pol_w);
+          if (zp) bulk_g2s(sc_ring + (size_t)s * G::SC_BYTES + G::SC_ZP_OFF, p.zq + scale_off(col, kb), sc_copy, &full[s], pol_w);
           mbar_expect_tx(&xfull[s], G::A_BYTES);
         }
         __syncwarp();
@@ -356,6 +361,10 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
     const uint16_t* sptr = reinterpret_cast<const uint16_t*>(p.sq) + (size_t)col * kTileN + spos;
 
     uint32_t sv4[4] = {0, 0, 0, 0};  // {scale, scale} of this thread's column for the four 32-row quarters of the k-block
+    // the subtrahends of the conversion per quarter: {1024 + z, 1024 + z} and {-(64 + z), -(64 + z)}, z = 8 without zero points
+    uint32_t zlo4[4] = {0x64086408u, 0x64086408u, 0x64086408u, 0x64086408u};
+    uint32_t zhi4[4] = {0xd480d480u, 0xd480d480u, 0xd480d480u, 0xd480d480u};
+    const bool zp = p.zq != nullptr;
     float sc_col = 1.f;  // the column's single scale
     if constexpr (!GR) sc_col = __half2float(__ushort_as_half(__ldg(sptr)));
     for (uint32_t x = 0; x < len; ++x, ++it) {
@@ -370,6 +379,15 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
           // quarter qd lies in scale row qd * sub_groups / 4 of the stage (row 0 for groups of 128 rows and more)
           const uint32_t sv = lds16(sbase + (uint32_t)((qd * p.sub_groups) >> 2) * G::SC_ROW_BYTES);
           sv4[qd] = sv | (sv << 16);
+        }
+        if (zp) {
+#pragma unroll
+          for (int qd = 0; qd < 4; ++qd) {
+            const uint32_t zv = lds16(sbase + G::SC_ZP_OFF + (uint32_t)((qd * p.sub_groups) >> 2) * G::SC_ROW_BYTES);
+            const uint32_t z2 = zv | (zv << 16);
+            zlo4[qd] = hadd2_u32(z2, 0x64006400u);   // 1024 + z
+            zhi4[qd] = hsub2_u32(0xd400d400u, z2);   // -64 - z
+          }
         }
       }
       const uint32_t wbase = smem_u32(stage0) + (uint32_t)s * G::STAGE_BYTES + G::A_BYTES + (SP ? (uint32_t)n256 * 16u : vec_off);
@@ -403,8 +421,8 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
           for (int c = 0; c < 4; ++c) {
             const uint32_t w0 = hh == 0 ? v[c].x : v[c].z, w1 = hh == 0 ? v[c].y : v[c].w;
             uint32_t lo[4], hi[4];
-            dequant8(w0, lo);  // rows 64hh + 16c + 0..7
-            dequant8(w1, hi);  // rows 64hh + 16c + 8..15
+            dequant8_zp(w0, lo, zlo4[2 * hh + (c >> 1)], zhi4[2 * hh + (c >> 1)]);  // rows 64hh + 16c + 0..7
+            dequant8_zp(w1, hi, zlo4[2 * hh + (c >> 1)], zhi4[2 * hh + (c >> 1)]);  // rows 64hh + 16c + 8..15
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
               // rows 64hh + 16c ..: quarter 2hh + c / 2 of the k-block

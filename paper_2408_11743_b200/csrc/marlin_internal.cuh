@@ -59,6 +59,7 @@ struct GemmParams {
   const uint8_t* wq;
   const uint8_t* sq;
   const uint8_t* meta;   // 2:4 variant only
+  const uint8_t* zq;     // packed zero points (fp16 values 0..15 in the order of the packed scales), or nullptr: z = 8
   uint16_t* C;
   int M, K, N;
   uint32_t kb;       // K / 128
@@ -108,6 +109,8 @@ cudaError_t launch_pack_dense(uint32_t* q, uint16_t* s, uint32_t* wq, uint16_t* 
 // round-to-nearest quantiser with clipping search (quantize.cu): W fp16 [K][N] -> canonical codes and scales
 cudaError_t launch_quantize_rtn(const uint16_t* W, uint32_t* q_kpacked, uint16_t* scales, int K, int N, int G, int n_grid,
                                 int n_candidates, cudaStream_t stream);
+// canonical zero points uint8 [K/G][N] (0..15) <-> fp16 values in the packed order of the scales
+cudaError_t launch_permute_zeros(uint8_t* z, uint16_t* zq, int K, int N, int G, bool inverse, cudaStream_t stream);
 // canonical scales [K/G][N] <-> packed order (shared by the dense and the 2:4 pack)
 cudaError_t launch_permute_scales(uint16_t* s, uint16_t* sq, int K, int N, int G, bool inverse, cudaStream_t stream);
 

@@ -131,7 +131,43 @@ __global__ void permute_scales_kernel(const uint16_t* __restrict__ in, uint16_t*
   }
 }
 
+// zero points: the same permutation, uint8 codes on the canonical side and fp16 values on the packed side
+__global__ void permute_zeros_kernel(uint8_t* __restrict__ z, uint16_t* __restrict__ zq, long long total, int N, int sub,
+                                     bool inverse) {
+  for (long long x = blockIdx.x * (long long)blockDim.x + threadIdx.x; x < total;
+       x += (long long)gridDim.x * blockDim.x) {
+    const int pos = (int)(x & 63);
+    const int g = pos >> 3, j = (pos >> 1) & 3, b = pos & 1;
+    const int c64 = 16 * j + 8 * b + g;
+    long long canon;
+    if (sub == 1) {
+      canon = (x & ~63LL) + c64;
+    } else {
+      const long long rec = x >> 8;
+      const int r = (int)(rec % sub);
+      const long long kt = rec / sub;
+      const int NT = N / 256;
+      const long long kb = kt / NT, tile = kt % NT;
+      canon = (kb * sub + r) * (long long)N + tile * 256 + (x & 192) + c64;
+    }
+    if (inverse)
+      z[canon] = (uint8_t)__half2float(__ushort_as_half(zq[x]));
+    else
+      zq[x] = __half_as_ushort(__float2half_rn((float)z[canon]));
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_permute_zeros(uint8_t* z, uint16_t* zq, int K, int N, int G, bool inverse, cudaStream_t stream) {
+  const long long ns = (long long)(K / G) * N;
+  const int sub = G >= kTileK ? 1 : kTileK / G;
+  const int threads = 256;
+  int blocks = (int)((ns + threads - 1) / threads);
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  permute_zeros_kernel<<<blocks, threads, 0, stream>>>(z, zq, ns, N, sub, inverse);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_pack_dense(uint32_t* q, uint16_t* s, uint32_t* wq, uint16_t* sq, int K, int N, int G, bool inverse,
                               cudaStream_t stream) {
