@@ -256,6 +256,62 @@ class LayerBench:
         return r
 
 
+def mlp_chain(marlin, dev, stream, l2, capture, time_graph, rng, K=4096, I=11008, N=4096, Ms=(1, 16, 64)):
+    import torch
+    G = GROUP
+
+    def rand_layer(k, n):
+        q = torch.from_numpy(rng.integers(-2**31, 2**31 - 1, size=(k // 8, n), dtype=np.int64).astype(np.int32)).to(dev)
+        S = torch.from_numpy(rng.uniform(0.005, 0.02, size=(k // G, n)).astype(np.float16)).to(dev)
+        return q, S
+    qg, sg = rand_layer(K, I)
+    qu, su = rand_layer(K, I)
+    q_gu, s_gu = marlin.interleave_gate_up(qg, sg, qu, su, G)
+    gu0 = marlin.pack(q_gu, s_gu, G)
+    d0 = marlin.pack(*rand_layer(I, N), G)
+    wb = roofline.weight_bytes(K, 2 * I, G) + roofline.weight_bytes(I, N, G)
+    copies = max(2, int(np.ceil(2.0 * l2 / wb)) + 1)
+    gus = [tuple(t.clone() for t in gu0) for _ in range(copies)]
+    ds = [tuple(t.clone() for t in d0) for _ in range(copies)]
+    res = []
+    for M in Ms:
+        A = torch.from_numpy(rng.standard_normal((M, K), dtype=np.float32).astype(np.float16)).to(dev)
+        H = torch.empty((M, I), dtype=torch.float16, device=dev)
+        H2 = torch.empty((M, 2 * I), dtype=torch.float16, device=dev)
+        C = torch.empty((M, N), dtype=torch.float16, device=dev)
+        ws = torch.zeros(max(marlin.workspace_bytes(M, K, 2 * I), marlin.workspace_bytes(M, I, N)), dtype=torch.uint8, device=dev)
+        rot = [0]
+
+        def fused():
+            i = rot[0] % copies
+            rot[0] += 1
+            marlin.mlp_swiglu(A, gus[i][0], gus[i][1], ds[i][0], ds[i][1], K, I, N, G, ws, H=H, out=C, stream=stream)
+
+        def unfused():
+            i = rot[0] % copies
+            rot[0] += 1
+            marlin.gemm(A, gus[i][0], gus[i][1], K, 2 * I, G, ws, out=H2, stream=stream)
+            v = H2.view(M, I // 8, 2, 8)
+            torch.mul(torch.nn.functional.silu(v[:, :, 0, :]), v[:, :, 1, :], out=H.view(M, I // 8, 8))
+            marlin.gemm(H, ds[i][0], ds[i][1], I, N, G, ws, out=C, stream=stream)
+        t = {}
+        for name, fn in (("fused", fused), ("unfused", unfused)):
+            with torch.cuda.stream(stream):
+                for _ in range(3):
+                    fn()
+            torch.cuda.synchronize(dev)
+            reps = 2 * copies
+            g = capture(fn, reps)
+            time_graph(g)
+            t[name] = min(time_graph(g) for _ in range(5)) / reps
+        if marlin.read_status(ws, stream=stream) != 0:
+            raise RuntimeError("device-side wait expired")
+        res.append({"layer": "llama2-7b MLP chain (gate_up + SwiGLU + down)", "config": 3, "M": M, "K": K, "I": I, "N": N,
+                    "G": G, "fused_us": round(t["fused"] * 1e6, 2), "unfused_us": round(t["unfused"] * 1e6, 2),
+                    "weight_gbs": round(wb / t["fused"] / 1e9, 1)})
+    return res
+
+
 def extra_layers(marlin, dev, stream, l2, peaks, capture, time_graph):
     """Per-layer numbers outside the timed step: every layer and batch size of configs 3 (Llama-2-7B shapes), 4
     (Llama-2-70B shapes, group 128 and one scale per column) and 5 (the 2:4 layer, with the dense layer beside it),
@@ -293,6 +349,10 @@ def extra_layers(marlin, dev, stream, l2, peaks, capture, time_graph):
                     "us": round(tq * 1e6, 1), "gweights_per_s": round(8192 * 8192 / tq / 1e9, 1),
                     "algorithmic_gbs": round((8192 * 8192 * 2.5 + 2 * 64 * 8192) / tq / 1e9, 1)})
         del Wq
+    # the gated MLP of a Llama-2-7B layer as a chain: gate_up with the activation fused into its epilogue, then down
+    # (two launches, the second under programmatic dependent launch), against the same layers with the activation
+    # as separate elementwise kernels on the wide intermediate
+    out.extend(mlp_chain(marlin, dev, stream, l2, capture, time_graph, rng))
     for name, K, N in inputs.LLAMA70B_LAYERS:
         for G in (GROUP, K):
             sweep(K, N, G, False, (1, 16, 64, 128),

@@ -145,6 +145,31 @@ MARLIN_API int marlin_gemm(const void* A, const void* w_packed, const void* s_pa
                 void* workspace, size_t workspace_bytes, marlin_stream stream);
 
 
+/* ---- the gated MLP of a decoder layer as a chain of two launches (Section 5.1 names the per-kernel overheads on
+ *      real layer shapes; fusing the activation removes one launch and the round trip of the wide intermediate) -- */
+
+/* Gate and up projections of one MLP side by side, in the column order the fused epilogue expects: output column
+ * n = 16 b + r holds gate channel 8 b + r for r < 8 and up channel 8 b + r - 8 otherwise.
+ *   q_gate, q_up   device, uint32 [K/8][I] canonical codes;   s_gate, s_up   device, fp16 [K/G][I]
+ *   q_out          device, out, uint32 [K/8][2 I];            s_out          device, out, fp16 [K/G][2 I]
+ * Feed q_out, s_out to marlin_pack with N = 2 I.  I % 32 == 0. */
+MARLIN_API int marlin_interleave_gate_up(const uint32_t* q_gate, const void* s_gate, const uint32_t* q_up, const void* s_up,
+                              uint32_t* q_out, void* s_out, int K, int I, int group_size, marlin_stream stream);
+
+/* marlin_gemm on such a layer (N = 2 I columns) with the activation fused into the epilogue:
+ *   H[m][c] = fp16( silu(g) * u ),  g = fp16(A . W)[m][gate channel c],  u = fp16(A . W)[m][up channel c],
+ * silu(g) = g / (1 + exp(-g)) in fp32.  H is device, out, fp16 [M][N/2] row-major.  Everything else as marlin_gemm
+ * (the product is rounded to fp16 before the activation, as it would be if H were computed from a stored C). */
+MARLIN_API int marlin_gemm_swiglu(const void* A, const void* w_packed, const void* s_packed, void* H, int M, int K, int N,
+                       int group_size, void* workspace, size_t workspace_bytes, marlin_stream stream);
+
+/* C = (silu(A . W_gate) * (A . W_up)) . W_down: marlin_gemm_swiglu into H (device scratch, fp16 [M][I]), then
+ * marlin_gemm of H with the down projection (I x N).  One workspace serves both launches (they run one after the
+ * other on `stream`): at least max(marlin_workspace_bytes(M, K, 2 I), marlin_workspace_bytes(M, I, N)) bytes. */
+MARLIN_API int marlin_mlp_swiglu(const void* A, const void* w_gate_up, const void* s_gate_up, const void* w_down,
+                      const void* s_down, void* H, void* C, int M, int K, int I, int N, int group_size,
+                      void* workspace, size_t workspace_bytes, marlin_stream stream);
+
 /* The layer with zero points: C = A . W, W[k][n] = (q[k][n] - z[k/G][n]) * s[k/G][n].  Arguments as marlin_gemm, plus
  * z_packed from marlin_pack_zeros.  N % 256 == 0 (else MARLIN_ERR_SHAPE); every batch size runs on the tcgen05
  * kernel, where the zero point replaces the constant 8 inside the conversion (the subtrahend of the exponent

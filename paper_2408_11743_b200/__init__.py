@@ -9,8 +9,11 @@ from .binding import (  # noqa: F401
     gemm,
     gemm_sparse24,
     gemm_static_ws,
+    gemm_swiglu,
+    interleave_gate_up,
     gemm_zp,
     lib,
+    mlp_swiglu,
     library_path,
     new_workspace,
     pack,

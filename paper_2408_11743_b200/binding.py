@@ -18,6 +18,7 @@ EXPORTS = [
     "marlin_workspace_bytes", "marlin_pack", "marlin_unpack", "marlin_gemm", "marlin_pack_sparse24",
     "marlin_unpack_sparse24", "marlin_gemm_sparse24", "marlin_read_status", "marlin_plan_stripes",
     "marlin_gemm_static_ws", "marlin_quantize_rtn", "marlin_pack_zeros", "marlin_unpack_zeros", "marlin_gemm_zp",
+    "marlin_interleave_gate_up", "marlin_gemm_swiglu", "marlin_mlp_swiglu",
 ]
 STATIC_WS_MAX_M = 16  # MARLIN_STATIC_WS_MAX_M of the header
 
@@ -61,6 +62,9 @@ def lib():
     L.marlin_pack_zeros.argtypes = [vp, vp, i, i, i, vp]
     L.marlin_unpack_zeros.argtypes = [vp, vp, i, i, i, vp]
     L.marlin_gemm_zp.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
+    L.marlin_interleave_gate_up.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, vp]
+    L.marlin_gemm_swiglu.argtypes = [vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
+    L.marlin_mlp_swiglu.argtypes = [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp, sz, vp]
     L.marlin_gemm.argtypes = [vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
     L.marlin_gemm_static_ws.argtypes = [vp, vp, vp, vp, i, i, i, i, vp]
     L.marlin_pack_sparse24.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, vp]
@@ -68,7 +72,7 @@ def lib():
     L.marlin_gemm_sparse24.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
     L.marlin_read_status.argtypes = [vp, vp]
     L.marlin_plan_stripes.argtypes = [i, i, i, i, vp, vp, vp, i]
-    for name in ("marlin_pack_zeros", "marlin_unpack_zeros", "marlin_gemm_zp", "marlin_quantize_rtn", "marlin_gemm_static_ws", "marlin_pack", "marlin_unpack", "marlin_gemm", "marlin_pack_sparse24", "marlin_unpack_sparse24",
+    for name in ("marlin_interleave_gate_up", "marlin_gemm_swiglu", "marlin_mlp_swiglu", "marlin_pack_zeros", "marlin_unpack_zeros", "marlin_gemm_zp", "marlin_quantize_rtn", "marlin_gemm_static_ws", "marlin_pack", "marlin_unpack", "marlin_gemm", "marlin_pack_sparse24", "marlin_unpack_sparse24",
                  "marlin_gemm_sparse24", "marlin_read_status", "marlin_plan_stripes"):
         getattr(L, name).restype = i
     _lib = L
@@ -247,6 +251,75 @@ def gemm_zp(A, w_packed, s_packed, z_packed, K: int, N: int, group_size: int, wo
             raise ValueError("out must be [M, N]")
     _check(L.marlin_gemm_zp(A.data_ptr(), w.data_ptr(), s.data_ptr(), z.data_ptr(), out.data_ptr(), M, K, N, group_size,
                             ws.data_ptr(), ws.numel(), _stream_ptr(stream)), "marlin_gemm_zp")
+    return out
+
+
+def interleave_gate_up(q_gate, s_gate, q_up, s_up, group_size: int, stream=None):
+    """marlin_interleave_gate_up: canonical (codes, scales) of the gate and up projections [K, I] each -> those of the
+    fused layer [K, 2 I] in blocks of 16 columns (8 gate, 8 up)."""
+    torch = _torch()
+    qg, qu = _dev(q_gate, torch.int32, "q_gate"), _dev(q_up, torch.int32, "q_up")
+    sg, su = _dev(s_gate, torch.float16, "s_gate"), _dev(s_up, torch.float16, "s_up")
+    if qg.shape != qu.shape or sg.shape != su.shape or qg.shape[1] != sg.shape[1]:
+        raise ValueError("gate and up must have the same shapes")
+    K, I = qg.shape[0] * 8, qg.shape[1]
+    q = torch.empty((K // 8, 2 * I), dtype=torch.int32, device=qg.device)
+    s = torch.empty((sg.shape[0], 2 * I), dtype=torch.float16, device=qg.device)
+    _check(lib().marlin_interleave_gate_up(qg.data_ptr(), sg.data_ptr(), qu.data_ptr(), su.data_ptr(), q.data_ptr(),
+                                           s.data_ptr(), K, I, group_size, _stream_ptr(stream)), "marlin_interleave_gate_up")
+    return q, s
+
+
+def gemm_swiglu(A, w_packed, s_packed, K: int, N: int, group_size: int, workspace, out=None, stream=None):
+    """marlin_gemm_swiglu: H[M, N/2] = silu(gate) * up of the fused gate_up layer (see interleave_gate_up)."""
+    torch = _torch()
+    A = _dev(A, torch.float16, "A")
+    if A.dim() != 2 or A.shape[1] != K:
+        raise ValueError("A must be [M, K]")
+    M = A.shape[0]
+    w = _dev(w_packed, torch.uint8, "w_packed")
+    s = _dev(s_packed, torch.uint8, "s_packed")
+    ws = _dev(workspace, torch.uint8, "workspace")
+    L = lib()
+    if w.numel() != L.marlin_packed_weight_bytes(K, N, 0) or s.numel() != L.marlin_packed_scale_bytes(K, N, group_size):
+        raise ValueError("packed buffer sizes do not match K, N, group_size")
+    if out is None:
+        out = torch.empty((M, N // 2), dtype=torch.float16, device=A.device)
+    else:
+        _dev(out, torch.float16, "out")
+        if tuple(out.shape) != (M, N // 2):
+            raise ValueError("out must be [M, N / 2]")
+    _check(L.marlin_gemm_swiglu(A.data_ptr(), w.data_ptr(), s.data_ptr(), out.data_ptr(), M, K, N, group_size,
+                                ws.data_ptr(), ws.numel(), _stream_ptr(stream)), "marlin_gemm_swiglu")
+    return out
+
+
+def mlp_swiglu(A, w_gate_up, s_gate_up, w_down, s_down, K: int, I: int, N: int, group_size: int, workspace, H=None, out=None,
+               stream=None):
+    """marlin_mlp_swiglu: (silu(A . W_gate) * (A . W_up)) . W_down as two launches; returns C [M, N]."""
+    torch = _torch()
+    A = _dev(A, torch.float16, "A")
+    if A.dim() != 2 or A.shape[1] != K:
+        raise ValueError("A must be [M, K]")
+    M = A.shape[0]
+    ws = _dev(workspace, torch.uint8, "workspace")
+    L = lib()
+    wg, sg = _dev(w_gate_up, torch.uint8, "w_gate_up"), _dev(s_gate_up, torch.uint8, "s_gate_up")
+    wd, sd = _dev(w_down, torch.uint8, "w_down"), _dev(s_down, torch.uint8, "s_down")
+    if (wg.numel() != L.marlin_packed_weight_bytes(K, 2 * I, 0) or sg.numel() != L.marlin_packed_scale_bytes(K, 2 * I, group_size)
+            or wd.numel() != L.marlin_packed_weight_bytes(I, N, 0) or sd.numel() != L.marlin_packed_scale_bytes(I, N, group_size)):
+        raise ValueError("packed buffer sizes do not match K, I, N, group_size")
+    if H is None:
+        H = torch.empty((M, I), dtype=torch.float16, device=A.device)
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float16, device=A.device)
+    _dev(H, torch.float16, "H")
+    _dev(out, torch.float16, "out")
+    if tuple(H.shape) != (M, I) or tuple(out.shape) != (M, N):
+        raise ValueError("H must be [M, I] and out [M, N]")
+    _check(L.marlin_mlp_swiglu(A.data_ptr(), wg.data_ptr(), sg.data_ptr(), wd.data_ptr(), sd.data_ptr(), H.data_ptr(),
+                               out.data_ptr(), M, K, I, N, group_size, ws.data_ptr(), ws.numel(), _stream_ptr(stream)),
+           "marlin_mlp_swiglu")
     return out
 
 

@@ -39,6 +39,35 @@ def needs_build() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
+PTXAS_LOG = os.path.join(_HERE, "ptxas_report.log")
+
+
+def spill_report():
+    """{kernel name: (registers, spill store bytes)} from the last build of the product library, or {} if there is none."""
+    import re
+    try:
+        text = open(PTXAS_LOG).read()
+    except OSError:
+        return {}
+    out = {}
+    name = None
+    spills = 0
+    for line in text.splitlines():
+        m = re.search(r"Function properties for (\S+)", line)
+        if m:
+            name = m.group(1)
+            continue
+        m = re.search(r"(\d+) bytes spill stores", line)
+        if m and name:
+            spills = int(m.group(1))
+            continue
+        m = re.search(r"Used (\d+) registers", line)
+        if m and name:
+            out[name] = (int(m.group(1)), spills)
+            name, spills = None, 0
+    return out
+
+
 def build(force: bool = False, verbose: bool = False, extra_flags=(), out: str = LIB) -> str:
     """Compiles every .cu of the library and links `out`.  `extra_flags` (for example -DMARLIN_TIMING)
     and a different `out` give an instrumented variant beside the product library."""
@@ -50,20 +79,26 @@ def build(force: bool = False, verbose: bool = False, extra_flags=(), out: str =
         obj = os.path.join(CSRC, src.replace(".cu", ".o" if out == LIB else ".variant.o"))
         cmd = [_nvcc(), *NVCC_FLAGS, *extra_flags, "-I", os.path.join(_ROOT, "include"), "-I", CSRC, "-c",
                os.path.join(CSRC, src), "-o", obj]
+        # the register allocator's report is kept beside the library: spill_report() reads it
+        cmd.insert(1, "-Xptxas")
+        cmd.insert(2, "-v")
         if verbose:
-            cmd.insert(1, "-Xptxas")
-            cmd.insert(2, "-v")
             print(" ".join(cmd), flush=True)
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
         objs.append(obj)
     failed = False
+    logs = []
     for src, proc in procs:
         log, _ = proc.communicate()
+        logs.append(log)
         if proc.returncode != 0 or verbose:
             sys.stderr.write(log)
         failed |= proc.returncode != 0
     if failed:
         raise RuntimeError("nvcc failed")
+    if out == LIB:
+        with open(PTXAS_LOG, "w") as f:
+            f.write("".join(logs))
     link = [_nvcc(), "-shared", "-o", out, *objs, "-cudart", "static",
             "-gencode", "arch=compute_100a,code=sm_100a"]
     subprocess.run(link, check=True)

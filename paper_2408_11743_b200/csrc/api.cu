@@ -208,7 +208,7 @@ int marlin_unpack(const void* w_packed, const void* s_packed, uint32_t* q_kpacke
 // Shared body of marlin_gemm and marlin_gemm_sparse24 (meta_packed == nullptr: dense).
 static int gemm_common(const void* A, const void* w_packed, const void* meta_packed, const void* s_packed, void* C, int M,
                        int K, int N, int group_size, void* workspace, size_t workspace_bytes, marlin_stream stream,
-                       bool sparse24, const void* z_packed = nullptr) {
+                       bool sparse24, const void* z_packed = nullptr, bool swiglu = false) {
   if (!A || !w_packed || !s_packed || !C || !workspace || (sparse24 && !meta_packed)) return MARLIN_ERR_NULL;
   // layers with zero points run on the tcgen05 kernel alone (N a multiple of 256), at every batch size
   const bool zero_points = z_packed != nullptr;
@@ -239,7 +239,8 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
     const bool tc_ok = tc_path_supported(1, K, N);
     // groups of 64 or 32 rows likewise (accepted only where N is a multiple of 256)
     const bool small_groups = G < kTileK || zero_points;
-    const bool use_tcd = !sparse24 && !small_groups && tcd_path_supported(1, K, N) &&
+    // (the kernel with deferred scales has no fused activation: those layers go through the warp-level kernel then)
+    const bool use_tcd = !swiglu && !sparse24 && !small_groups && tcd_path_supported(1, K, N) &&
                          (tmode == 1 || (tmode == 2 && rem >= tc_min_m() && !tc_ok));
     const bool use_tc = !use_tcd && tc_ok && (sparse24 || small_groups || rem >= tc_min_m());
     const int m_slab = use_tcd ? (rem < kTcdMaxSlabM ? rem : kTcdMaxSlabM)
@@ -251,7 +252,8 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
     p.sq = static_cast<const uint8_t*>(s_packed);
     p.meta = static_cast<const uint8_t*>(meta_packed);
     p.zq = static_cast<const uint8_t*>(z_packed);
-    p.C = static_cast<uint16_t*>(C) + (size_t)m0 * N;
+    p.C = static_cast<uint16_t*>(C) + (size_t)m0 * (swiglu ? N / 2 : N);
+    p.swiglu = swiglu ? 1 : 0;
     p.M = m_slab;
     p.K = K;
     p.N = N;
@@ -296,6 +298,37 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
 int marlin_gemm(const void* A, const void* w_packed, const void* s_packed, void* C, int M, int K, int N,
                 int group_size, void* workspace, size_t workspace_bytes, marlin_stream stream) {
   return gemm_common(A, w_packed, nullptr, s_packed, C, M, K, N, group_size, workspace, workspace_bytes, stream, false);
+}
+
+int marlin_gemm_swiglu(const void* A, const void* w_packed, const void* s_packed, void* H, int M, int K, int N,
+                       int group_size, void* workspace, size_t workspace_bytes, marlin_stream stream) {
+  return gemm_common(A, w_packed, nullptr, s_packed, H, M, K, N, group_size, workspace, workspace_bytes, stream, false,
+                     nullptr, true);
+}
+
+int marlin_interleave_gate_up(const uint32_t* q_gate, const void* s_gate, const uint32_t* q_up, const void* s_up,
+                              uint32_t* q_out, void* s_out, int K, int I, int group_size, marlin_stream stream) {
+  if (!q_gate || !s_gate || !q_up || !s_up || !q_out || !s_out) return MARLIN_ERR_NULL;
+  if (I < 32 || I % 32 || !shape_ok(K, 2 * I)) return MARLIN_ERR_SHAPE;
+  int G = normalise_group(K, 2 * I, group_size);
+  if (!G) return MARLIN_ERR_GROUP;
+  if (!aligned16(q_gate) || !aligned16(s_gate) || !aligned16(q_up) || !aligned16(s_up) || !aligned16(q_out) ||
+      !aligned16(s_out))
+    return MARLIN_ERR_ALIGN;
+  cudaError_t err = launch_interleave_gate_up(q_gate, static_cast<const uint16_t*>(s_gate), q_up,
+                                              static_cast<const uint16_t*>(s_up), q_out, static_cast<uint16_t*>(s_out), K, I,
+                                              G, static_cast<cudaStream_t>(stream));
+  return err == cudaSuccess ? MARLIN_OK : MARLIN_ERR_CUDA;
+}
+
+int marlin_mlp_swiglu(const void* A, const void* w_gate_up, const void* s_gate_up, const void* w_down, const void* s_down,
+                      void* H, void* C, int M, int K, int I, int N, int group_size, void* workspace, size_t workspace_bytes,
+                      marlin_stream stream) {
+  // two launches: gate_up with the activation fused into its epilogue, then down; the second starts under
+  // programmatic dependent launch and prefetches its weights while the first finishes
+  int st = marlin_gemm_swiglu(A, w_gate_up, s_gate_up, H, M, K, 2 * I, group_size, workspace, workspace_bytes, stream);
+  if (st != MARLIN_OK) return st;
+  return marlin_gemm(H, w_down, s_down, C, M, I, N, group_size, workspace, workspace_bytes, stream);
 }
 
 int marlin_gemm_zp(const void* A, const void* w_packed, const void* s_packed, const void* z_packed, void* C, int M, int K,

@@ -96,6 +96,11 @@ __device__ __forceinline__ uint64_t policy_evict_last() {
   asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
   return pol;
 }
+__device__ __forceinline__ uint64_t policy_evict_normal() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
 // global -> shared bulk copy; dst, src 16-byte aligned, bytes a multiple of 16.
 __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar, uint64_t pol) {
   asm volatile(
@@ -248,6 +253,18 @@ __device__ __forceinline__ void mma_sp_16832(float (&d)[4], const uint32_t (&a)[
 
 // Explicit shared-space loads from a 32-bit shared address (the stage ring is addressed through a pointer
 // that is re-aligned at run time, which can hide the address space from the compiler).
+// silu(gate) * up for eight fp16 pairs: fp16 -> fp32, g / (1 + exp(-g)) * u in fp32, one rounding to fp16
+__device__ __forceinline__ uint32_t swiglu2(uint32_t gate, uint32_t up) {
+  const float2 g = __half22float2(*reinterpret_cast<const __half2*>(&gate));
+  const float2 u = __half22float2(*reinterpret_cast<const __half2*>(&up));
+  const float y0 = __fdividef(g.x, 1.f + __expf(-g.x)) * u.x;
+  const float y1 = __fdividef(g.y, 1.f + __expf(-g.y)) * u.y;
+  const __half2 r = __floats2half2_rn(y0, y1);
+  return *reinterpret_cast<const uint32_t*>(&r);
+}
+__device__ __forceinline__ uint4 swiglu8(uint4 gate, uint4 up) {
+  return make_uint4(swiglu2(gate.x, up.x), swiglu2(gate.y, up.y), swiglu2(gate.z, up.z), swiglu2(gate.w, up.w));
+}
 __device__ __forceinline__ uint4 lds128(uint32_t saddr) {
   uint4 v;
   asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(saddr));

@@ -291,6 +291,29 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
     }
   };
 
+  // The finished fp16 tile goes from its staging buffer to C with 16-byte row stores, by the first `nthr` consumer
+  // threads.  With the fused activation the tile's 16-column blocks hold eight gate and eight up channels: one
+  // 16-byte piece of silu(gate) * up per pair of pieces, into a C of half the width.
+  auto store_tile = [&](uint32_t col, int nthr) {
+    if (!p.swiglu) {
+      constexpr int CH = NW * 8;  // 16-byte pieces per row of the tile
+      for (int x = ctid; x < p.M * CH; x += nthr) {
+        const int m = x / CH, ch = x % CH;
+        const uint4 v = *reinterpret_cast<const uint4*>(cst + m * G::CST_STRIDE + ch * 8);
+        *reinterpret_cast<uint4*>(p.C + (size_t)m * p.N + (size_t)col * G::NT + ch * 8) = v;
+      }
+    } else {
+      constexpr int CH2 = NW * 4;
+      const int ldc = p.N / 2;
+      for (int x = ctid; x < p.M * CH2; x += nthr) {
+        const int m = x / CH2, c2 = x % CH2;
+        const uint4 gate = *reinterpret_cast<const uint4*>(cst + m * G::CST_STRIDE + (2 * c2) * 8);
+        const uint4 up = *reinterpret_cast<const uint4*>(cst + m * G::CST_STRIDE + (2 * c2 + 1) * 8);
+        *reinterpret_cast<uint4*>(p.C + (size_t)m * ldc + (size_t)col * (G::NT / 2) + c2 * 8) = swiglu8(gate, up);
+      }
+    }
+  };
+
   uint32_t u = u0;
   uint32_t it0 = 0;  // iteration index of the segment's first unit, relative to u0
   while (u < u1) {
@@ -517,12 +540,7 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
             cst[(m + 1) * G::CST_STRIDE + n + 8] = __half_as_ushort(__float2half_rn(acc[r][3]));
           }
           named_bar_sync(2, kG0);
-          constexpr int CH = NW * 8;
-          for (int x = ctid; x < p.M * CH; x += kG0) {
-            const int m = x / CH, ch = x % CH;
-            const uint4 v = *reinterpret_cast<const uint4*>(cst + m * G::CST_STRIDE + ch * 8);
-            *reinterpret_cast<uint4*>(p.C + (size_t)m * p.N + (size_t)col * G::NT + ch * 8) = v;
-          }
+          store_tile(col, kG0);
         }
         named_bar_sync(2, kG0);  // cst and last_flag[1] are free again
       }
@@ -656,12 +674,7 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
     }
     if (tile_in_cst) {
       named_bar_sync(1, kConsumerThreads);
-      constexpr int CH = NW * 8;  // 16-byte chunks per row of the tile
-      for (int x = ctid; x < p.M * CH; x += kConsumerThreads) {
-        const int m = x / CH, ch = x % CH;
-        const uint4 v = *reinterpret_cast<const uint4*>(cst + m * G::CST_STRIDE + ch * 8);
-        *reinterpret_cast<uint4*>(p.C + (size_t)m * p.N + (size_t)col * G::NT + ch * 8) = v;
-      }
+      store_tile(col, kConsumerThreads);
       named_bar_sync(1, kConsumerThreads);  // the tile buffer is free again
     }
 

@@ -176,7 +176,8 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       const int pw = warp - kDequantWarps;
       if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
       // one slab: every weight byte is read once; several slabs read the layer once each, from the L2 after the first
-      const uint64_t pol_w = p.slabs > 1 ? policy_evict_last() : policy_evict_first();
+      // (normal priority: marked to stay, the weights of the layers before would crowd the L2)
+      const uint64_t pol_w = p.slabs > 1 ? policy_evict_normal() : policy_evict_first();
       const uint64_t pol_a = policy_evict_last();
       // weights and activations complete barriers of their own: the converting warps need only the former, and
       // on the first pass over the ring those arrive before the dependency wait
@@ -530,12 +531,25 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       named_bar_sync(1, kDequantThreads);
       {
         const int rows_here = 4 * (b1 - b0);
-        for (int vec = ctid; vec < rows_here * (kTileN / 8); vec += kDequantThreads) {
-          const int row = vec / (kTileN / 8), c16 = vec % (kTileN / 8);
-          const int m = 4 * b0 + row;
-          if (m < m_lim)
-            *reinterpret_cast<uint4*>(p.C + ((size_t)slab * MPAD + m) * p.N + (size_t)col * kTileN + c16 * 8) =
-                *reinterpret_cast<const uint4*>(out + row * kTileN + c16 * 8);
+        if (!p.swiglu) {
+          for (int vec = ctid; vec < rows_here * (kTileN / 8); vec += kDequantThreads) {
+            const int row = vec / (kTileN / 8), c16 = vec % (kTileN / 8);
+            const int m = 4 * b0 + row;
+            if (m < m_lim)
+              *reinterpret_cast<uint4*>(p.C + ((size_t)slab * MPAD + m) * p.N + (size_t)col * kTileN + c16 * 8) =
+                  *reinterpret_cast<const uint4*>(out + row * kTileN + c16 * 8);
+          }
+        } else {
+          // fused activation: every block of 16 columns is eight gate channels and the same eight up channels
+          const int ldc = p.N / 2;
+          for (int vec = ctid; vec < rows_here * (kTileN / 16); vec += kDequantThreads) {
+            const int row = vec / (kTileN / 16), c2 = vec % (kTileN / 16);
+            const int m = 4 * b0 + row;
+            if (m < m_lim)
+              *reinterpret_cast<uint4*>(p.C + ((size_t)slab * MPAD + m) * ldc + (size_t)col * (kTileN / 2) + c2 * 8) =
+                  swiglu8(*reinterpret_cast<const uint4*>(out + row * kTileN + (2 * c2) * 8),
+                          *reinterpret_cast<const uint4*>(out + row * kTileN + (2 * c2 + 1) * 8));
+          }
         }
       }
       cluster_sync_all();                       // nobody reads this CTA's shared memory any more
@@ -554,6 +568,44 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
     const uint32_t fix = (uint32_t)p.ncols <= P ? vcol : (uint32_t)first_w;
     float4* mine = reinterpret_cast<float4*>(p.tc_tiles + (size_t)fix * (kTileN * MPAD)) + n256;
     uint16_t* cptr = p.C + (size_t)slab * MPAD * p.N + (size_t)col * kTileN + n256;
+    // Row m of this thread's column goes to C.  With the fused activation the thread of a gate channel (columns
+    // 0..7 of a block of 16) fetches the up channel's value from the lane eight further on and stores
+    // silu(gate) * up into a C of half the width; every lane of the warp takes part in the exchange.
+    const int ldc = p.N / 2;
+    uint16_t* hptr = p.C + (size_t)slab * MPAD * ldc + (size_t)col * (kTileN / 2) + (n256 >> 4) * 8 + (n256 & 7);
+    auto put_plain = [&](int m, float v) {
+      if (m < m_lim) cptr[(size_t)m * p.N] = __half_as_ushort(__float2half_rn(v));
+    };
+    auto put_act = [&](int m, float v) {
+      const uint32_t h = __half_as_ushort(__float2half_rn(v));
+      const uint32_t other = __shfl_xor_sync(0xffffffffu, h, 8);
+      if ((lane & 8) == 0 && m < m_lim) hptr[(size_t)m * ldc] = (uint16_t)(swiglu2(h, other) & 0xffffu);
+    };
+    if (p.swiglu && !shared_tile) {
+      // fused activation on a tile of its own: 32 batch rows at a time (the exchange between lanes and the
+      // activation need registers of their own)
+#pragma unroll 1
+      for (int cc = 0; cc < MPAD / 32; ++cc) {
+        float part[32];
+        tc_ld_x32(tmem_lane + (uint32_t)(tile * KH * MPAD + cc * 32), part);
+        if constexpr (KH == 2) {
+          float part2[32];
+          tc_ld_x32(tmem_lane + (uint32_t)((tile * KH + 1) * MPAD + cc * 32), part2);
+          tc_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) part[e] += part2[e];
+        } else {
+          tc_wait_ld();
+        }
+#pragma unroll
+        for (int e = 0; e < 32; ++e) put_act(cc * 32 + e, GR ? part[e] : part[e] * sc_col);
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(dempty);
+      u += len;
+      continue;
+    }
     // All accumulators of this thread's channel out of tensor memory first: the MMAs of the next segment may then
     // start while the partial tile goes to the L2 or C is stored.
     float acc[MPAD];
@@ -582,8 +634,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         red_add_f32x4(mine + m4 * kTileN, acc[4 * m4], acc[4 * m4 + 1], acc[4 * m4 + 2], acc[4 * m4 + 3]);
     } else {
 #pragma unroll
-      for (int m = 0; m < MPAD; ++m)
-        if (m < m_lim) cptr[(size_t)m * p.N] = __half_as_ushort(__float2half_rn(acc[m]));
+      for (int m = 0; m < MPAD; ++m) put_plain(m, acc[m]);
     }
 
     if (shared_tile) {
@@ -596,19 +647,39 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       }
       named_bar_sync(1, kDequantThreads);
       if (*last_flag != 0) {
-        // all loads of the total in flight at once: this CTA is alone on the critical path of the tile
-        float4 t4[MPAD / 4];
+        if (!p.swiglu) {
+          // all loads of the total in flight at once: this CTA is alone on the critical path of the tile
+          float4 t4[MPAD / 4];
 #pragma unroll
-        for (int m4 = 0; m4 < MPAD / 4; ++m4) t4[m4] = ld_cg_f4(mine + m4 * kTileN);
+          for (int m4 = 0; m4 < MPAD / 4; ++m4) t4[m4] = ld_cg_f4(mine + m4 * kTileN);
 #pragma unroll
-        for (int m4 = 0; m4 < MPAD / 4; ++m4) mine[m4 * kTileN] = make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int m4 = 0; m4 < MPAD / 4; ++m4) mine[m4 * kTileN] = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int m4 = 0; m4 < MPAD / 4; ++m4) {
-          const int m = 4 * m4;
-          if (m < m_lim) cptr[(size_t)m * p.N] = __half_as_ushort(__float2half_rn(t4[m4].x));
-          if (m + 1 < m_lim) cptr[(size_t)(m + 1) * p.N] = __half_as_ushort(__float2half_rn(t4[m4].y));
-          if (m + 2 < m_lim) cptr[(size_t)(m + 2) * p.N] = __half_as_ushort(__float2half_rn(t4[m4].z));
-          if (m + 3 < m_lim) cptr[(size_t)(m + 3) * p.N] = __half_as_ushort(__float2half_rn(t4[m4].w));
+          for (int m4 = 0; m4 < MPAD / 4; ++m4) {
+            const int m = 4 * m4;
+            put_plain(m, t4[m4].x);
+            put_plain(m + 1, t4[m4].y);
+            put_plain(m + 2, t4[m4].z);
+            put_plain(m + 3, t4[m4].w);
+          }
+        } else {
+          // fused activation: 32 batch rows at a time
+#pragma unroll 1
+          for (int c8 = 0; c8 < MPAD / 32; ++c8) {
+            float4 t4[8];
+#pragma unroll
+            for (int m4 = 0; m4 < 8; ++m4) t4[m4] = ld_cg_f4(mine + (c8 * 8 + m4) * kTileN);
+#pragma unroll
+            for (int m4 = 0; m4 < 8; ++m4) mine[(c8 * 8 + m4) * kTileN] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int m4 = 0; m4 < 8; ++m4) {
+              const int m = 4 * (c8 * 8 + m4);
+              put_act(m, t4[m4].x);
+              put_act(m + 1, t4[m4].y);
+              put_act(m + 2, t4[m4].z);
+              put_act(m + 3, t4[m4].w);
+            }
+          }
         }
       }
       named_bar_sync(1, kDequantThreads);  // last_flag may be rewritten by the next segment

@@ -77,6 +77,8 @@ struct GemmParams {
   float* partials;   // warp-MMA kernel: partial-tile slots
   float* tc_tiles;   // tcgen05 kernel: one fp32 accumulation tile per 256-column tile
   int slot_floats;   // floats per partial-tile slot
+  int swiglu;        // 1: the columns come in blocks of 16 (eight gate channels, then the same eight up channels) and the
+                     // kernel stores silu(gate) * up, N / 2 columns per row of C
   uint32_t cluster;  // tcgen05 kernel: 1 = launched as thread-block clusters of `split` CTAs (the CTAs of one column tile)
   uint32_t slabs;    // tcgen05 kernel: slabs of 128 batch rows in this launch (1 up to 128 rows); virtual column tile
                      // v = column tile v / slabs of W, batch rows 128 * (v % slabs) ..
@@ -109,6 +111,9 @@ cudaError_t launch_pack_dense(uint32_t* q, uint16_t* s, uint32_t* wq, uint16_t* 
 // round-to-nearest quantiser with clipping search (quantize.cu): W fp16 [K][N] -> canonical codes and scales
 cudaError_t launch_quantize_rtn(const uint16_t* W, uint32_t* q_kpacked, uint16_t* scales, int K, int N, int G, int n_grid,
                                 int n_candidates, cudaStream_t stream);
+// gate and up projections side by side in blocks of 16 columns (8 gate, 8 up), canonical codes and scales
+cudaError_t launch_interleave_gate_up(const uint32_t* q_gate, const uint16_t* s_gate, const uint32_t* q_up, const uint16_t* s_up,
+                                      uint32_t* q_out, uint16_t* s_out, int K, int I, int G, cudaStream_t stream);
 // canonical zero points uint8 [K/G][N] (0..15) <-> fp16 values in the packed order of the scales
 cudaError_t launch_permute_zeros(uint8_t* z, uint16_t* zq, int K, int N, int G, bool inverse, cudaStream_t stream);
 // canonical scales [K/G][N] <-> packed order (shared by the dense and the 2:4 pack)

@@ -157,7 +157,33 @@ __global__ void permute_zeros_kernel(uint8_t* __restrict__ z, uint16_t* __restri
   }
 }
 
+// out[row][n], n = 16 b + r: r < 8 -> gate[row][8 b + r], else up[row][8 b + r - 8]
+template <typename T>
+__global__ void interleave_gate_up_kernel(const T* __restrict__ gate, const T* __restrict__ up, T* __restrict__ out,
+                                          long long rows, int I) {
+  const long long total = rows * 2 * I;
+  for (long long x = blockIdx.x * (long long)blockDim.x + threadIdx.x; x < total; x += (long long)gridDim.x * blockDim.x) {
+    const long long row = x / (2 * I);
+    const int n = (int)(x % (2 * I));
+    const int b = n >> 4, r = n & 15;
+    out[x] = r < 8 ? gate[row * I + 8 * b + r] : up[row * I + 8 * b + r - 8];
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_interleave_gate_up(const uint32_t* q_gate, const uint16_t* s_gate, const uint32_t* q_up, const uint16_t* s_up,
+                                      uint32_t* q_out, uint16_t* s_out, int K, int I, int G, cudaStream_t stream) {
+  const int threads = 256;
+  const long long qrows = K / 8, srows = K / G;
+  int blocks = (int)((qrows * 2 * I + threads - 1) / threads);
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  interleave_gate_up_kernel<uint32_t><<<blocks, threads, 0, stream>>>(q_gate, q_up, q_out, qrows, I);
+  blocks = (int)((srows * 2 * I + threads - 1) / threads);
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  interleave_gate_up_kernel<uint16_t><<<blocks, threads, 0, stream>>>(s_gate, s_up, s_out, srows, I);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_permute_zeros(uint8_t* z, uint16_t* zq, int K, int N, int G, bool inverse, cudaStream_t stream) {
   const long long ns = (long long)(K / G) * N;

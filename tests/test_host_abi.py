@@ -142,3 +142,18 @@ def test_byte_model_matches_paper():
     # with scales: 2 bytes per (group, column)
     assert roofline.weight_bytes(8192, 8192, 128) == 8192 * 8192 // 2 + 2 * 64 * 8192
     assert roofline.weight_bytes(8192, 8192, 128, sparse24=True) == 8192 * 8192 // 4 + 8192 * 8192 // 8 + 2 * 64 * 8192
+
+
+def test_no_kernel_of_the_built_library_spills_registers_to_memory():
+    # the register allocator's report of the last build: a kernel that starts spilling hundreds of bytes has lost its
+    # place in the register file (seen once: an epilogue variant cost the large-batch kernel a third of its speed)
+    from paper_2408_11743_b200 import build
+    build.build()
+    report = build.spill_report()
+    if not report:
+        build.build(force=True)
+        report = build.spill_report()
+    assert report, "no ptxas report beside the library"
+    assert len(report) >= 20
+    bad = {k: v for k, v in report.items() if v[1] > 64}
+    assert not bad, bad
