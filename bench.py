@@ -4,6 +4,7 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-extra]
     python bench.py --sustain SECONDS          # the same step replayed for that long, rate per SM-clock bin
     python bench.py --case M,K,N,G[,sparse]    # one layer shape a few times (for profiler captures)
+    python bench.py --case C,K,N,G,quantize    # the quantiser with C clipping candidates on a K x N matrix
 
 Workload (config 2 of this build): K = N = 8192, group size 128, M in {1,2,4,8,16,32,64,128};
 A ~ fp16 N(0,1), codes uniform 0..15 (zero point 8), scales uniform in [0.005, 0.02]; synthetic.
@@ -372,6 +373,21 @@ def run_case(args):
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
     stream = torch.cuda.Stream(device=dev)
+    if len(parts) > 4 and parts[4].startswith("quantize"):
+        # M is the number of clipping candidates here: the quantiser on a K x N matrix, a few launches
+        W = torch.randn((K, N), device=dev, dtype=torch.float32).mul_(0.02).half()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            marlin.quantize_rtn(W, G, 20, M, stream=stream)
+            e0.record(stream)
+            for _ in range(args.iters):
+                marlin.quantize_rtn(W, G, 20, M, stream=stream)
+            e1.record(stream)
+        e1.synchronize()
+        t = e0.elapsed_time(e1) * 1e-3 / args.iters
+        print(json.dumps({"quantize_rtn": True, "K": K, "N": N, "G": G, "n_grid": 20, "n_candidates": M,
+                          "us": round(t * 1e6, 1), "gweights_per_s": round(K * N / t / 1e9, 1)}), flush=True)
+        return
     peaks = roofline.load_peaks(ROOT)
     l2 = args.copies_bytes
     layer = LayerBench(marlin, dev, stream, l2, K, N, G, sparse, np.random.default_rng(1), with_fp16=False)
