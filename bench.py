@@ -3,7 +3,7 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-extra]
     python bench.py --sustain SECONDS          # the same step replayed for that long, rate per SM-clock bin
-    python bench.py --case M,K,N,G[,sparse]    # one layer shape a few times (for profiler captures)
+    python bench.py --case M,K,N,G[,sparse|w8] # one layer shape a few times (for profiler captures)
     python bench.py --case C,K,N,G,quantize    # the quantiser with C clipping candidates on a K x N matrix
 
 Workload (config 2 of this build): K = N = 8192, group size 128, M in {1,2,4,8,16,32,64,128};
@@ -187,13 +187,17 @@ def run_reference(args):
 class LayerBench:
     """One packed layer resident on the GPU (several cold copies) and its cuBLAS fp16 counterpart, timed per batch size."""
 
-    def __init__(self, marlin, dev, stream, l2, K, N, G, sparse, rng, with_fp16=True):
+    def __init__(self, marlin, dev, stream, l2, K, N, G, sparse, rng, with_fp16=True, w8=False):
         import torch
         self.m, self.dev, self.stream, self.K, self.N, self.G, self.sparse = marlin, dev, stream, K, N, G, sparse
-        self.wb = roofline.weight_bytes(K, N, G, sparse24=sparse)
+        self.w8 = w8
+        self.wb = roofline.weight_bytes(K, N, G, sparse24=sparse, bits=8 if w8 else 4)
         self.copies = max(2, int(np.ceil(2.0 * l2 / self.wb)) + 1)
         S = torch.from_numpy(rng.uniform(0.005, 0.02, size=(K // G, N)).astype(np.float16)).to(dev)
-        if sparse:
+        if w8:
+            q8 = torch.from_numpy(rng.integers(0, 256, size=(K, N), dtype=np.uint8)).to(dev)
+            packed0 = marlin.pack_w8(q8, S, G)
+        elif sparse:
             qc = torch.from_numpy(rng.integers(-2**31, 2**31 - 1, size=(K // 16, N), dtype=np.int64).astype(np.int32)).to(dev)
             pat = rng.integers(0, 6, size=(K // 4, N))
             idx = np.empty((K // 2, N), dtype=np.uint8)
@@ -220,7 +224,9 @@ class LayerBench:
         def call():
             pk = self.packed[rot[0] % self.copies]
             rot[0] += 1
-            if self.sparse:
+            if self.w8:
+                marlin.gemm_w8(A, pk[0], pk[1], K, N, G, ws, out=C, stream=stream)
+            elif self.sparse:
                 marlin.gemm_sparse24(A, pk[0], pk[1], pk[2], K, N, G, ws, out=C, stream=stream)
             else:
                 marlin.gemm(A, pk[0], pk[1], K, N, G, ws, out=C, stream=stream)
@@ -232,7 +238,7 @@ class LayerBench:
         g = capture(call, reps)
         time_graph(g)
         t = min(time_graph(g) for _ in range(5)) / reps
-        troof = roofline.roofline_seconds(M, K, N, G, peaks, sparse24=self.sparse)
+        troof = roofline.roofline_seconds(M, K, N, G, peaks, sparse24=self.sparse, bits=8 if self.w8 else 4)
         if marlin.read_status(ws, stream=stream) != 0:
             raise RuntimeError("device-side wait expired")
         r = {"K": K, "N": N, "G": G, "M": M, "sparse24": self.sparse, "us": round(t * 1e6, 3),
@@ -321,8 +327,8 @@ def extra_layers(marlin, dev, stream, l2, peaks, capture, time_graph):
     out = []
     rng = np.random.default_rng(1234)
 
-    def sweep(K, N, G, sparse, Ms, label, config):
-        layer = LayerBench(marlin, dev, stream, l2, K, N, G, sparse, rng)
+    def sweep(K, N, G, sparse, Ms, label, config, w8=False):
+        layer = LayerBench(marlin, dev, stream, l2, K, N, G, sparse, rng, w8=w8)
         for M in Ms:
             r = layer.time(M, capture, time_graph, peaks)
             r["layer"], r["config"] = label, config
@@ -350,6 +356,8 @@ def extra_layers(marlin, dev, stream, l2, peaks, capture, time_graph):
                     "us": round(tq * 1e6, 1), "gweights_per_s": round(8192 * 8192 / tq / 1e9, 1),
                     "algorithmic_gbs": round((8192 * 8192 * 2.5 + 2 * 64 * 8192) / tq / 1e9, 1)})
         del Wq
+    # 8-bit weights on the same layer (twice the bytes per weight: the roofline time doubles)
+    sweep(8192, 8192, GROUP, False, (1, 16, 64, 128), "8-bit weights 8192x8192", 2, w8=True)
     # the gated MLP of a Llama-2-7B layer as a chain: gate_up with the activation fused into its epilogue, then down
     # (two launches, the second under programmatic dependent launch), against the same layers with the activation
     # as separate elementwise kernels on the wide intermediate
@@ -368,6 +376,7 @@ def run_case(args):
     parts = args.case.split(",")
     M, K, N, G = (int(x) for x in parts[:4])
     sparse = len(parts) > 4 and parts[4].startswith("sparse")
+    w8 = len(parts) > 4 and parts[4].startswith("w8")
     if G <= 0:
         G = K
     torch.cuda.set_device(0)
@@ -390,7 +399,7 @@ def run_case(args):
         return
     peaks = roofline.load_peaks(ROOT)
     l2 = args.copies_bytes
-    layer = LayerBench(marlin, dev, stream, l2, K, N, G, sparse, np.random.default_rng(1), with_fp16=False)
+    layer = LayerBench(marlin, dev, stream, l2, K, N, G, sparse, np.random.default_rng(1), with_fp16=False, w8=w8)
 
     def capture(fn, reps):
         g = torch.cuda.CUDAGraph()

@@ -170,6 +170,21 @@ MARLIN_API int marlin_mlp_swiglu(const void* A, const void* w_gate_up, const voi
                       const void* s_down, void* H, void* C, int M, int K, int I, int N, int group_size,
                       void* workspace, size_t workspace_bytes, marlin_stream stream);
 
+/* ---- 8-bit weights (Section 6 names other formats the approach extends to): W = (q - 128) * s, q in 0..255 ------ */
+
+/* q8: device, uint8 [K][N] row-major codes; scales as for marlin_pack.  w_packed: marlin_packed_weight_bytes_w8(K, N)
+ * = K * N bytes.  N % 256 == 0 (these layers run on the tcgen05 kernel at every batch size).  Integer-only
+ * permutation; marlin_unpack_w8 is its inverse bit for bit. */
+MARLIN_API size_t marlin_packed_weight_bytes_w8(int K, int N);
+MARLIN_API int marlin_pack_w8(const uint8_t* q8, const void* scales, void* w_packed, void* s_packed, int K, int N,
+                   int group_size, marlin_stream stream);
+MARLIN_API int marlin_unpack_w8(const void* w_packed, const void* s_packed, uint8_t* q8, void* scales, int K, int N,
+                     int group_size, marlin_stream stream);
+/* C = A . W as marlin_gemm; the conversion places a code byte under the exponent of 1024 and subtracts 1152 (the
+ * 8-bit form of the exponent trick of Section 3.4 "Dequantization and Tensor Cores"), scales in the loop. */
+MARLIN_API int marlin_gemm_w8(const void* A, const void* w_packed, const void* s_packed, void* C, int M, int K, int N,
+                   int group_size, void* workspace, size_t workspace_bytes, marlin_stream stream);
+
 /* The layer with zero points: C = A . W, W[k][n] = (q[k][n] - z[k/G][n]) * s[k/G][n].  Arguments as marlin_gemm, plus
  * z_packed from marlin_pack_zeros.  N % 256 == 0 (else MARLIN_ERR_SHAPE); every batch size runs on the tcgen05
  * kernel, where the zero point replaces the constant 8 inside the conversion (the subtrahend of the exponent

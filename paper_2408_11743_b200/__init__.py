@@ -10,6 +10,7 @@ from .binding import (  # noqa: F401
     gemm_sparse24,
     gemm_static_ws,
     gemm_swiglu,
+    gemm_w8,
     interleave_gate_up,
     gemm_zp,
     lib,
@@ -18,12 +19,14 @@ from .binding import (  # noqa: F401
     new_workspace,
     pack,
     pack_sparse24,
+    pack_w8,
     pack_zeros,
     plan_stripes,
     quantize_rtn,
     read_status,
     unpack,
     unpack_sparse24,
+    unpack_w8,
     unpack_zeros,
     workspace_bytes,
 )

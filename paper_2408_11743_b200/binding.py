@@ -19,6 +19,7 @@ EXPORTS = [
     "marlin_unpack_sparse24", "marlin_gemm_sparse24", "marlin_read_status", "marlin_plan_stripes",
     "marlin_gemm_static_ws", "marlin_quantize_rtn", "marlin_pack_zeros", "marlin_unpack_zeros", "marlin_gemm_zp",
     "marlin_interleave_gate_up", "marlin_gemm_swiglu", "marlin_mlp_swiglu",
+    "marlin_packed_weight_bytes_w8", "marlin_pack_w8", "marlin_unpack_w8", "marlin_gemm_w8",
 ]
 STATIC_WS_MAX_M = 16  # MARLIN_STATIC_WS_MAX_M of the header
 
@@ -62,6 +63,11 @@ def lib():
     L.marlin_pack_zeros.argtypes = [vp, vp, i, i, i, vp]
     L.marlin_unpack_zeros.argtypes = [vp, vp, i, i, i, vp]
     L.marlin_gemm_zp.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
+    L.marlin_packed_weight_bytes_w8.restype = sz
+    L.marlin_packed_weight_bytes_w8.argtypes = [i, i]
+    L.marlin_pack_w8.argtypes = [vp, vp, vp, vp, i, i, i, vp]
+    L.marlin_unpack_w8.argtypes = [vp, vp, vp, vp, i, i, i, vp]
+    L.marlin_gemm_w8.argtypes = [vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
     L.marlin_interleave_gate_up.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, vp]
     L.marlin_gemm_swiglu.argtypes = [vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
     L.marlin_mlp_swiglu.argtypes = [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp, sz, vp]
@@ -72,7 +78,7 @@ def lib():
     L.marlin_gemm_sparse24.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, vp, sz, vp]
     L.marlin_read_status.argtypes = [vp, vp]
     L.marlin_plan_stripes.argtypes = [i, i, i, i, vp, vp, vp, i]
-    for name in ("marlin_interleave_gate_up", "marlin_gemm_swiglu", "marlin_mlp_swiglu", "marlin_pack_zeros", "marlin_unpack_zeros", "marlin_gemm_zp", "marlin_quantize_rtn", "marlin_gemm_static_ws", "marlin_pack", "marlin_unpack", "marlin_gemm", "marlin_pack_sparse24", "marlin_unpack_sparse24",
+    for name in ("marlin_pack_w8", "marlin_unpack_w8", "marlin_gemm_w8", "marlin_interleave_gate_up", "marlin_gemm_swiglu", "marlin_mlp_swiglu", "marlin_pack_zeros", "marlin_unpack_zeros", "marlin_gemm_zp", "marlin_quantize_rtn", "marlin_gemm_static_ws", "marlin_pack", "marlin_unpack", "marlin_gemm", "marlin_pack_sparse24", "marlin_unpack_sparse24",
                  "marlin_gemm_sparse24", "marlin_read_status", "marlin_plan_stripes"):
         getattr(L, name).restype = i
     _lib = L
@@ -320,6 +326,67 @@ def mlp_swiglu(A, w_gate_up, s_gate_up, w_down, s_down, K: int, I: int, N: int, 
     _check(L.marlin_mlp_swiglu(A.data_ptr(), wg.data_ptr(), sg.data_ptr(), wd.data_ptr(), sd.data_ptr(), H.data_ptr(),
                                out.data_ptr(), M, K, I, N, group_size, ws.data_ptr(), ws.numel(), _stream_ptr(stream)),
            "marlin_mlp_swiglu")
+    return out
+
+
+def pack_w8(q8, scales, group_size: int, stream=None):
+    """marlin_pack_w8: 8-bit codes uint8 [K, N] + fp16 scales [K/G, N] -> (w_packed, s_packed); N % 256 == 0."""
+    torch = _torch()
+    q = _dev(q8, torch.uint8, "q8")
+    s = _dev(scales, torch.float16, "scales")
+    K, N = q.shape
+    L = lib()
+    wb, sb = L.marlin_packed_weight_bytes_w8(K, N), L.marlin_packed_scale_bytes(K, N, group_size)
+    if wb == 0:
+        raise MarlinError(2, "marlin_pack_w8")
+    if sb == 0:
+        raise MarlinError(3, "marlin_pack_w8")
+    if s.numel() * 2 != sb:
+        raise ValueError(f"scales has {s.numel()} elements, expected {sb // 2}")
+    w_packed = torch.empty(wb, dtype=torch.uint8, device=q.device)
+    s_packed = torch.empty(sb, dtype=torch.uint8, device=q.device)
+    _check(L.marlin_pack_w8(q.data_ptr(), s.data_ptr(), w_packed.data_ptr(), s_packed.data_ptr(), K, N, group_size,
+                            _stream_ptr(stream)), "marlin_pack_w8")
+    return w_packed, s_packed
+
+
+def unpack_w8(w_packed, s_packed, K: int, N: int, group_size: int, stream=None):
+    """marlin_unpack_w8: the inverse of pack_w8; returns (q8 uint8 [K, N], scales fp16 [K/G, N])."""
+    torch = _torch()
+    w = _dev(w_packed, torch.uint8, "w_packed")
+    s = _dev(s_packed, torch.uint8, "s_packed")
+    L = lib()
+    sb = L.marlin_packed_scale_bytes(K, N, group_size)
+    if w.numel() != L.marlin_packed_weight_bytes_w8(K, N) or s.numel() != sb or sb == 0:
+        raise ValueError("packed buffer sizes do not match K, N, group_size")
+    q = torch.empty((K, N), dtype=torch.uint8, device=w.device)
+    sc = torch.empty((sb // (2 * N), N), dtype=torch.float16, device=w.device)
+    _check(L.marlin_unpack_w8(w.data_ptr(), s.data_ptr(), q.data_ptr(), sc.data_ptr(), K, N, group_size, _stream_ptr(stream)),
+           "marlin_unpack_w8")
+    return q, sc
+
+
+def gemm_w8(A, w_packed, s_packed, K: int, N: int, group_size: int, workspace, out=None, stream=None):
+    """marlin_gemm_w8: C = A . ((q - 128) * s) for 8-bit codes."""
+    torch = _torch()
+    A = _dev(A, torch.float16, "A")
+    if A.dim() != 2 or A.shape[1] != K:
+        raise ValueError("A must be [M, K]")
+    M = A.shape[0]
+    w = _dev(w_packed, torch.uint8, "w_packed")
+    s = _dev(s_packed, torch.uint8, "s_packed")
+    ws = _dev(workspace, torch.uint8, "workspace")
+    L = lib()
+    if w.numel() != L.marlin_packed_weight_bytes_w8(K, N) or s.numel() != L.marlin_packed_scale_bytes(K, N, group_size):
+        raise ValueError("packed buffer sizes do not match K, N, group_size")
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float16, device=A.device)
+    else:
+        _dev(out, torch.float16, "out")
+        if tuple(out.shape) != (M, N):
+            raise ValueError("out must be [M, N]")
+    _check(L.marlin_gemm_w8(A.data_ptr(), w.data_ptr(), s.data_ptr(), out.data_ptr(), M, K, N, group_size,
+                            ws.data_ptr(), ws.numel(), _stream_ptr(stream)), "marlin_gemm_w8")
     return out
 
 

@@ -208,18 +208,19 @@ int marlin_unpack(const void* w_packed, const void* s_packed, uint32_t* q_kpacke
 // Shared body of marlin_gemm and marlin_gemm_sparse24 (meta_packed == nullptr: dense).
 static int gemm_common(const void* A, const void* w_packed, const void* meta_packed, const void* s_packed, void* C, int M,
                        int K, int N, int group_size, void* workspace, size_t workspace_bytes, marlin_stream stream,
-                       bool sparse24, const void* z_packed = nullptr, bool swiglu = false) {
+                       bool sparse24, const void* z_packed = nullptr, bool swiglu = false, bool w8 = false) {
   if (!A || !w_packed || !s_packed || !C || !workspace || (sparse24 && !meta_packed)) return MARLIN_ERR_NULL;
   // layers with zero points run on the tcgen05 kernel alone (N a multiple of 256), at every batch size
   const bool zero_points = z_packed != nullptr;
   if (zero_points && (N % 256 || !aligned16(z_packed))) return N % 256 ? MARLIN_ERR_SHAPE : MARLIN_ERR_ALIGN;
+  if (w8 && N % 256) return MARLIN_ERR_SHAPE;  // 8-bit codes: the tcgen05 kernel alone, at every batch size
   if (M < 1 || !shape_ok(K, N)) return MARLIN_ERR_SHAPE;
   int G = normalise_group(K, N, group_size);
   if (!G) return MARLIN_ERR_GROUP;
   if (!aligned16(A) || !aligned16(w_packed) || !aligned16(s_packed) || !aligned16(C) || !aligned16(workspace) ||
       (sparse24 && !aligned16(meta_packed)))
     return MARLIN_ERR_ALIGN;
-  if (workspace_bytes < workspace_bytes_for(M, K, N, sparse24 || G < kTileK || zero_points)) return MARLIN_ERR_WORKSPACE;
+  if (workspace_bytes < workspace_bytes_for(M, K, N, sparse24 || G < kTileK || zero_points || w8)) return MARLIN_ERR_WORKSPACE;
   DeviceInfo info;
   int st = device_info(&info);
   if (st != MARLIN_OK) return st;
@@ -238,7 +239,7 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
     // it takes every batch size there
     const bool tc_ok = tc_path_supported(1, K, N);
     // groups of 64 or 32 rows likewise (accepted only where N is a multiple of 256)
-    const bool small_groups = G < kTileK || zero_points;
+    const bool small_groups = G < kTileK || zero_points || w8;
     // (the kernel with deferred scales has no fused activation: those layers go through the warp-level kernel then)
     const bool use_tcd = !swiglu && !sparse24 && !small_groups && tcd_path_supported(1, K, N) &&
                          (tmode == 1 || (tmode == 2 && rem >= tc_min_m() && !tc_ok));
@@ -277,7 +278,7 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
     if (use_tcd) {
       if (launch_gemm_tcd(p, info.sm_count, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MARLIN_ERR_CUDA;
     } else if (use_tc) {
-      if (launch_gemm_dense_tc(p, info.sm_count, sparse24, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+      if (launch_gemm_dense_tc(p, info.sm_count, sparse24, static_cast<cudaStream_t>(stream), w8) != cudaSuccess)
         return MARLIN_ERR_CUDA;
     } else {
       DensePlan plan;
@@ -329,6 +330,47 @@ int marlin_mlp_swiglu(const void* A, const void* w_gate_up, const void* s_gate_u
   int st = marlin_gemm_swiglu(A, w_gate_up, s_gate_up, H, M, K, 2 * I, group_size, workspace, workspace_bytes, stream);
   if (st != MARLIN_OK) return st;
   return marlin_gemm(H, w_down, s_down, C, M, I, N, group_size, workspace, workspace_bytes, stream);
+}
+
+size_t marlin_packed_weight_bytes_w8(int K, int N) {
+  if (!shape_ok(K, N) || N % 256) return 0;
+  return (size_t)K * N;
+}
+
+int marlin_pack_w8(const uint8_t* q8, const void* scales, void* w_packed, void* s_packed, int K, int N, int group_size,
+                   marlin_stream stream) {
+  if (!q8 || !scales || !w_packed || !s_packed) return MARLIN_ERR_NULL;
+  if (!shape_ok(K, N) || N % 256) return MARLIN_ERR_SHAPE;
+  int G = normalise_group(K, N, group_size);
+  if (!G) return MARLIN_ERR_GROUP;
+  if (!aligned16(q8) || !aligned16(scales) || !aligned16(w_packed) || !aligned16(s_packed)) return MARLIN_ERR_ALIGN;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (launch_pack_w8(const_cast<uint8_t*>(q8), static_cast<uint8_t*>(w_packed), K, N, false, st) != cudaSuccess)
+    return MARLIN_ERR_CUDA;
+  cudaError_t err = launch_permute_scales(static_cast<uint16_t*>(const_cast<void*>(scales)), static_cast<uint16_t*>(s_packed),
+                                          K, N, G, false, st);
+  return err == cudaSuccess ? MARLIN_OK : MARLIN_ERR_CUDA;
+}
+
+int marlin_unpack_w8(const void* w_packed, const void* s_packed, uint8_t* q8, void* scales, int K, int N, int group_size,
+                     marlin_stream stream) {
+  if (!q8 || !scales || !w_packed || !s_packed) return MARLIN_ERR_NULL;
+  if (!shape_ok(K, N) || N % 256) return MARLIN_ERR_SHAPE;
+  int G = normalise_group(K, N, group_size);
+  if (!G) return MARLIN_ERR_GROUP;
+  if (!aligned16(q8) || !aligned16(scales) || !aligned16(w_packed) || !aligned16(s_packed)) return MARLIN_ERR_ALIGN;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (launch_pack_w8(q8, static_cast<uint8_t*>(const_cast<void*>(w_packed)), K, N, true, st) != cudaSuccess)
+    return MARLIN_ERR_CUDA;
+  cudaError_t err = launch_permute_scales(static_cast<uint16_t*>(scales), static_cast<uint16_t*>(const_cast<void*>(s_packed)),
+                                          K, N, G, true, st);
+  return err == cudaSuccess ? MARLIN_OK : MARLIN_ERR_CUDA;
+}
+
+int marlin_gemm_w8(const void* A, const void* w_packed, const void* s_packed, void* C, int M, int K, int N, int group_size,
+                   void* workspace, size_t workspace_bytes, marlin_stream stream) {
+  return gemm_common(A, w_packed, nullptr, s_packed, C, M, K, N, group_size, workspace, workspace_bytes, stream, false,
+                     nullptr, false, true);
 }
 
 int marlin_gemm_zp(const void* A, const void* w_packed, const void* s_packed, const void* z_packed, void* C, int M, int K,

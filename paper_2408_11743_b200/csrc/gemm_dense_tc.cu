@@ -62,11 +62,17 @@ constexpr int kDequantRegs = 216;    // 512 threads start with 128 each: 2 x 128
 // SP: the 2:4 variant (Section 4).  A stage then holds the 64 kept codes per column of the k-block (8 KB) and the
 // metadata words of the 256 tensor-memory lanes (4 KB); an A-operand slot holds 32 columns of kept values and 4
 // columns of metadata per 128-channel tile.
-template <int MPAD, bool SP>
+// FMT: 0 = dense 4-bit codes, 1 = the 2:4 variant, 2 = dense 8-bit codes (W = (q - 128) * s: a stage holds 128 bytes per
+// column, [8 vectors][256 columns][16 bytes], the conversion places a byte under the exponent 0x64 with one byte
+// permute per pair of weights and subtracts 1152; everything after the conversion is the 4-bit path).
+constexpr int kFmtDense4 = 0, kFmtSparse4 = 1, kFmtDense8 = 2;
+template <int MPAD, int FMT>
 struct TcGeometry {
+  static constexpr bool SP = FMT == kFmtSparse4;
+  static constexpr bool W8 = FMT == kFmtDense8;
   static constexpr int A_HALF_BYTES = MPAD * 128;
   static constexpr int A_BYTES = 2 * A_HALF_BYTES;
-  static constexpr int W_BYTES = SP ? 2 * kChunkBytes : 4 * kChunkBytes;
+  static constexpr int W_BYTES = SP ? 2 * kChunkBytes : (W8 ? 8 * kChunkBytes : 4 * kChunkBytes);
   static constexpr int META_BYTES = SP ? kChunkBytes : 0;
   static constexpr int STAGE_BYTES = A_BYTES + W_BYTES + META_BYTES;
   static constexpr int SC_ROW_BYTES = kTileN * 2;                   // one row of the tile's group scales
@@ -107,10 +113,12 @@ struct TcGeometry {
 // ---------------------------------------------------------------------------------------------
 // GR: the layer has group scales (multiplied into the weights in the loop); otherwise one scale per column,
 // applied to the accumulators in the epilogue.
-template <int MPAD, bool GR, bool SP>
+template <int MPAD, bool GR, int FMT>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a) {
-  using G = TcGeometry<MPAD, SP>;
+  using G = TcGeometry<MPAD, FMT>;
+  constexpr bool SP = G::SP;
+  constexpr bool W8 = G::W8;
   constexpr int NSTAGES = G::STAGES;
   constexpr int NSLOTS = G::A_SLOTS;
   constexpr int NM = G::MMA_WARPS;
@@ -391,9 +399,12 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
           }
         }
       }
-      const uint32_t wbase = smem_u32(stage0) + (uint32_t)s * G::STAGE_BYTES + G::A_BYTES + (SP ? (uint32_t)n256 * 16u : vec_off);
-      uint4 v[4];
-      if constexpr (!SP) {
+      const uint32_t wbase = smem_u32(stage0) + (uint32_t)s * G::STAGE_BYTES + G::A_BYTES + ((SP || W8) ? (uint32_t)n256 * 16u : vec_off);
+      uint4 v[W8 ? 8 : 4];
+      if constexpr (W8) {
+#pragma unroll
+        for (int c = 0; c < 8; ++c) v[c] = lds128(wbase + c * 256 * 16);  // codes of rows 16c .. 16c + 15 of this column
+      } else if constexpr (!SP) {
 #pragma unroll
         for (int c = 0; c < 4; ++c) v[c] = lds128(wbase + c * 16);
       } else {
@@ -412,7 +423,28 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       }
       tc_fence_after_sync();
       const uint32_t slot_col = tmem_lane + (uint32_t)(G::A_COL0 + slot * G::SLOT_COLS);
-      if constexpr (!SP) {
+      if constexpr (W8) {
+        const uint32_t a_col = slot_col + (uint32_t)(tile * 64);
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+          uint32_t r[32];
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const uint4 vv = v[4 * hh + c];
+            const uint32_t w4[4] = {vv.x, vv.y, vv.z, vv.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              // bytes (b0, b1) and (b2, b3) of the word under the exponent of 1024: 1024 + b, minus 1152 = b - 128
+              const uint32_t lo = hsub2_u32(__byte_perm(w4[e], 0x64646464u, 0x4140), 0x64806480u);
+              const uint32_t hi = hsub2_u32(__byte_perm(w4[e], 0x64646464u, 0x4342), 0x64806480u);
+              // rows 64hh + 16c ..: quarter 2hh + c / 2 of the k-block
+              r[8 * c + 2 * e] = GR ? hmul2_u32(lo, sv4[2 * hh + (c >> 1)]) : lo;
+              r[8 * c + 2 * e + 1] = GR ? hmul2_u32(hi, sv4[2 * hh + (c >> 1)]) : hi;
+            }
+          }
+          tc_st_x32(a_col + (uint32_t)(32 * hh), r);  // column = row / 2
+        }
+      } else if constexpr (!SP) {
         const uint32_t a_col = slot_col + (uint32_t)(tile * 64);
 #pragma unroll
         for (int hh = 0; hh < 2; ++hh) {
@@ -691,10 +723,10 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
   named_bar_sync(2, kDequantThreads + 32);
 }
 
-template <int MPAD, bool GR, bool SP>
+template <int MPAD, bool GR, int FMT>
 cudaError_t launch_tc(const GemmParams& p, int workers, cudaStream_t stream) {
-  using G = TcGeometry<MPAD, SP>;
-  auto kernel = gemm_dense_tc_kernel<MPAD, GR, SP>;
+  using G = TcGeometry<MPAD, FMT>;
+  auto kernel = gemm_dense_tc_kernel<MPAD, GR, FMT>;
   static bool attr_set[64] = {};
   int dev = 0;
   cudaError_t err = cudaGetDevice(&dev);
@@ -768,7 +800,7 @@ size_t tc_fixup_tiles(int M, int N, int workers) {
 
 int tc_mpad(int m_slab) { return m_slab <= 32 ? 32 : (m_slab <= 64 ? 64 : 128); }
 
-cudaError_t launch_gemm_dense_tc(GemmParams p, int sm_count, bool sparse24, cudaStream_t stream) {
+cudaError_t launch_gemm_dense_tc(GemmParams p, int sm_count, bool sparse24, cudaStream_t stream, bool w8) {
   // stripe plan for 256-column tiles
   // above 128 rows the layer is replicated in the unit numbering, once per slab of 128 rows (Section 3.4, last
   // paragraph): one launch, its stripes running over (column tile, slab, k-block)
@@ -807,6 +839,16 @@ cudaError_t launch_gemm_dense_tc(GemmParams p, int sm_count, bool sparse24, cuda
   }
   p.workers = (uint32_t)workers;
   const int mpad = tc_mpad(p.M < kTcMaxSlabM ? p.M : kTcMaxSlabM);
+  if (w8) {
+    if (p.grouped) {
+      if (mpad == 32) return launch_tc<32, true, kFmtDense8>(p, (int)workers, stream);
+      if (mpad == 64) return launch_tc<64, true, kFmtDense8>(p, (int)workers, stream);
+      return launch_tc<128, true, kFmtDense8>(p, (int)workers, stream);
+    }
+    if (mpad == 32) return launch_tc<32, false, kFmtDense8>(p, (int)workers, stream);
+    if (mpad == 64) return launch_tc<64, false, kFmtDense8>(p, (int)workers, stream);
+    return launch_tc<128, false, kFmtDense8>(p, (int)workers, stream);
+  }
   if (sparse24) {
     if (p.grouped) {
       if (mpad == 32) return launch_tc<32, true, true>(p, (int)workers, stream);

@@ -98,7 +98,10 @@ int tc_max_rows(int K, int N, int sm_count);      // most rows one launch takes 
 size_t tc_fixup_tiles(int M, int N, int workers); // fp32 accumulation tiles (256 columns x padded rows) the fix-up needs
 // fills the plan fields of `p` (ncols, units, workers) itself; sparse24: the 2:4 instances (tcgen05.mma.sp), which read
 // the wide 2:4 layout (N a multiple of 256)
-cudaError_t launch_gemm_dense_tc(GemmParams p, int sm_count, bool sparse24, cudaStream_t stream);
+// w8: the instances for 8-bit codes (N a multiple of 256)
+cudaError_t launch_gemm_dense_tc(GemmParams p, int sm_count, bool sparse24, cudaStream_t stream, bool w8 = false);
+// 8-bit codes uint8 [K][N] <-> packed [N/256][K/128][8 vectors][256 columns][16 bytes]
+cudaError_t launch_pack_w8(uint8_t* q8, uint8_t* wq, int K, int N, bool inverse, cudaStream_t stream);
 // tcgen05 kernel with deferred scales (gemm_tcd.cu): 128-column tiles, up to 64 rows of A per launch.
 bool tcd_path_supported(int m_slab, int K, int N);
 int tcd_mpad(int m_slab);            // rows of A padded to the MMA's N: 16, 32 or 64

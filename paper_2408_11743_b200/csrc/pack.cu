@@ -170,7 +170,38 @@ __global__ void interleave_gate_up_kernel(const T* __restrict__ gate, const T* _
   }
 }
 
+// 8-bit codes: one thread per 16-byte vector of the packed buffer = rows 128 kb + 16 c + 0..15 of column 256 T + n
+__global__ void pack_w8_kernel(uint8_t* __restrict__ q8, uint8_t* __restrict__ wq, int K, int N, bool inverse) {
+  const long long vecs = (long long)K * N / 16;
+  const int KB = K / 128;
+  for (long long v = blockIdx.x * (long long)blockDim.x + threadIdx.x; v < vecs; v += (long long)gridDim.x * blockDim.x) {
+    const int n = (int)(v & 255);
+    const int c = (int)((v >> 8) & 7);
+    const long long rec = v >> 11;  // T * KB + kb
+    const int kb = (int)(rec % KB);
+    const long long T = rec / KB;
+    uint8_t* canon = q8 + ((size_t)kb * 128 + 16 * c) * N + T * 256 + n;
+    uint8_t* packed = wq + v * 16;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      if (inverse)
+        canon[(size_t)j * N] = packed[j];
+      else
+        packed[j] = canon[(size_t)j * N];
+    }
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_pack_w8(uint8_t* q8, uint8_t* wq, int K, int N, bool inverse, cudaStream_t stream) {
+  const long long vecs = (long long)K * N / 16;
+  const int threads = 256;
+  int blocks = (int)((vecs + threads - 1) / threads);
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  pack_w8_kernel<<<blocks, threads, 0, stream>>>(q8, wq, K, N, inverse);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_interleave_gate_up(const uint32_t* q_gate, const uint16_t* s_gate, const uint32_t* q_up, const uint16_t* s_up,
                                       uint32_t* q_out, uint16_t* s_out, int K, int I, int G, cudaStream_t stream) {

@@ -15,15 +15,20 @@ def weight_bits_w4(G: int) -> float:
     return 4.0 + 16.0 / G
 
 
-def weight_bytes(K: int, N: int, G: int, sparse24: bool = False) -> int:
+def weight_bytes(K: int, N: int, G: int, sparse24: bool = False, bits: int = 4) -> int:
     scales = 2 * (K // G) * N
+    if bits == 8:
+        return K * N + scales
     if sparse24:
         return K * N // 4 + K * N // 8 + scales
     return K * N // 2 + scales
 
 
-def algorithmic_bytes(M: int, K: int, N: int, G: int, scales: bool = True, sparse24: bool = False) -> int:
-    w = weight_bytes(K, N, G, sparse24) if scales else (K * N // 4 + K * N // 8 if sparse24 else K * N // 2)
+def algorithmic_bytes(M: int, K: int, N: int, G: int, scales: bool = True, sparse24: bool = False, bits: int = 4) -> int:
+    if bits == 8:
+        w = weight_bytes(K, N, G, bits=8) if scales else K * N
+    else:
+        w = weight_bytes(K, N, G, sparse24) if scales else (K * N // 4 + K * N // 8 if sparse24 else K * N // 2)
     return w + 2 * M * K + 2 * M * N
 
 
@@ -47,8 +52,8 @@ def load_peaks(root: str):
         return dict(FALLBACK_PEAKS, source="fallback")
 
 
-def roofline_seconds(M: int, K: int, N: int, G: int, peaks, sparse24: bool = False) -> float:
-    t_mem = algorithmic_bytes(M, K, N, G, sparse24=sparse24) / (peaks["hbm_gbs"] * 1e9)
+def roofline_seconds(M: int, K: int, N: int, G: int, peaks, sparse24: bool = False, bits: int = 4) -> float:
+    t_mem = algorithmic_bytes(M, K, N, G, sparse24=sparse24, bits=bits) / (peaks["hbm_gbs"] * 1e9)
     executed = flops(M, K, N) / (2 if sparse24 else 1)
     t_flop = executed / (peaks["bf16_tflops"] * 1e12)
     return max(t_mem, t_flop)
