@@ -820,7 +820,19 @@ cudaError_t launch_gemm_dense_tc(GemmParams p, int sm_count, bool sparse24, cuda
     if (S > (long long)p.kb) S = p.kb;
     if (S > 8) S = 8;  // the CTAs of a tile form a thread-block cluster: at most the portable size
     const char* e = getenv("MARLIN_B200_TC_SPLIT");  // tuning knob: 0 forces even stripes
-    if (S >= 2 && S * p.ncols * 100 >= workers * 85 && !(e && atoi(e) == 0)) {
+    // Clusters of eight do not all fit on the device at once, so eight k-ranges per tile go through the L2, which
+    // above 64 rows costs about 5 us more than the exchange inside clusters of four: on short layers four longer
+    // k-ranges win (measured: 13.4 against 15.9 us on 4096 x 4096 at 128 rows; from about 56 k-blocks up eight win).
+    bool chosen = false;
+    if (S == 8 && p.M > 64 && p.kb <= 56 && 4 * p.ncols * 100 >= workers * 40) {
+      S = 4;
+      chosen = true;
+    }
+    if (e && atoi(e) >= 2 && atoi(e) <= 8 && atoi(e) <= workers / p.ncols) {  // tuning knob: 2..8 k-ranges per tile
+      S = atoi(e);
+      chosen = true;
+    }
+    if (S >= 2 && (S * p.ncols * 100 >= workers * 85 || chosen) && !(e && atoi(e) == 0)) {
       p.split = (uint32_t)S;
       workers = S * p.ncols;
     }
