@@ -112,7 +112,7 @@ MARLIN_API int marlin_unpack(const void* w_packed, const void* s_packed, uint32_
  * activation-aware format the paper names in Section 6).  Codes and scales go through marlin_pack as usual.
  *   zeros      device, uint8 [K/G][N] row-major, values 0..15
  *   z_packed   device, out, marlin_packed_scale_bytes(K, N, G) bytes (fp16 values in the order of the packed scales)
- * Layers with zero points need N % 256 == 0 (they run on the tcgen05 kernel at every batch size). */
+ * Shapes and group sizes as for marlin_pack. */
 MARLIN_API int marlin_pack_zeros(const uint8_t* zeros, void* z_packed, int K, int N, int group_size, marlin_stream stream);
 MARLIN_API int marlin_unpack_zeros(const void* z_packed, uint8_t* zeros, int K, int N, int group_size, marlin_stream stream);
 
@@ -186,10 +186,12 @@ MARLIN_API int marlin_gemm_w8(const void* A, const void* w_packed, const void* s
                    int group_size, void* workspace, size_t workspace_bytes, marlin_stream stream);
 
 /* The layer with zero points: C = A . W, W[k][n] = (q[k][n] - z[k/G][n]) * s[k/G][n].  Arguments as marlin_gemm, plus
- * z_packed from marlin_pack_zeros.  N % 256 == 0 (else MARLIN_ERR_SHAPE); every batch size runs on the tcgen05
- * kernel, where the zero point replaces the constant 8 inside the conversion (the subtrahend of the exponent
- * trick of Section 3.4 "Dequantization and Tensor Cores" becomes 1024 + z): no extra instruction per weight.
- * workspace: marlin_workspace_bytes(M, K, N). */
+ * z_packed from marlin_pack_zeros.  Up to 16 rows (and in slabs of 16 rows where N is not a multiple of 256) the
+ * warp-level kernel runs: the weights enter the MMAs as for the symmetric layer and one more MMA per 16 rows of k,
+ * with an all-ones weight operand, gives sum_k a[k][m] per group, so that the group closes with
+ * s * (sum_k a (q - 8) + (8 - z) sum_k a).  Above, the tcgen05 kernel, where the zero point replaces the constant 8
+ * inside the conversion (the subtrahend of the exponent trick of Section 3.4 "Dequantization and Tensor Cores"
+ * becomes 1024 + z): no extra instruction per weight.  workspace: marlin_workspace_bytes(M, K, N). */
 MARLIN_API int marlin_gemm_zp(const void* A, const void* w_packed, const void* s_packed, const void* z_packed, void* C,
                    int M, int K, int N, int group_size, void* workspace, size_t workspace_bytes,
                    marlin_stream stream);

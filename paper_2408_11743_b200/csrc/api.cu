@@ -170,7 +170,7 @@ int marlin_quantize_rtn(const void* W, uint32_t* q_kpacked, void* scales, int K,
 
 int marlin_pack_zeros(const uint8_t* zeros, void* z_packed, int K, int N, int group_size, marlin_stream stream) {
   if (!zeros || !z_packed) return MARLIN_ERR_NULL;
-  if (!shape_ok(K, N) || N % 256) return MARLIN_ERR_SHAPE;
+  if (!shape_ok(K, N)) return MARLIN_ERR_SHAPE;
   int G = normalise_group(K, N, group_size);
   if (!G) return MARLIN_ERR_GROUP;
   if (!aligned16(zeros) || !aligned16(z_packed)) return MARLIN_ERR_ALIGN;
@@ -181,7 +181,7 @@ int marlin_pack_zeros(const uint8_t* zeros, void* z_packed, int K, int N, int gr
 
 int marlin_unpack_zeros(const void* z_packed, uint8_t* zeros, int K, int N, int group_size, marlin_stream stream) {
   if (!zeros || !z_packed) return MARLIN_ERR_NULL;
-  if (!shape_ok(K, N) || N % 256) return MARLIN_ERR_SHAPE;
+  if (!shape_ok(K, N)) return MARLIN_ERR_SHAPE;
   int G = normalise_group(K, N, group_size);
   if (!G) return MARLIN_ERR_GROUP;
   if (!aligned16(zeros) || !aligned16(z_packed)) return MARLIN_ERR_ALIGN;
@@ -210,9 +210,10 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
                        int K, int N, int group_size, void* workspace, size_t workspace_bytes, marlin_stream stream,
                        bool sparse24, const void* z_packed = nullptr, bool swiglu = false, bool w8 = false) {
   if (!A || !w_packed || !s_packed || !C || !workspace || (sparse24 && !meta_packed)) return MARLIN_ERR_NULL;
-  // layers with zero points run on the tcgen05 kernel alone (N a multiple of 256), at every batch size
+  // layers with zero points: the warp-level kernel up to 16 rows (and in slabs where N is not a multiple of 256), the
+  // tcgen05 kernel above
   const bool zero_points = z_packed != nullptr;
-  if (zero_points && (N % 256 || !aligned16(z_packed))) return N % 256 ? MARLIN_ERR_SHAPE : MARLIN_ERR_ALIGN;
+  if (zero_points && !aligned16(z_packed)) return MARLIN_ERR_ALIGN;
   if (w8 && N % 256) return MARLIN_ERR_SHAPE;  // 8-bit codes: the tcgen05 kernel alone, at every batch size
   if (M < 1 || !shape_ok(K, N)) return MARLIN_ERR_SHAPE;
   int G = normalise_group(K, N, group_size);
@@ -239,9 +240,9 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
     // it takes every batch size there
     const bool tc_ok = tc_path_supported(1, K, N);
     // groups of 64 or 32 rows likewise (accepted only where N is a multiple of 256)
-    const bool small_groups = G < kTileK || zero_points || w8;
+    const bool small_groups = G < kTileK || w8;
     // (the kernel with deferred scales has no fused activation: those layers go through the warp-level kernel then)
-    const bool use_tcd = !swiglu && !sparse24 && !small_groups && tcd_path_supported(1, K, N) &&
+    const bool use_tcd = !swiglu && !sparse24 && !small_groups && !zero_points && tcd_path_supported(1, K, N) &&
                          (tmode == 1 || (tmode == 2 && rem >= tc_min_m() && !tc_ok));
     const bool use_tc = !use_tcd && tc_ok && (sparse24 || small_groups || rem >= tc_min_m());
     const int m_slab = use_tcd ? (rem < kTcdMaxSlabM ? rem : kTcdMaxSlabM)
@@ -282,14 +283,15 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
         return MARLIN_ERR_CUDA;
     } else {
       DensePlan plan;
-      if (!make_dense_plan(m_slab, K, N, info.sm_count, sparse24, &plan)) return MARLIN_ERR_SHAPE;
+      const int fmt = sparse24 ? 1 : (zero_points ? 2 : 0);
+      if (!make_dense_plan(m_slab, K, N, info.sm_count, fmt, &plan)) return MARLIN_ERR_SHAPE;
       p.ncols = plan.ncols;
       p.units = (uint32_t)plan.units;
       p.workers = (uint32_t)plan.workers;
       p.split = (uint32_t)plan.split;
       p.stages = plan.stages;
       p.stage_bytes = plan.stage_bytes;
-      if (launch_gemm_dense(plan, p, sparse24, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MARLIN_ERR_CUDA;
+      if (launch_gemm_dense(plan, p, fmt, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MARLIN_ERR_CUDA;
     }
     m0 += m_slab;
   }

@@ -58,8 +58,13 @@ constexpr int kBarBytes = 1024;  // full[32] at 0, empty[32] at 256, flags at 51
 // tcgen05 kernel, or through this one as slabs of 16 rows where that kernel does not apply.
 constexpr int consumer_warps_for(int /*mb*/) { return 8; }
 
-template <int MB, int NW, int CW, bool SP>
+// FMT: 0 = dense, 1 = the 2:4 variant, 2 = dense with per-group zero points (W = (q - z) s: the zero-point row of a
+// group travels with the stage behind its scale row)
+constexpr int kFmtDense = 0, kFmtSparse = 1, kFmtZero = 2;
+template <int MB, int NW, int CW, int FMT>
 struct Geometry {
+  static constexpr bool SP = FMT == kFmtSparse;
+  static constexpr bool ZP = FMT == kFmtZero;
   static constexpr int SK = CW / NW;             // groups of warps that split K
   static constexpr int MPAD = MB * 8;
   static constexpr int NT = NW * kChunkN;
@@ -75,7 +80,8 @@ struct Geometry {
   static constexpr int RED_BYTES = (SK - 1) * TILE_F4 * 16;  // parked tiles of groups 1 .. SK - 1
   static constexpr int CST_STRIDE = NT + 8;                  // halves
   static constexpr int CST_BYTES = MPAD * CST_STRIDE * 2;
-  static constexpr int SC_BYTES = NT * 2;                    // group scales of one stage (one row of the tile)
+  static constexpr int SC_ROW_BYTES = NT * 2;                // one row of the tile's group scales (or zero points)
+  static constexpr int SC_BYTES = (ZP ? 2 : 1) * SC_ROW_BYTES;  // per stage: the scale row, then the zero-point row
   static constexpr int SC_OFF = kBarBytes + RED_BYTES + CST_BYTES;
   static constexpr int ALIGN_SLACK = 1024;                   // the stage ring is placed on a 1024-byte boundary
   // stages: what fits after the fixed areas, each stage bringing its scale row along
@@ -96,10 +102,12 @@ struct Geometry {
 // ---------------------------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------------------------
-template <int MB, int NW, int CW, bool SP>
+template <int MB, int NW, int CW, int FMT>
 __global__ void __launch_bounds__((CW + 4) * 32, 1)
 gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a) {
-  using G = Geometry<MB, NW, CW, SP>;
+  using G = Geometry<MB, NW, CW, FMT>;
+  constexpr bool SP = G::SP;
+  constexpr bool ZP = G::ZP;
   constexpr int SK = G::SK;
   constexpr int kConsumerWarps = CW;
   constexpr int kConsumerThreads = CW * 32;
@@ -155,7 +163,7 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
     const uint64_t pol_w = policy_evict_first();
     const uint64_t pol_a = policy_evict_last();
     // out-of-range rows of the A box count too; grouped layers bring the scale row of the k-block along
-    const uint32_t tx_bytes = G::W_BYTES + G::META_BYTES + G::A_BYTES + (p.grouped ? G::SC_BYTES : 0);
+    const uint32_t tx_bytes = G::W_BYTES + G::META_BYTES + G::A_BYTES + (p.grouped ? G::SC_BYTES : 0);  // ZP layers are grouped
     auto scale_src = [&](uint32_t col, uint32_t kb) -> const uint8_t* {
       const uint32_t gi = p.group_shift >= 0 ? (kb >> p.group_shift) : (kb / (uint32_t)p.kb_per_group);
       return p.sq + ((size_t)gi * p.N + (size_t)col * G::NT) * 2;
@@ -192,7 +200,10 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
         if constexpr (SP)
           bulk_g2s(stage0 + (size_t)s * G::STAGE_BYTES + G::A_BYTES + G::W_BYTES, meta_src(col, kb), G::META_BYTES,
                    &full[s], pol_w);
-        if (p.grouped) bulk_g2s(sc_ring + (size_t)s * G::SC_BYTES, scale_src(col, kb), G::SC_BYTES, &full[s], pol_w);
+        if (p.grouped) bulk_g2s(sc_ring + (size_t)s * G::SC_BYTES, scale_src(col, kb), G::SC_ROW_BYTES, &full[s], pol_w);
+        if constexpr (ZP)
+          bulk_g2s(sc_ring + (size_t)s * G::SC_BYTES + G::SC_ROW_BYTES, p.zq + (scale_src(col, kb) - p.sq), G::SC_ROW_BYTES,
+                   &full[s], pol_w);
       }
     }
     __syncwarp();
@@ -218,7 +229,10 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
         mbar_expect_tx(&full[s], tx_bytes);
         bulk_g2s(st + G::A_BYTES, wsrc, G::W_BYTES, &full[s], pol_w);
         if constexpr (SP) bulk_g2s(st + G::A_BYTES + G::W_BYTES, meta_src(col, kb), G::META_BYTES, &full[s], pol_w);
-        if (p.grouped) bulk_g2s(sc_ring + (size_t)s * G::SC_BYTES, scale_src(col, kb), G::SC_BYTES, &full[s], pol_w);
+        if (p.grouped) bulk_g2s(sc_ring + (size_t)s * G::SC_BYTES, scale_src(col, kb), G::SC_ROW_BYTES, &full[s], pol_w);
+        if constexpr (ZP)
+          bulk_g2s(sc_ring + (size_t)s * G::SC_BYTES + G::SC_ROW_BYTES, p.zq + (scale_src(col, kb) - p.sq), G::SC_ROW_BYTES,
+                   &full[s], pol_w);
       }
       __syncwarp();
       if (lane < 2) tma_load_2d(st + lane * G::A_HALF_BYTES, &tmap_a, (int)(kb * kTileK + lane * 64), 0, &full[s], pol_a);
@@ -262,15 +276,28 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
   constexpr bool kBiased = !SP && MB == 1;
   float bias[kBiased ? MB : 1][4];
   uint4 cur_raw = make_uint4(0, 0, 0, 0);  // 8 fp16 scales of the open group: columns 16j+g and 16j+8+g, j = 0..3
+  // Zero points: sum_k a (q - z) = sum_k a (q - 8) + (8 - z) sum_k a.  asum[mb] collects sum_k a[k][m] of the open group
+  // with one more MMA per 16 rows of k whose weight operand is all ones (the same number in every output channel),
+  // and the group closes with acc += s (tmp + (8 - z) asum).
+  uint4 cur_z = make_uint4(0, 0, 0, 0);    // the 8 zero points of the open group, as fp16 values, same order
+  float asum[ZP ? MB : 1][4];
 
   auto close_group = [&]() {
     const __half2* h2 = reinterpret_cast<const __half2*>(&cur_raw);
+    const __half2* z2 = reinterpret_cast<const __half2*>(&cur_z);
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const float2 sc2 = __half22float2(h2[j]);
 #pragma unroll
       for (int mb = 0; mb < MB; ++mb) {
         const int r = j * MB + mb;
+        if constexpr (ZP) {
+          const float2 zf = __half22float2(z2[j]);
+          tmp[r][0] += (8.f - zf.x) * asum[mb][0];
+          tmp[r][1] += (8.f - zf.x) * asum[mb][1];
+          tmp[r][2] += (8.f - zf.y) * asum[mb][2];
+          tmp[r][3] += (8.f - zf.y) * asum[mb][3];
+        }
         if constexpr (!kBiased) {
           acc[r][0] += sc2.x * tmp[r][0];
           acc[r][1] += sc2.x * tmp[r][1];
@@ -288,6 +315,10 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
     if constexpr (kBiased) {
 #pragma unroll
       for (int mb = 0; mb < MB; ++mb) bias[mb][0] = bias[mb][1] = bias[mb][2] = bias[mb][3] = 0.f;
+    }
+    if constexpr (ZP) {
+#pragma unroll
+      for (int mb = 0; mb < MB; ++mb) asum[mb][0] = asum[mb][1] = asum[mb][2] = asum[mb][3] = 0.f;
     }
   };
 
@@ -330,6 +361,10 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
 #pragma unroll
       for (int mb = 0; mb < MB; ++mb) bias[mb][0] = bias[mb][1] = bias[mb][2] = bias[mb][3] = 0.f;
     }
+    if constexpr (ZP) {
+#pragma unroll
+      for (int mb = 0; mb < MB; ++mb) asum[mb][0] = asum[mb][1] = asum[mb][2] = asum[mb][3] = 0.f;
+    }
     int cur_group = -1;
     if (!p.grouped) cur_raw = __ldg(reinterpret_cast<const uint4*>(srow));
 
@@ -339,12 +374,17 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
       const uint32_t kb = kb0 + x;
       mbar_wait(&full[s], ph, abort_flag, p.status);
       if (p.grouped) {
-        const int gi = p.group_shift >= 0 ? (int)(kb >> p.group_shift) : (int)(kb / (uint32_t)p.kb_per_group);
+        int gi = p.group_shift >= 0 ? (int)(kb >> p.group_shift) : (int)(kb / (uint32_t)p.kb_per_group);
+        // with zero points also a long group (one scale per column) is folded into `acc` every 1024 rows of k, so
+        // that the offsets carried in `tmp` never cost more than a few of its low bits
+        if constexpr (ZP) gi = (gi << 12) | (int)(kb >> 3);
         if (gi != cur_group) {
           if (cur_group >= 0) close_group();
           // the group's scales came with the stage (a read from global memory here would be a cold DRAM
           // access whose latency every warp would wait out once per stage)
           cur_raw = lds128(smem_u32(sc_ring) + (uint32_t)s * G::SC_BYTES + (uint32_t)(wn * 64 + g * 8) * 2);
+          if constexpr (ZP)
+            cur_z = lds128(smem_u32(sc_ring) + (uint32_t)s * G::SC_BYTES + G::SC_ROW_BYTES + (uint32_t)(wn * 64 + g * 8) * 2);
           cur_group = gi;
         }
       } else {
@@ -454,6 +494,14 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
             for (int mb = 0; mb < MB; ++mb) {
               mma_16816(bias[mb], kc, bf[mb][4 * u], bf[mb][4 * u + 1]);
               mma_16816(bias[mb], kc, bf[mb][4 * u + 2], bf[mb][4 * u + 3]);
+            }
+          }
+          if constexpr (ZP) {
+            const uint32_t ones[4] = {0x3c003c00u, 0x3c003c00u, 0x3c003c00u, 0x3c003c00u};
+#pragma unroll
+            for (int mb = 0; mb < MB; ++mb) {
+              mma_16816(asum[mb], ones, bf[mb][4 * u], bf[mb][4 * u + 1]);
+              mma_16816(asum[mb], ones, bf[mb][4 * u + 2], bf[mb][4 * u + 3]);
             }
           }
         }
@@ -732,11 +780,11 @@ bool make_a_tensor_map_3d(CUtensorMap* map, const void* A, int M, int K, int box
 
 namespace {
 
-template <int MB, int NW, bool SP>
+template <int MB, int NW, int FMT>
 cudaError_t launch_one(const DensePlan& plan, const GemmParams& p, cudaStream_t stream) {
   constexpr int CW = consumer_warps_for(MB);
-  constexpr size_t G_TILE_BYTES = (size_t)Geometry<MB, NW, CW, SP>::TILE_F4 * 16;
-  auto kernel = gemm_dense_kernel<MB, NW, CW, SP>;
+  constexpr size_t G_TILE_BYTES = (size_t)Geometry<MB, NW, CW, FMT>::TILE_F4 * 16;
+  auto kernel = gemm_dense_kernel<MB, NW, CW, FMT>;
   static bool attr_set[64] = {};  // per device
   int dev = 0;
   cudaError_t err = cudaGetDevice(&dev);
@@ -784,9 +832,9 @@ cudaError_t launch_one(const DensePlan& plan, const GemmParams& p, cudaStream_t 
   return cudaLaunchKernelEx(&cfg, kernel, q, tmap);
 }
 
-template <int MB, int NW, bool SP>
+template <int MB, int NW, int FMT>
 void fill_geometry(DensePlan* plan) {
-  using G = Geometry<MB, NW, consumer_warps_for(MB), SP>;
+  using G = Geometry<MB, NW, consumer_warps_for(MB), FMT>;
   plan->stage_bytes = G::STAGE_BYTES;
   int stages = G::STAGES;
   if (const char* e = getenv("MARLIN_B200_STAGES")) { int v = atoi(e); if (v >= 2 && v < stages) stages = v; }
@@ -810,7 +858,7 @@ void fill_geometry(DensePlan* plan) {
 #define MARLIN_DISPATCH(MBV, NWV, STMT)         \
   if (plan_mb == MBV && plan_nw == NWV) { STMT; }
 
-bool make_dense_plan(int m_slab, int K, int N, int sm_count, bool sparse24, DensePlan* plan) {
+bool make_dense_plan(int m_slab, int K, int N, int sm_count, int fmt, DensePlan* plan) {
   if (m_slab < 1 || m_slab > kMaxSlabM || K < kTileK || K % kTileK || N < kChunkN || N % kChunkN) return false;
   if (sm_count < 1) return false;
   int mb = m_slab <= 8 ? 1 : 2;
@@ -855,23 +903,23 @@ bool make_dense_plan(int m_slab, int K, int N, int sm_count, bool sparse24, Dens
   if (workers > plan->units) workers = plan->units;
   plan->workers = (int)workers;
   const int plan_mb = mb, plan_nw = nw;
-  MARLIN_DISPATCH(1, 1, (sparse24 ? fill_geometry<1, 1, true>(plan) : fill_geometry<1, 1, false>(plan)))
-  MARLIN_DISPATCH(1, 2, (sparse24 ? fill_geometry<1, 2, true>(plan) : fill_geometry<1, 2, false>(plan)))
-  MARLIN_DISPATCH(1, 4, (sparse24 ? fill_geometry<1, 4, true>(plan) : fill_geometry<1, 4, false>(plan)))
-  MARLIN_DISPATCH(2, 1, (sparse24 ? fill_geometry<2, 1, true>(plan) : fill_geometry<2, 1, false>(plan)))
-  MARLIN_DISPATCH(2, 2, (sparse24 ? fill_geometry<2, 2, true>(plan) : fill_geometry<2, 2, false>(plan)))
-  MARLIN_DISPATCH(2, 4, (sparse24 ? fill_geometry<2, 4, true>(plan) : fill_geometry<2, 4, false>(plan)))
+  MARLIN_DISPATCH(1, 1, (fmt == 1 ? fill_geometry<1, 1, 1>(plan) : fmt == 2 ? fill_geometry<1, 1, 2>(plan) : fill_geometry<1, 1, 0>(plan)))
+  MARLIN_DISPATCH(1, 2, (fmt == 1 ? fill_geometry<1, 2, 1>(plan) : fmt == 2 ? fill_geometry<1, 2, 2>(plan) : fill_geometry<1, 2, 0>(plan)))
+  MARLIN_DISPATCH(1, 4, (fmt == 1 ? fill_geometry<1, 4, 1>(plan) : fmt == 2 ? fill_geometry<1, 4, 2>(plan) : fill_geometry<1, 4, 0>(plan)))
+  MARLIN_DISPATCH(2, 1, (fmt == 1 ? fill_geometry<2, 1, 1>(plan) : fmt == 2 ? fill_geometry<2, 1, 2>(plan) : fill_geometry<2, 1, 0>(plan)))
+  MARLIN_DISPATCH(2, 2, (fmt == 1 ? fill_geometry<2, 2, 1>(plan) : fmt == 2 ? fill_geometry<2, 2, 2>(plan) : fill_geometry<2, 2, 0>(plan)))
+  MARLIN_DISPATCH(2, 4, (fmt == 1 ? fill_geometry<2, 4, 1>(plan) : fmt == 2 ? fill_geometry<2, 4, 2>(plan) : fill_geometry<2, 4, 0>(plan)))
   return plan->stages >= consumer_warps_for(mb) / nw && plan->stages >= kProducerWarps;
 }
 
-cudaError_t launch_gemm_dense(const DensePlan& plan, const GemmParams& p, bool sparse24, cudaStream_t stream) {
+cudaError_t launch_gemm_dense(const DensePlan& plan, const GemmParams& p, int fmt, cudaStream_t stream) {
   const int plan_mb = plan.mb, plan_nw = plan.nw;
-  MARLIN_DISPATCH(1, 1, return (sparse24 ? launch_one<1, 1, true>(plan, p, stream) : launch_one<1, 1, false>(plan, p, stream)))
-  MARLIN_DISPATCH(1, 2, return (sparse24 ? launch_one<1, 2, true>(plan, p, stream) : launch_one<1, 2, false>(plan, p, stream)))
-  MARLIN_DISPATCH(1, 4, return (sparse24 ? launch_one<1, 4, true>(plan, p, stream) : launch_one<1, 4, false>(plan, p, stream)))
-  MARLIN_DISPATCH(2, 1, return (sparse24 ? launch_one<2, 1, true>(plan, p, stream) : launch_one<2, 1, false>(plan, p, stream)))
-  MARLIN_DISPATCH(2, 2, return (sparse24 ? launch_one<2, 2, true>(plan, p, stream) : launch_one<2, 2, false>(plan, p, stream)))
-  MARLIN_DISPATCH(2, 4, return (sparse24 ? launch_one<2, 4, true>(plan, p, stream) : launch_one<2, 4, false>(plan, p, stream)))
+  MARLIN_DISPATCH(1, 1, return (fmt == 1 ? launch_one<1, 1, 1>(plan, p, stream) : fmt == 2 ? launch_one<1, 1, 2>(plan, p, stream) : launch_one<1, 1, 0>(plan, p, stream)))
+  MARLIN_DISPATCH(1, 2, return (fmt == 1 ? launch_one<1, 2, 1>(plan, p, stream) : fmt == 2 ? launch_one<1, 2, 2>(plan, p, stream) : launch_one<1, 2, 0>(plan, p, stream)))
+  MARLIN_DISPATCH(1, 4, return (fmt == 1 ? launch_one<1, 4, 1>(plan, p, stream) : fmt == 2 ? launch_one<1, 4, 2>(plan, p, stream) : launch_one<1, 4, 0>(plan, p, stream)))
+  MARLIN_DISPATCH(2, 1, return (fmt == 1 ? launch_one<2, 1, 1>(plan, p, stream) : fmt == 2 ? launch_one<2, 1, 2>(plan, p, stream) : launch_one<2, 1, 0>(plan, p, stream)))
+  MARLIN_DISPATCH(2, 2, return (fmt == 1 ? launch_one<2, 2, 1>(plan, p, stream) : fmt == 2 ? launch_one<2, 2, 2>(plan, p, stream) : launch_one<2, 2, 0>(plan, p, stream)))
+  MARLIN_DISPATCH(2, 4, return (fmt == 1 ? launch_one<2, 4, 1>(plan, p, stream) : fmt == 2 ? launch_one<2, 4, 2>(plan, p, stream) : launch_one<2, 4, 0>(plan, p, stream)))
   return cudaErrorInvalidValue;
 }
 

@@ -52,7 +52,8 @@ struct DensePlan {
 
 // Chooses tile width, worker count and pipeline depth for one slab of m_slab <= 32 rows.
 // Pure host arithmetic.  Returns false on an unsupported shape.
-bool make_dense_plan(int m_slab, int K, int N, int sm_count, bool sparse24, DensePlan* plan);
+// fmt: 0 dense, 1 the 2:4 variant, 2 dense with zero points (the stage then carries a zero-point row)
+bool make_dense_plan(int m_slab, int K, int N, int sm_count, int fmt, DensePlan* plan);
 
 struct GemmParams {
   const uint16_t* A;
@@ -87,7 +88,7 @@ struct GemmParams {
                      // k-ranges and worker w owns range w % S of tile w / S (one segment per CTA)
 };
 
-cudaError_t launch_gemm_dense(const DensePlan& plan, const GemmParams& p, bool sparse24, cudaStream_t stream);
+cudaError_t launch_gemm_dense(const DensePlan& plan, const GemmParams& p, int fmt, cudaStream_t stream);
 cudaError_t launch_pack_sparse24(uint32_t* qc, uint8_t* idx, uint16_t* s, uint32_t* wq, uint32_t* meta, uint16_t* sq, int K,
                                  int N, int G, bool inverse, cudaStream_t stream);
 
