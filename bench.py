@@ -49,7 +49,7 @@ K_DIM, N_DIM, GROUP = 8192, 8192, 128
 SWEEP = (1, 2, 4, 8, 16, 32, 64, 128)
 METRIC = "w4a16_gemm_weight_stream_rate_batch_sweep_M1-128_K8192_N8192_g128"
 UNIT = "GB/s"
-CPU_SAMPLE_MS = (16, 64)      # cpu_baseline leg of the GPU arm
+CPU_SAMPLE_MS = (1, 2, 4, 8, 16, 32, 64, 128)  # cpu_baseline leg of the GPU arm: one whole step (about 25 core-seconds)
 REFERENCE_SAMPLE_MS = (16,)   # one step of --impl reference
 
 
@@ -707,7 +707,7 @@ def run_ours(args):
             "per_m": per_m,
             "other_layers": extra,
             "cpu_baseline": {"value": round(cpu_v, 4), "unit": UNIT, "cores": cores, "kind": "oracle",
-                             "sample": f"full layer at M in {list(CPU_SAMPLE_MS)} ({cpu_t:.1f} s)"},
+                             "sample": f"one whole step: the full layer at M in {list(CPU_SAMPLE_MS)} ({cpu_t:.1f} s on {cores} threads)"},
             "e2e": {"value": round(world * step_wbytes / e2e_s / 1e9, 2), "unit": UNIT,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_s * 1e3, 5)},
             "gpu_launches": launches_per_step * args.steps,
