@@ -813,19 +813,20 @@ cudaError_t launch_one(const DensePlan& plan, const GemmParams& p, cudaStream_t 
   if (S >= 2 && S <= 8 && (size_t)(S - 1) * G_TILE_BYTES <= (size_t)plan.stages * plan.stage_bytes && !(e && atoi(e) == 0)) {
     // the S CTAs of a column tile as one thread-block cluster, if all clusters of the grid fit on the device
     // at once (a GPC holds only so many clusters of a size; a second wave would cost more than it saves)
-    static int cluster_ok[64][9] = {};  // per device and cluster size: 0 unknown, 1 yes, -1 no
-    int ok = (dev >= 0 && dev < 64) ? cluster_ok[dev][S] : 0;
+    static int max_clusters[64][9] = {};  // per device and cluster size: clusters resident at once (0 unknown, -1 none)
+    int nmax = (dev >= 0 && dev < 64) ? max_clusters[dev][S] : 0;
     attr[1].id = cudaLaunchAttributeClusterDimension;
     attr[1].val.clusterDim.x = (unsigned)S;
     attr[1].val.clusterDim.y = 1;
     attr[1].val.clusterDim.z = 1;
-    if (ok == 0) {
+    if (nmax == 0) {
       cfg.numAttrs = 2;
       int n = 0;
-      ok = (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) == cudaSuccess && n * S >= plan.workers) ? 1 : -1;
+      nmax = (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) == cudaSuccess && n > 0) ? n : -1;
       (void)cudaGetLastError();
-      if (dev >= 0 && dev < 64) cluster_ok[dev][S] = ok;
+      if (dev >= 0 && dev < 64) max_clusters[dev][S] = nmax;
     }
+    const int ok = (nmax > 0 && (long long)nmax * S >= plan.workers) ? 1 : -1;  // all clusters of THIS grid at once
     cfg.numAttrs = ok > 0 ? 2 : 1;
     q.cluster = ok > 0 ? 1u : 0u;
   }

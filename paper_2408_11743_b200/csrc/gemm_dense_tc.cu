@@ -412,9 +412,6 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         v[1] = lds128(wbase + 256 * 16);             // kept values 32..63
         v[2] = lds128(wbase + (uint32_t)G::W_BYTES); // the four metadata words of this tensor-memory lane
       }
-      // the codes are in registers: the weight part of the stage is free as far as this warp is concerned
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&empty[s]);
 
       if (it >= (uint32_t)NSLOTS) {
         // the slot was last read by the MMAs of stage it - NSLOTS
@@ -484,6 +481,12 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         const uint32_t mw[4] = {v[2].x, v[2].y, v[2].z, v[2].w};
         tc_st_x4(slot_col + (uint32_t)(64 + tile * 4), mw);
       }
+      // The codes have been converted, so the shared loads that fetched them have certainly delivered: only now is
+      // the weight part of the stage released.  (An arrival issued right behind the loads can be performed before a
+      // multi-wavefront shared load has read its data: with a weight ring refilled without waiting for the MMAs, a
+      // refill that followed at once overwrote codes still being read.)
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&empty[s]);
       tc_wait_st();
       tc_fence_before_sync();
       __syncwarp();
@@ -754,20 +757,21 @@ cudaError_t launch_tc(const GemmParams& p, int workers, cudaStream_t stream) {
     // the S CTAs of a column tile as one thread-block cluster, if this device can co-schedule such a cluster
     // (all of them at once: a GPC holds only so many clusters of a size, and a second wave would cost far
     // more than the reduction through the L2 that is the alternative)
-    static int cluster_ok[64][9] = {};  // per device and cluster size: 0 unknown, 1 yes, -1 no
+    static int max_clusters[64][9] = {};  // per device and cluster size: clusters resident at once (0 unknown, -1 none)
     const int S = (int)p.split;
-    int ok = (dev >= 0 && dev < 64) ? cluster_ok[dev][S] : 0;
+    int nmax = (dev >= 0 && dev < 64) ? max_clusters[dev][S] : 0;
     attr[1].id = cudaLaunchAttributeClusterDimension;
     attr[1].val.clusterDim.x = (unsigned)S;
     attr[1].val.clusterDim.y = 1;
     attr[1].val.clusterDim.z = 1;
-    if (ok == 0) {
+    if (nmax == 0) {
       cfg.numAttrs = 2;
       int n = 0;
-      ok = (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) == cudaSuccess && n * S >= workers) ? 1 : -1;
+      nmax = (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) == cudaSuccess && n > 0) ? n : -1;
       (void)cudaGetLastError();
-      if (dev >= 0 && dev < 64) cluster_ok[dev][S] = ok;
+      if (dev >= 0 && dev < 64) max_clusters[dev][S] = nmax;
     }
+    const int ok = (nmax > 0 && (long long)nmax * S >= workers) ? 1 : -1;  // all clusters of THIS grid at once
     cfg.numAttrs = ok > 0 ? 2 : 1;
     q.cluster = ok > 0 ? 1u : 0u;
   }

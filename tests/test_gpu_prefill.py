@@ -85,7 +85,9 @@ def test_smaller_batches_reuse_a_large_workspace(marlin, oracle_lib):
         C = layer(case.A[:M])
         bad, worst, _ = oracle_lib.check_tolerance(C, np.ascontiguousarray(C_ref[:M]))
         assert bad == 0, (M, worst)
-        assert np.all(to_host(layer.ws)[256:] == 0)
+        ws = to_host(layer.ws)
+        assert np.all(ws[256:8192] == 0)            # arrival counters
+        assert np.all(ws[-N * 128 * 4:] == 0)       # accumulation tiles of the tcgen05 kernel (at the end of the buffer)
 
 
 @pytest.mark.parametrize("M,K,N,G", [(200, 1024, 512, 128), (513, 2048, 256, -1)])
