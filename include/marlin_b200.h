@@ -67,11 +67,13 @@ MARLIN_API size_t marlin_packed_scale_bytes(int K, int N, int group_size);
 MARLIN_API size_t marlin_packed_meta_bytes(int K, int N);
 /* Bytes of the workspace marlin_gemm* needs for any M <= max_M on this K x N layer.
  * The workspace holds a status word, per-column-tile arrival counters and the fp32 partial tiles
- * of the stripe fix-up (the global reduction of Section 3.4 "Striped Partitioning"); it grows with max_M up
- * to 128 rows and, above, with the number of (column tile, 128-row slab) pairs up to the number of CTAs
- * (at most 20 MB).
+ * of the stripe fix-up (the global reduction of Section 3.4 "Striped Partitioning"): a part of fixed size
+ * (10.5 MB) and one that grows with N and with max_M up to 128 rows and, above, with the number of
+ * (column tile, 128-row slab) pairs up to the number of CTAs (at most 20 MB more).
  * The caller zeroes it ONCE after allocation (cudaMemset); every call leaves the counters zero.
- * One workspace must not be used by two calls that can run at the same time. */
+ * One workspace must not be used by two calls that can run at the same time.  It may serve calls on
+ * different layers, formats and batch sizes one after the other (one stream, or ordered by events) if it
+ * has the largest of their sizes: the parts lie at the same offsets for every call. */
 MARLIN_API size_t marlin_workspace_bytes(int max_M, int K, int N);
 
 /* ---- offline quantiser (Section 3.5 (a): group scales picked by a search over group-wise clipping

@@ -107,19 +107,20 @@ size_t marlin_packed_meta_bytes(int K, int N) {
   return (size_t)K * N / 8;
 }
 
-// Workspace map: [status word, counters: 8192 bytes][partial-tile slots of the warp-MMA kernel]
-// ... [fp32 accumulation tiles of the tcgen05 kernel, placed at the END of the buffer].  Everything is
-// zero at rest; both kernels leave it that way.
-static size_t mma_slot_bytes(int max_M, int N) {
-  // two slots per worker, each the widest partial tile of the warp-level kernel: 16 rows x 256 columns
-  size_t b = (size_t)2 * kMaxWorkers * kWsSlotCols * kMaxSlabM * sizeof(float);
-  // the tcgen05 kernel with deferred scales: 128 columns x 16, 32 or 64 rows
-  if (tcd_mode() != 0 && N % 128 == 0) {
-    const size_t t = (size_t)2 * kMaxWorkers * tcd_slot_floats(max_M < kTcdMaxSlabM ? max_M : kTcdMaxSlabM) * sizeof(float);
-    if (t > b) b = t;
-  }
-  return b;
-}
+// Workspace map: [status word, counters: 8192 bytes][partial-tile slots of the warp-MMA kernel and of the tcgen05
+// kernel with deferred scales: a region of FIXED size][fp32 accumulation tiles of the tcgen05 kernel].
+// The counters and the accumulation tiles are zero at rest and every kernel leaves them that way; the slots are
+// written before they are read in every call and keep what the last call left.  Both boundaries are the same for
+// every layer, batch size and buffer size, so one buffer may serve calls on different layers one after the other:
+// the slots of one call never fall into the accumulation tiles of another.
+// two slots per worker, each the widest partial tile: 16 rows x 256 columns (warp-level kernel) or 64 rows x 128
+// columns (deferred scales)
+constexpr size_t kWsSlotFloats = (size_t)kWsSlotCols * kMaxSlabM > (size_t)128 * kTcdMaxSlabM ? (size_t)kWsSlotCols * kMaxSlabM
+                                                                                                : (size_t)128 * kTcdMaxSlabM;
+constexpr size_t kWsSlotRegionBytes = (size_t)2 * kMaxWorkers * kWsSlotFloats * sizeof(float);
+constexpr size_t kWsTcOff = kWsPartialOff + kWsSlotRegionBytes;
+// what the warp-level kernel alone needs: counters and its own slots
+constexpr size_t kWarpOnlyWsBytes = kWsPartialOff + (size_t)2 * kMaxWorkers * kWsSlotCols * kMaxSlabM * sizeof(float);
 // sparse24: 2:4 layers on the wide layout run on the tcgen05 kernel at every batch size
 static size_t tc_tile_bytes(int max_M, int N, bool sparse24) {
   if ((!sparse24 && max_M < tc_min_m()) || N % 256) return 0;
@@ -129,7 +130,7 @@ static size_t tc_tile_bytes(int max_M, int N, bool sparse24) {
 }
 static size_t workspace_bytes_for(int max_M, int K, int N, bool sparse24) {
   (void)K;
-  return kWsPartialOff + mma_slot_bytes(max_M, N) + tc_tile_bytes(max_M, N, sparse24);
+  return kWsTcOff + tc_tile_bytes(max_M, N, sparse24);
 }
 
 size_t marlin_workspace_bytes(int max_M, int K, int N) {
@@ -208,7 +209,8 @@ int marlin_unpack(const void* w_packed, const void* s_packed, uint32_t* q_kpacke
 // Shared body of marlin_gemm and marlin_gemm_sparse24 (meta_packed == nullptr: dense).
 static int gemm_common(const void* A, const void* w_packed, const void* meta_packed, const void* s_packed, void* C, int M,
                        int K, int N, int group_size, void* workspace, size_t workspace_bytes, marlin_stream stream,
-                       bool sparse24, const void* z_packed = nullptr, bool swiglu = false, bool w8 = false) {
+                       bool sparse24, const void* z_packed = nullptr, bool swiglu = false, bool w8 = false,
+                       bool warp_kernel_only = false) {
   if (!A || !w_packed || !s_packed || !C || !workspace || (sparse24 && !meta_packed)) return MARLIN_ERR_NULL;
   // layers with zero points: the warp-level kernel up to 16 rows (and in slabs where N is not a multiple of 256), the
   // tcgen05 kernel above
@@ -221,7 +223,10 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
   if (!aligned16(A) || !aligned16(w_packed) || !aligned16(s_packed) || !aligned16(C) || !aligned16(workspace) ||
       (sparse24 && !aligned16(meta_packed)))
     return MARLIN_ERR_ALIGN;
-  if (workspace_bytes < workspace_bytes_for(M, K, N, sparse24 || G < kTileK || zero_points || w8)) return MARLIN_ERR_WORKSPACE;
+  // (warp_kernel_only: the built-in array of marlin_gemm_static_ws, which holds the counters and the slots of the
+  // warp-level kernel and nothing else; its caller has checked that this kernel serves the call)
+  if (workspace_bytes < (warp_kernel_only ? kWarpOnlyWsBytes : workspace_bytes_for(M, K, N, sparse24 || G < kTileK || zero_points || w8)))
+    return MARLIN_ERR_WORKSPACE;
   DeviceInfo info;
   int st = device_info(&info);
   if (st != MARLIN_OK) return st;
@@ -242,9 +247,9 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
     // groups of 64 or 32 rows likewise (accepted only where N is a multiple of 256)
     const bool small_groups = G < kTileK || w8;
     // (the kernel with deferred scales has no fused activation: those layers go through the warp-level kernel then)
-    const bool use_tcd = !swiglu && !sparse24 && !small_groups && !zero_points && tcd_path_supported(1, K, N) &&
-                         (tmode == 1 || (tmode == 2 && rem >= tc_min_m() && !tc_ok));
-    const bool use_tc = !use_tcd && tc_ok && (sparse24 || small_groups || rem >= tc_min_m());
+    const bool use_tcd = !warp_kernel_only && !swiglu && !sparse24 && !small_groups && !zero_points &&
+                         tcd_path_supported(1, K, N) && (tmode == 1 || (tmode == 2 && rem >= tc_min_m() && !tc_ok));
+    const bool use_tc = !warp_kernel_only && !use_tcd && tc_ok && (sparse24 || small_groups || rem >= tc_min_m());
     const int m_slab = use_tcd ? (rem < kTcdMaxSlabM ? rem : kTcdMaxSlabM)
                                : use_tc ? (rem < tc_max_rows(K, N, info.sm_count) ? rem : tc_max_rows(K, N, info.sm_count))
                                         : (rem < kMaxSlabM ? rem : kMaxSlabM);
@@ -269,8 +274,7 @@ static int gemm_common(const void* A, const void* w_packed, const void* meta_pac
     p.status = reinterpret_cast<int*>(ws + kWsStatusOff);
     p.counters = reinterpret_cast<int*>(ws + kWsCounterOff);
     p.partials = reinterpret_cast<float*>(ws + kWsPartialOff);
-    p.tc_tiles = use_tc ? reinterpret_cast<float*>(ws + ((workspace_bytes & ~(size_t)255) - tc_tile_bytes(m_slab, N, sparse24 || small_groups)))
-                        : nullptr;
+    p.tc_tiles = use_tc ? reinterpret_cast<float*>(ws + kWsTcOff) : nullptr;
     p.split = 0;
     p.whole = 0;
     p.slabs = 1;
@@ -386,8 +390,8 @@ int marlin_gemm_zp(const void* A, const void* w_packed, const void* s_packed, co
 // Scratch for marlin_gemm_static_ws: the workspace of one layer call with M <= MARLIN_STATIC_WS_MAX_M,
 // as a file-scope device array.  In host code the name `g_static_workspace` is only a handle for
 // cudaGetSymbolAddress; the kernels get the device address that call returns.
-constexpr size_t kStaticWsBytes =
-    kWsPartialOff + (size_t)2 * kMaxWorkers * kWsSlotCols * MARLIN_STATIC_WS_MAX_M * sizeof(float);
+static_assert(MARLIN_STATIC_WS_MAX_M <= kMaxSlabM, "the built-in workspace serves the warp-level kernel alone");
+constexpr size_t kStaticWsBytes = kWarpOnlyWsBytes;
 static __device__ __align__(256) unsigned char g_static_workspace[kStaticWsBytes];
 
 int marlin_gemm_static_ws(const void* A, const void* w_packed, const void* s_packed, void* C, int M, int K, int N,
@@ -398,7 +402,6 @@ int marlin_gemm_static_ws(const void* A, const void* w_packed, const void* s_pac
   const int Gs = normalise_group(K, N, group_size);
   if (!Gs || Gs < kTileK) return MARLIN_ERR_GROUP;  // groups of 64 / 32 rows need the tcgen05 kernel's share of a workspace
   if (!aligned16(A) || !aligned16(w_packed) || !aligned16(s_packed) || !aligned16(C)) return MARLIN_ERR_ALIGN;
-  if (workspace_bytes_for(M, K, N, false) > kStaticWsBytes) return MARLIN_ERR_WORKSPACE;
   DeviceInfo info;
   int st = device_info(&info);
   if (st != MARLIN_OK) return st;
@@ -418,7 +421,8 @@ int marlin_gemm_static_ws(const void* A, const void* w_packed, const void* s_pac
   if (cudaMemsetAsync(ws + kWsCounterOff, 0, kWsPartialOff - kWsCounterOff, static_cast<cudaStream_t>(stream)) !=
       cudaSuccess)
     return MARLIN_ERR_CUDA;
-  return marlin_gemm(A, w_packed, s_packed, C, M, K, N, group_size, ws, kStaticWsBytes, stream);
+  return gemm_common(A, w_packed, nullptr, s_packed, C, M, K, N, group_size, ws, kStaticWsBytes, stream, false, nullptr,
+                     false, false, true);
 }
 
 int marlin_pack_sparse24(const uint32_t* qc_kpacked, const uint8_t* idx, const void* scales, void* w_packed,

@@ -8,7 +8,7 @@ import numpy as np
 import pytest
 
 from paper_2408_11743_b200 import inputs
-from gpu_util import DenseLayer, SparseLayer, to_host
+from gpu_util import DenseLayer, SparseLayer, to_dev, to_host
 
 pytestmark = pytest.mark.gpu
 
@@ -135,3 +135,41 @@ def test_nothing_is_written_outside_the_workspace(marlin, oracle_lib, monkeypatc
     assert bad == 0, worst
     assert bool((big[:guard] == 0xA5).all()) and bool((big[guard + need:] == 0xA5).all())
     assert bool((big[guard + 256:guard + need] == 0).all())
+
+
+def test_one_workspace_serves_layers_of_different_kinds_in_turn(marlin, oracle_lib, monkeypatch):
+    # One buffer, sized as the largest of the calls' own requirements (each asked for at its own batch size), serves a
+    # layer of the kernel with deferred scales (64 rows: partial-tile slots as wide as they get), a 2:4 layer and a
+    # layer with groups of 64 rows on the tcgen05 kernel (accumulation tiles that must be zero at rest) and a layer
+    # of the warp-level kernel forced onto the workspace fix-up, in turn on one stream without a synchronisation in
+    # between.  The slots keep what a call left: they must never fall into another call's accumulation tiles.
+    import torch
+    monkeypatch.setenv("MARLIN_B200_CLUSTER", "0")
+    d1 = inputs.make_dense(64, 2048, 2432, 128, seed=1)      # N not a multiple of 256: deferred scales, slots of every CTA
+    sp = inputs.make_sparse24(16, 1024, 8192, 128, seed=2)   # 16 rows: 1 MB of accumulation tiles in the L2
+    d3 = inputs.make_dense(8, 4096, 512, 128, seed=3)        # warp-level kernel, slots
+    d4 = inputs.make_dense(24, 1024, 1024, 64, seed=4)       # groups of 64: tcgen05 kernel, accumulation tiles
+    need = max(marlin.workspace_bytes(64, 2048, 2432), marlin.workspace_bytes(16, 1024, 8192),
+               marlin.workspace_bytes(8, 4096, 512), marlin.workspace_bytes(24, 1024, 1024))
+    ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
+    L1, L3, L4 = (DenseLayer(marlin, c.q_kpacked, c.S, c.G if c.G != c.K else -1, max_M=1) for c in (d1, d3, d4))
+    L2 = SparseLayer(marlin, sp, 1)
+    refs = {1: oracle_lib.gemm(d1.A, d1.q_kpacked, d1.S, d1.G), 3: oracle_lib.gemm(d3.A, d3.q_kpacked, d3.S, d3.G),
+            4: oracle_lib.gemm(d4.A, d4.q_kpacked, d4.S, d4.G),
+            2: oracle_lib.gemm_sparse24(sp.A, sp.qc_kpacked, sp.idx, sp.S, sp.G)}
+    A = {1: to_dev(d1.A), 2: to_dev(sp.A), 3: to_dev(d3.A), 4: to_dev(d4.A)}
+    outs = []
+    for which in (1, 3, 2, 4, 1, 2, 3, 4, 2, 1):
+        if which == 2:
+            C = marlin.gemm_sparse24(A[2], L2.w, L2.meta, L2.s, L2.K, L2.N, L2.G, ws)
+        else:
+            L = {1: L1, 3: L3, 4: L4}[which]
+            C = marlin.gemm(A[which], L.w, L.s, L.K, L.N, L.G, ws)
+        outs.append((which, C))
+    torch.cuda.synchronize()
+    assert marlin.read_status(ws) == 0
+    for i, (which, C) in enumerate(outs):
+        bad, worst, _ = oracle_lib.check_tolerance(to_host(C), refs[which])
+        assert bad == 0, (i, which, bad, worst)
+    host = to_host(ws)
+    assert np.all(host[256:8192] == 0)  # arrival counters
