@@ -57,6 +57,10 @@ constexpr int kBarBytes = 1024;  // full[32] at 0, empty[32] at 256, flags at 51
 // that error in two of three timing runs on the 8192 x 8192 layer; batches above 16 rows go to the
 // tcgen05 kernel, or through this one as slabs of 16 rows where that kernel does not apply.
 constexpr int consumer_warps_for(int /*mb*/) { return 8; }
+// Twelve consumer warps (three per scheduler, 152 registers each: the 8-row instances need no more; the 16-row ones
+// would spill) hide more of the latency of the conversion -> MMA chains: the loop runs about 10 % faster.  The plan
+// takes them where that shows in the launch time (make_dense_plan).
+constexpr int kWideConsumerWarps = 12;
 
 // FMT: 0 = dense, 1 = the 2:4 variant, 2 = dense with per-group zero points (W = (q - z) s: the zero-point row of a
 // group travels with the stage behind its scale row)
@@ -780,9 +784,8 @@ bool make_a_tensor_map_3d(CUtensorMap* map, const void* A, int M, int K, int box
 
 namespace {
 
-template <int MB, int NW, int FMT>
+template <int MB, int NW, int FMT, int CW = consumer_warps_for(MB)>
 cudaError_t launch_one(const DensePlan& plan, const GemmParams& p, cudaStream_t stream) {
-  constexpr int CW = consumer_warps_for(MB);
   constexpr size_t G_TILE_BYTES = (size_t)Geometry<MB, NW, CW, FMT>::TILE_F4 * 16;
   auto kernel = gemm_dense_kernel<MB, NW, CW, FMT>;
   static bool attr_set[64] = {};  // per device
@@ -833,9 +836,10 @@ cudaError_t launch_one(const DensePlan& plan, const GemmParams& p, cudaStream_t 
   return cudaLaunchKernelEx(&cfg, kernel, q, tmap);
 }
 
-template <int MB, int NW, int FMT>
+template <int MB, int NW, int FMT, int CW = consumer_warps_for(MB)>
 void fill_geometry(DensePlan* plan) {
-  using G = Geometry<MB, NW, consumer_warps_for(MB), FMT>;
+  using G = Geometry<MB, NW, CW, FMT>;
+  plan->cw = CW;
   plan->stage_bytes = G::STAGE_BYTES;
   int stages = G::STAGES;
   if (const char* e = getenv("MARLIN_B200_STAGES")) { int v = atoi(e); if (v >= 2 && v < stages) stages = v; }
@@ -846,18 +850,31 @@ void fill_geometry(DensePlan* plan) {
   // finishes segments in the middle of a stripe) could ask for the filling after next of a barrier: a parity wait
   // cannot tell that from the last completed one and falls through, after which the stage's transaction counts
   // no longer add up.
-  constexpr int kRingUnit = G::SK > kProducerWarps ? G::SK : kProducerWarps;
+  constexpr int kRingUnit = (G::SK % kProducerWarps == 0) ? G::SK
+                            : (kProducerWarps % G::SK == 0) ? kProducerWarps
+                                                            : G::SK * kProducerWarps / (G::SK % 2 == 0 ? 2 : 1);
   static_assert(kRingUnit % G::SK == 0 && kRingUnit % kProducerWarps == 0, "ring unit must be a common multiple");
   stages -= stages % kRingUnit;
   plan->stages = stages;
   plan->smem_bytes = G::FIXED_BYTES + G::ALIGN_SLACK + stages * G::STAGE_BYTES;
 }
 
+template <int MB, int NW, int CW>
+void fill_geometry_fmt(int fmt, DensePlan* plan) {
+  if (fmt == kFmtSparse) fill_geometry<MB, NW, kFmtSparse, CW>(plan);
+  else if (fmt == kFmtZero) fill_geometry<MB, NW, kFmtZero, CW>(plan);
+  else fill_geometry<MB, NW, kFmtDense, CW>(plan);
+}
+
+template <int MB, int NW, int CW>
+cudaError_t launch_one_fmt(int fmt, const DensePlan& plan, const GemmParams& p, cudaStream_t stream) {
+  if (fmt == kFmtSparse) return launch_one<MB, NW, kFmtSparse, CW>(plan, p, stream);
+  if (fmt == kFmtZero) return launch_one<MB, NW, kFmtZero, CW>(plan, p, stream);
+  return launch_one<MB, NW, kFmtDense, CW>(plan, p, stream);
+}
+
 }  // namespace
 
-
-#define MARLIN_DISPATCH(MBV, NWV, STMT)         \
-  if (plan_mb == MBV && plan_nw == NWV) { STMT; }
 
 bool make_dense_plan(int m_slab, int K, int N, int sm_count, int fmt, DensePlan* plan) {
   if (m_slab < 1 || m_slab > kMaxSlabM || K < kTileK || K % kTileK || N < kChunkN || N % kChunkN) return false;
@@ -869,19 +886,40 @@ bool make_dense_plan(int m_slab, int K, int N, int sm_count, int fmt, DensePlan*
   // is cut into S equal k-ranges, one per CTA, so that all CTAs do the same work and run the fix-up once
   // (S = 1: not at all), with the tile width (64, 128 or 256 columns) that suits the shape.  Even stripes
   // over all units (the paper's form, 128-column tiles): every SM is busy to the end, but a CTA whose
-  // stripe crosses a tile boundary pays the fix-up twice and finishes microseconds after the others.  A
-  // cost in units of one 4 KB chunk (about 0.1 us of a CTA's time), fitted to measurements on B200, picks
-  // between them: chunks per CTA, plus 0.6 per chunk-width and partial tile of the fix-up, plus 22 for the
-  // late finishers of even stripes.
+  // stripe crosses a tile boundary pays the fix-up twice and finishes microseconds after the others.
+  // A cost in microseconds picks between them, fitted to launch times measured on B200 for every candidate on 36
+  // layer shapes (K, N from 2048 to 28672), at one row and at sixteen.  Up to eight rows it picks the fastest
+  // candidate on 34 of the 36 and is within 5 % on the other two: 2.2 fixed, the chunks of the longest CTA at
+  // 0.128 (64-column tiles), 0.108 (128 columns; 0.095 with twelve consumer warps) or 0.103 (256 columns) each, the
+  // cluster fix-up at 0.4 / 0.95 / 0.8 by tile width plus 0.08 per CTA of the tile (1.0 more through the
+  // workspace, above eight CTAs), 3.8 for the late finishers of even stripes.  Sixteen rows (twice the MMAs per
+  // chunk, a ring of fewer and larger stages) have constants of their own and leave out split 256-column tiles,
+  // whose times the linear model does not follow (mean regret 0.2 %, at most 5 %).
   int forced_nw = 0;
   if (const char* e = getenv("MARLIN_B200_NW")) { int v = atoi(e); if (v == 1 || v == 2 || v == 4) forced_nw = v; }
   bool allow_split = true;
   if (const char* e = getenv("MARLIN_B200_SPLIT")) allow_split = atoi(e) != 0;
+  int want_cw = 0;  // MARLIN_B200_CW: tuning knob, 8 or 12
+  if (const char* e = getenv("MARLIN_B200_CW")) want_cw = atoi(e);
+  // twelve consumer warps: 128-column tiles from 16 stages per CTA on (see kWideConsumerWarps)
+  auto wide_pays = [&](int nw_, long long n) { return mb == 1 && nw_ == 2 && n >= 16 && fmt != kFmtSparse; };
+  auto chunk_us = [&](int nw_, long long n) {
+    if (mb != 1) return nw_ == 1 ? 0.1535 : nw_ == 4 ? 0.1425 : 0.1307;
+    const bool wide = want_cw == kWideConsumerWarps || (want_cw != consumer_warps_for(mb) && wide_pays(nw_, n));
+    return nw_ == 1 ? 0.128 : nw_ == 4 ? 0.103 : (wide ? 0.095 : 0.108);
+  };
+  const double base_us = mb == 1 ? 2.2 : 2.54, even_us = mb == 1 ? 3.8 : 4.6;
+  auto fixup_us = [&](int nw_, long long S) {
+    if (S <= 1) return 0.0;
+    if (mb == 1) return (nw_ == 1 ? 0.4 : nw_ == 2 ? 0.95 : 0.8) + 0.08 * (double)S + (S > 8 ? 1.0 : 0.0);
+    return (nw_ == 1 ? 0.0 : nw_ == 2 ? 0.28 : 1.09) + 0.26 * (double)S + (S > 8 ? 0.34 : 0.0);
+  };
   int even_nw = forced_nw ? forced_nw : 2;
   while (even_nw > 1 && N % (kChunkN * even_nw)) even_nw >>= 1;
   const long long even_units = (long long)(N / (kChunkN * even_nw)) * kb;
   const long long even_workers = even_units < max_workers ? even_units : max_workers;
-  double best = (double)((even_units + even_workers - 1) / even_workers * even_nw) + 22.0;
+  const long long even_n = (even_units + even_workers - 1) / even_workers;
+  double best = base_us + even_us + chunk_us(even_nw, even_n) * (double)(even_n * even_nw);
   int nw = even_nw, split = 0;
   for (int cand = 1; cand <= 4 && allow_split; cand *= 2) {
     if (forced_nw && cand != forced_nw) continue;
@@ -891,7 +929,8 @@ bool make_dense_plan(int m_slab, int K, int N, int sm_count, int fmt, DensePlan*
     if (S > kb) S = kb;
     if (S < 1) continue;
     const long long stages_per_cta = (kb + S - 1) / S;
-    const double cost = (double)(stages_per_cta * cand) + (S > 1 ? 0.6 * (double)(S * cand) : 0.0);
+    if (mb != 1 && cand == 4 && S > 1 && !forced_nw) continue;
+    const double cost = base_us + chunk_us(cand, stages_per_cta) * (double)(stages_per_cta * cand) + fixup_us(cand, S);
     if (cost < best) { nw = cand; split = (int)S; best = cost; }
   }
   plan->mb = mb;
@@ -903,24 +942,51 @@ bool make_dense_plan(int m_slab, int K, int N, int sm_count, int fmt, DensePlan*
   long long workers = split ? (long long)split * plan->ncols : max_workers;
   if (workers > plan->units) workers = plan->units;
   plan->workers = (int)workers;
-  const int plan_mb = mb, plan_nw = nw;
-  MARLIN_DISPATCH(1, 1, (fmt == 1 ? fill_geometry<1, 1, 1>(plan) : fmt == 2 ? fill_geometry<1, 1, 2>(plan) : fill_geometry<1, 1, 0>(plan)))
-  MARLIN_DISPATCH(1, 2, (fmt == 1 ? fill_geometry<1, 2, 1>(plan) : fmt == 2 ? fill_geometry<1, 2, 2>(plan) : fill_geometry<1, 2, 0>(plan)))
-  MARLIN_DISPATCH(1, 4, (fmt == 1 ? fill_geometry<1, 4, 1>(plan) : fmt == 2 ? fill_geometry<1, 4, 2>(plan) : fill_geometry<1, 4, 0>(plan)))
-  MARLIN_DISPATCH(2, 1, (fmt == 1 ? fill_geometry<2, 1, 1>(plan) : fmt == 2 ? fill_geometry<2, 1, 2>(plan) : fill_geometry<2, 1, 0>(plan)))
-  MARLIN_DISPATCH(2, 2, (fmt == 1 ? fill_geometry<2, 2, 1>(plan) : fmt == 2 ? fill_geometry<2, 2, 2>(plan) : fill_geometry<2, 2, 0>(plan)))
-  MARLIN_DISPATCH(2, 4, (fmt == 1 ? fill_geometry<2, 4, 1>(plan) : fmt == 2 ? fill_geometry<2, 4, 2>(plan) : fill_geometry<2, 4, 0>(plan)))
-  return plan->stages >= consumer_warps_for(mb) / nw && plan->stages >= kProducerWarps;
+  // Consumer warps: twelve for 128-column tiles (nw = 2) from 16 stages per CTA on.  Measured on B200 over 42 layer
+  // shapes (K, N from 2048 to 28672, one row): with 128-column tiles twelve warps are 5.5-7.7 % faster at every
+  // shape from 16 stages per CTA up; with 64-column tiles they are 3-5 % slower (the ring, capped at 32 stages, holds
+  // only two rounds of twelve stages, too few to cover the refill latency); with 256-column tiles it makes no
+  // difference; the 2:4 instance gains nothing.
+  int cw = consumer_warps_for(mb);
+  if (mb == 1) {
+    const long long n = split ? (kb + split - 1) / split : (plan->units + workers - 1) / workers;
+    if (want_cw == kWideConsumerWarps || (want_cw != consumer_warps_for(mb) && wide_pays(nw, n))) cw = kWideConsumerWarps;
+  }
+  for (;;) {
+    if (cw == kWideConsumerWarps) {
+      if (nw == 1) fill_geometry_fmt<1, 1, kWideConsumerWarps>(fmt, plan);
+      else if (nw == 2) fill_geometry_fmt<1, 2, kWideConsumerWarps>(fmt, plan);
+      else fill_geometry_fmt<1, 4, kWideConsumerWarps>(fmt, plan);
+    } else if (mb == 1) {
+      if (nw == 1) fill_geometry_fmt<1, 1, consumer_warps_for(1)>(fmt, plan);
+      else if (nw == 2) fill_geometry_fmt<1, 2, consumer_warps_for(1)>(fmt, plan);
+      else fill_geometry_fmt<1, 4, consumer_warps_for(1)>(fmt, plan);
+    } else {
+      if (nw == 1) fill_geometry_fmt<2, 1, consumer_warps_for(2)>(fmt, plan);
+      else if (nw == 2) fill_geometry_fmt<2, 2, consumer_warps_for(2)>(fmt, plan);
+      else fill_geometry_fmt<2, 4, consumer_warps_for(2)>(fmt, plan);
+    }
+    // the ring must hold one stage per group of warps and per producer warp
+    if (plan->stages >= plan->cw / nw && plan->stages >= kProducerWarps) return true;
+    if (cw == consumer_warps_for(mb)) return false;
+    cw = consumer_warps_for(mb);  // a ring too short for twelve warps (MARLIN_B200_STAGES): eight
+  }
 }
 
 cudaError_t launch_gemm_dense(const DensePlan& plan, const GemmParams& p, int fmt, cudaStream_t stream) {
-  const int plan_mb = plan.mb, plan_nw = plan.nw;
-  MARLIN_DISPATCH(1, 1, return (fmt == 1 ? launch_one<1, 1, 1>(plan, p, stream) : fmt == 2 ? launch_one<1, 1, 2>(plan, p, stream) : launch_one<1, 1, 0>(plan, p, stream)))
-  MARLIN_DISPATCH(1, 2, return (fmt == 1 ? launch_one<1, 2, 1>(plan, p, stream) : fmt == 2 ? launch_one<1, 2, 2>(plan, p, stream) : launch_one<1, 2, 0>(plan, p, stream)))
-  MARLIN_DISPATCH(1, 4, return (fmt == 1 ? launch_one<1, 4, 1>(plan, p, stream) : fmt == 2 ? launch_one<1, 4, 2>(plan, p, stream) : launch_one<1, 4, 0>(plan, p, stream)))
-  MARLIN_DISPATCH(2, 1, return (fmt == 1 ? launch_one<2, 1, 1>(plan, p, stream) : fmt == 2 ? launch_one<2, 1, 2>(plan, p, stream) : launch_one<2, 1, 0>(plan, p, stream)))
-  MARLIN_DISPATCH(2, 2, return (fmt == 1 ? launch_one<2, 2, 1>(plan, p, stream) : fmt == 2 ? launch_one<2, 2, 2>(plan, p, stream) : launch_one<2, 2, 0>(plan, p, stream)))
-  MARLIN_DISPATCH(2, 4, return (fmt == 1 ? launch_one<2, 4, 1>(plan, p, stream) : fmt == 2 ? launch_one<2, 4, 2>(plan, p, stream) : launch_one<2, 4, 0>(plan, p, stream)))
+  if (plan.mb == 1 && plan.cw == kWideConsumerWarps) {
+    if (plan.nw == 1) return launch_one_fmt<1, 1, kWideConsumerWarps>(fmt, plan, p, stream);
+    if (plan.nw == 2) return launch_one_fmt<1, 2, kWideConsumerWarps>(fmt, plan, p, stream);
+    if (plan.nw == 4) return launch_one_fmt<1, 4, kWideConsumerWarps>(fmt, plan, p, stream);
+  } else if (plan.mb == 1 && plan.cw == consumer_warps_for(1)) {
+    if (plan.nw == 1) return launch_one_fmt<1, 1, consumer_warps_for(1)>(fmt, plan, p, stream);
+    if (plan.nw == 2) return launch_one_fmt<1, 2, consumer_warps_for(1)>(fmt, plan, p, stream);
+    if (plan.nw == 4) return launch_one_fmt<1, 4, consumer_warps_for(1)>(fmt, plan, p, stream);
+  } else if (plan.mb == 2 && plan.cw == consumer_warps_for(2)) {
+    if (plan.nw == 1) return launch_one_fmt<2, 1, consumer_warps_for(2)>(fmt, plan, p, stream);
+    if (plan.nw == 2) return launch_one_fmt<2, 2, consumer_warps_for(2)>(fmt, plan, p, stream);
+    if (plan.nw == 4) return launch_one_fmt<2, 4, consumer_warps_for(2)>(fmt, plan, p, stream);
+  }
   return cudaErrorInvalidValue;
 }
 

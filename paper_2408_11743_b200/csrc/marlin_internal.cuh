@@ -40,6 +40,7 @@ constexpr int kWsSlotCols = 256;      // widest column tile
 struct DensePlan {
   int mb;          // 8-row blocks of A per launch (1, 2 or 4)
   int nw;          // chunks per stage; column tile = 64 * nw
+  int cw;          // consumer warps of the CTA (8 or 12)
   int kb;          // K / 128
   int ncols;       // N / (64 * nw)
   long long units; // ncols * kb

@@ -9,7 +9,8 @@ from gpu_util import to_dev, to_host
 
 pytestmark = pytest.mark.gpu
 
-SWITCHES = ["MARLIN_B200_SPLIT", "MARLIN_B200_TC_SPLIT", "MARLIN_B200_CLUSTER", "MARLIN_B200_TC_CLUSTER", "MARLIN_B200_NW"]
+SWITCHES = ["MARLIN_B200_SPLIT", "MARLIN_B200_TC_SPLIT", "MARLIN_B200_CLUSTER", "MARLIN_B200_TC_CLUSTER", "MARLIN_B200_NW",
+            "MARLIN_B200_CW"]
 BATCHES = [1, 2, 3, 5, 8, 9, 13, 16, 17, 24, 32, 33, 48, 64, 65, 100, 128, 129, 200, 256, 300, 513]
 
 
@@ -34,6 +35,8 @@ def test_random_cases_match_their_oracles(oracle_lib, monkeypatch, seed):
             monkeypatch.setenv("MARLIN_B200_NW", str(rng.choice([1, 2, 4])))
         elif mode == 4:
             monkeypatch.setenv("MARLIN_B200_TC_SPLIT", str(rng.choice([2, 4, 8])))
+        if rng.integers(0, 3) == 0:
+            monkeypatch.setenv("MARLIN_B200_CW", "12")   # twelve consumer warps wherever the batch allows them
         fmt = str(rng.choice(["dense", "dense", "sparse", "zp", "w8"]))
         K = 128 * int(rng.integers(1, 40))
         nmul = 256 if fmt == "w8" else 64

@@ -58,6 +58,10 @@ MODES = [
     {"MARLIN_B200_CLUSTER": "0", "MARLIN_B200_TC_CLUSTER": "0"},         # no clusters: fix-up through the workspace
     {"MARLIN_B200_NW": "1"}, {"MARLIN_B200_NW": "2"}, {"MARLIN_B200_NW": "4"},
     {"MARLIN_B200_NW": "4", "MARLIN_B200_SPLIT": "0"}, {"MARLIN_B200_NW": "1", "MARLIN_B200_CLUSTER": "0"},
+    # twelve consumer warps (the planner takes them on long stripes only) in every tile width, partition and fix-up
+    {"MARLIN_B200_CW": "12"}, {"MARLIN_B200_CW": "12", "MARLIN_B200_NW": "1", "MARLIN_B200_CLUSTER": "0"},
+    {"MARLIN_B200_CW": "12", "MARLIN_B200_NW": "2", "MARLIN_B200_SPLIT": "0"}, {"MARLIN_B200_CW": "12", "MARLIN_B200_NW": "4"},
+    {"MARLIN_B200_CW": "8"},
 ]
 MODE_SHAPES = [(1, 4096, 4096, 128), (8, 2048, 1536, 128), (16, 1024, 768, -1), (13, 11008, 512, 128),
                (40, 4096, 4096, 128), (128, 2048, 1024, 128), (64, 8192, 8192, 128)]

@@ -56,7 +56,9 @@ def test_sparse_gemm_matches_oracle(marlin, oracle_lib, M, K, N, G):
 
 # the partition and the fix-up the planner did not pick for a shape, forced through the library's tuning switches
 SPARSE_MODES = [{"MARLIN_B200_SPLIT": "0", "MARLIN_B200_TC_SPLIT": "0"}, {"MARLIN_B200_CLUSTER": "0", "MARLIN_B200_TC_CLUSTER": "0"},
-                {"MARLIN_B200_NW": "1"}, {"MARLIN_B200_NW": "2"}, {"MARLIN_B200_NW": "4", "MARLIN_B200_SPLIT": "0"}]
+                {"MARLIN_B200_NW": "1"}, {"MARLIN_B200_NW": "2"}, {"MARLIN_B200_NW": "4", "MARLIN_B200_SPLIT": "0"},
+                {"MARLIN_B200_CW": "12"}, {"MARLIN_B200_CW": "12", "MARLIN_B200_NW": "1", "MARLIN_B200_SPLIT": "0"},
+                {"MARLIN_B200_CW": "12", "MARLIN_B200_NW": "2", "MARLIN_B200_CLUSTER": "0"}]
 
 
 @pytest.mark.parametrize("mode", range(len(SPARSE_MODES)))

@@ -9,7 +9,9 @@ from gpu_util import to_dev, to_host
 pytestmark = pytest.mark.gpu
 
 MODES = [{}, {"MARLIN_B200_TC_SPLIT": "0", "MARLIN_B200_SPLIT": "0"}, {"MARLIN_B200_TC_CLUSTER": "0", "MARLIN_B200_CLUSTER": "0"},
-         {"MARLIN_B200_NW": "1"}, {"MARLIN_B200_NW": "4", "MARLIN_B200_SPLIT": "0"}]
+         {"MARLIN_B200_NW": "1"}, {"MARLIN_B200_NW": "4", "MARLIN_B200_SPLIT": "0"},
+         {"MARLIN_B200_CW": "12"}, {"MARLIN_B200_CW": "12", "MARLIN_B200_NW": "2", "MARLIN_B200_SPLIT": "0"},
+         {"MARLIN_B200_CW": "12", "MARLIN_B200_NW": "1", "MARLIN_B200_CLUSTER": "0"}]
 
 
 @pytest.fixture(scope="module")

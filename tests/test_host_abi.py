@@ -115,10 +115,11 @@ def test_stripe_partition_covers_every_unit_once(marlin, K, N, M, sms):
 
 
 @pytest.mark.parametrize("K,N,tile,workers,form", [
-    (8192, 8192, 64, 128, "aligned"),      # one 64-column tile and all of K per CTA: no fix-up across CTAs
+    (8192, 8192, 128, 128, "aligned"),     # 64 tiles x 2 k-ranges of 32 stages: twelve consumer warps pay from 16 on
     (4096, 4096, 64, 128, "aligned"),      # 64 tiles x 2 k-ranges
     (4096, 12288, 256, 144, "aligned"),    # 48 tiles x 3 k-ranges
-    (11008, 4096, 64, 128, "aligned"),     # 64 tiles x 2 k-ranges
+    (11008, 4096, 128, 128, "aligned"),    # 32 tiles x 4 k-ranges
+    (2048, 8192, 64, 128, "aligned"),      # short K: one 64-column tile and all of K per CTA, no fix-up across CTAs
     (4096, 22016, 128, 148, "even"),       # 172 tiles do not divide 148 SMs: even stripes
     (28672, 8192, 128, 148, "even"),       # long K: idle SMs would cost more than the late finishers
 ])
