@@ -816,27 +816,40 @@ cudaError_t launch_gemm_dense_tc(GemmParams p, int sm_count, bool sparse24, cuda
   p.units = (uint32_t)units;
   // With up to 128 rows the epilogue of a segment (accumulators out of tensor memory, L2 reductions, arrival
   // count) takes microseconds during which the CTA converts nothing, and under even stripes most CTAs run it
-  // twice.  Where the tiles divide the SMs well, each tile is cut into S k-ranges instead, one per CTA: one
-  // epilogue per CTA, all CTAs alike.  Otherwise (few CTAs per tile would idle many SMs) even stripes stay.
+  // twice.  So each tile is cut into S k-ranges instead, one per CTA (one epilogue per CTA, all CTAs alike),
+  // wherever that leaves few SMs idle, or where what the idle SMs would have taken costs less than the second
+  // epilogues of even stripes (about ten k-blocks of a CTA's time, six up to 32 rows: layers of 8-16 column tiles up
+  // to K of about 16 K; measured on B200 over 25 shapes at 64 and 128 rows, e.g. 8192 x 2048 at 128 rows: 14.7 us with eight
+  // k-ranges on 64 SMs against 20.0 us with even stripes on 148).
   p.split = 0;
   {
     long long S = workers / p.ncols;
     if (S > (long long)p.kb) S = p.kb;
     if (S > 8) S = 8;  // the CTAs of a tile form a thread-block cluster: at most the portable size
+    // at least four k-blocks per CTA (2048 x 4096 at 64 rows: 7.4 us with four k-ranges, 8.9 with eight); two up
+    // to 32 rows, where the epilogue is light (the same layer at 32 rows: 6.2 us with eight k-ranges, 6.5 with four)
+    const long long min_kb = p.M <= 32 ? 2 : 4;
+    if (S > (long long)p.kb / min_kb) S = p.kb / min_kb;
     const char* e = getenv("MARLIN_B200_TC_SPLIT");  // tuning knob: 0 forces even stripes
-    // Clusters of eight do not all fit on the device at once, so eight k-ranges per tile go through the L2, which
-    // above 64 rows costs about 5 us more than the exchange inside clusters of four: on short layers four longer
-    // k-ranges win (measured: 13.4 against 15.9 us on 4096 x 4096 at 128 rows; from about 56 k-blocks up eight win).
     bool chosen = false;
-    if (S == 8 && p.M > 64 && p.kb <= 56 && 4 * p.ncols * 100 >= workers * 40) {
-      S = 4;
+    // Above 64 rows the partial tiles are large.  Clusters of eight all fit on the device only for up to eight
+    // column tiles; beyond that eight k-ranges per tile go through the L2, which costs about 5 us more than the
+    // exchange inside clusters: shorter layers take four or six longer k-ranges instead (measured at 128 rows:
+    // 4096 x 4096 13.3 us with four against 15.7 with eight; 8192 x 4096 17.5 with six, 18.8 with eight, 19.0 with
+    // four; 14336 x 4096 23.3 with six, 23.8 with eight; 28672 x 4096 33.8 with eight, 37.1 with six).
+    if (S == 8 && p.M > 64 && p.ncols > 8 && p.kb <= 120 && 4 * p.ncols * 100 >= workers * 40) {
+      S = p.kb <= 56 ? 4 : 6;
       chosen = true;
     }
     if (e && atoi(e) >= 2 && atoi(e) <= 8 && atoi(e) <= workers / p.ncols) {  // tuning knob: 2..8 k-ranges per tile
       S = atoi(e);
       chosen = true;
     }
-    if (S >= 2 && (S * p.ncols * 100 >= workers * 85 || chosen) && !(e && atoi(e) == 0)) {
+    // k-blocks per CTA that the idle SMs of the split cost, against even stripes on all of them
+    // (up to 32 rows the second epilogue is cheaper: six k-blocks; 14336 x 2048 at 32 rows: 11.6 us even, 12.7 split)
+    const bool idle_is_cheap = S >= 2 && (double)p.kb * (1.0 / (double)S - (double)p.ncols / (double)workers) <
+                                             (p.M <= 32 ? 6.0 : 10.0);
+    if (S >= 2 && (S * p.ncols * 100 >= workers * 85 || chosen || idle_is_cheap) && !(e && atoi(e) == 0)) {
       p.split = (uint32_t)S;
       workers = S * p.ncols;
     }
