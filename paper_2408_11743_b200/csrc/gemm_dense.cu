@@ -248,8 +248,8 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
       for (int x = 0; x < 1000; ++x) __nanosleep(1000);
     }
     if (p.cluster) {
-      // every thread of every CTA of the cluster takes part in the two barriers of the fix-up
-      cluster_sync_all();
+      // every thread of every CTA of the cluster takes part in the barriers of the fix-up
+      if (p.cluster == 1) cluster_sync_all();
       cluster_sync_all();
     }
     return;
@@ -606,10 +606,13 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
       // The CTAs of this column tile form a thread-block cluster and finish side by side.  The partial tiles
       // go straight into the shared memory of the cluster's first CTA (its stage ring is free by now), which
       // adds them to its own in rank order: the order of the workspace path, without its L2 round trips.
+      // (cluster == 2: the launch has room for the partial tiles behind the stage ring, which nobody else touches:
+      // no need to wait until the first CTA is done with its ring)
       const int rank = (int)worker - first_w;
-      cluster_sync_all();  // every CTA of the tile is done with its stage ring
+      const uint32_t xbuf = p.cluster == 2 ? stage0_s + (uint32_t)nstages * G::STAGE_BYTES : stage0_s;
+      if (p.cluster == 1) cluster_sync_all();  // every CTA of the tile is done with its stage ring
       if (rank != 0 && grp == 0) {
-        const uint32_t dst = stage0_s + (uint32_t)(((rank - 1) * G::TILE_F4 + wn * G::FRAG_F4 * 32 + lane) * 16);
+        const uint32_t dst = xbuf + (uint32_t)(((rank - 1) * G::TILE_F4 + wn * G::FRAG_F4 * 32 + lane) * 16);
 #pragma unroll
         for (int r = 0; r < 4 * MB; ++r) st_cluster_f32x4(dst + (uint32_t)(r * 32 * 16), 0u, acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
       }
@@ -617,7 +620,7 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
       if (rank == 0) {
         if (grp == 0) {
           for (int src = 1; src <= last_w - first_w; ++src) {
-            const uint32_t from = stage0_s + (uint32_t)(((src - 1) * G::TILE_F4 + wn * G::FRAG_F4 * 32 + lane) * 16);
+            const uint32_t from = xbuf + (uint32_t)(((src - 1) * G::TILE_F4 + wn * G::FRAG_F4 * 32 + lane) * 16);
 #pragma unroll
             for (int r = 0; r < 4 * MB; ++r) {
               const uint4 v = lds128(from + (uint32_t)(r * 32 * 16));
@@ -832,6 +835,12 @@ cudaError_t launch_one(const DensePlan& plan, const GemmParams& p, cudaStream_t 
     const int ok = (nmax > 0 && (long long)nmax * S >= plan.workers) ? 1 : -1;  // all clusters of THIS grid at once
     cfg.numAttrs = ok > 0 ? 2 : 1;
     q.cluster = ok > 0 ? 1u : 0u;
+    // room behind the ring for the S - 1 partial tiles: the exchange then needs one cluster barrier instead of two
+    const char* x = getenv("MARLIN_B200_XBUF");  // tuning knob: 0 = partial tiles into the first CTA's ring
+    if (ok > 0 && (size_t)plan.smem_bytes + (size_t)(S - 1) * G_TILE_BYTES <= (size_t)kSmemBudget && !(x && atoi(x) == 0)) {
+      cfg.dynamicSmemBytes = plan.smem_bytes + (S - 1) * G_TILE_BYTES;
+      q.cluster = 2u;
+    }
   }
   return cudaLaunchKernelEx(&cfg, kernel, q, tmap);
 }
@@ -887,14 +896,14 @@ bool make_dense_plan(int m_slab, int K, int N, int sm_count, int fmt, DensePlan*
   // (S = 1: not at all), with the tile width (64, 128 or 256 columns) that suits the shape.  Even stripes
   // over all units (the paper's form, 128-column tiles): every SM is busy to the end, but a CTA whose
   // stripe crosses a tile boundary pays the fix-up twice and finishes microseconds after the others.
-  // A cost in microseconds picks between them, fitted to launch times measured on B200 for every candidate on 36
-  // layer shapes (K, N from 2048 to 28672), at one row and at sixteen.  Up to eight rows it picks the fastest
-  // candidate on 34 of the 36 and is within 5 % on the other two: 2.2 fixed, the chunks of the longest CTA at
-  // 0.128 (64-column tiles), 0.108 (128 columns; 0.095 with twelve consumer warps) or 0.103 (256 columns) each, the
-  // cluster fix-up at 0.4 / 0.95 / 0.8 by tile width plus 0.08 per CTA of the tile (1.0 more through the
-  // workspace, above eight CTAs), 3.8 for the late finishers of even stripes.  Sixteen rows (twice the MMAs per
-  // chunk, a ring of fewer and larger stages) have constants of their own and leave out split 256-column tiles,
-  // whose times the linear model does not follow (mean regret 0.2 %, at most 5 %).
+  // A cost in microseconds picks between them: a least-squares fit (relative error) to the launch times measured
+  // on B200 for every candidate on 36 layer shapes (K, N from 2048 to 28672), at one row and at sixteen.  Up to
+  // eight rows: 2.33 fixed, the chunks of the longest CTA at 0.121 (64-column tiles), 0.099 (128 columns; 0.096
+  // with twelve consumer warps) or 0.105 (256 columns) each, the cluster fix-up at 0 / 0.36 / 0.68 by tile width
+  // plus 0.137 per CTA of the tile (1.11 more through the workspace, above eight CTAs), 4.14 for the late finishers
+  // of even stripes: the pick is within 3 % of the fastest candidate on all 36 shapes (0.1 % on average).  Sixteen
+  // rows (twice the MMAs per chunk, a ring of fewer and larger stages) have constants of their own and leave out
+  // split 256-column tiles, whose times the linear model does not follow (0.3 % on average, at most 5 %).
   int forced_nw = 0;
   if (const char* e = getenv("MARLIN_B200_NW")) { int v = atoi(e); if (v == 1 || v == 2 || v == 4) forced_nw = v; }
   bool allow_split = true;
@@ -904,15 +913,15 @@ bool make_dense_plan(int m_slab, int K, int N, int sm_count, int fmt, DensePlan*
   // twelve consumer warps: 128-column tiles from 16 stages per CTA on (see kWideConsumerWarps)
   auto wide_pays = [&](int nw_, long long n) { return mb == 1 && nw_ == 2 && n >= 16 && fmt != kFmtSparse; };
   auto chunk_us = [&](int nw_, long long n) {
-    if (mb != 1) return nw_ == 1 ? 0.1535 : nw_ == 4 ? 0.1425 : 0.1307;
+    if (mb != 1) return nw_ == 1 ? 0.1536 : nw_ == 4 ? 0.1424 : 0.1303;
     const bool wide = want_cw == kWideConsumerWarps || (want_cw != consumer_warps_for(mb) && wide_pays(nw_, n));
-    return nw_ == 1 ? 0.128 : nw_ == 4 ? 0.103 : (wide ? 0.095 : 0.108);
+    return nw_ == 1 ? 0.1213 : nw_ == 4 ? 0.1051 : (wide ? 0.0964 : 0.0991);
   };
-  const double base_us = mb == 1 ? 2.2 : 2.54, even_us = mb == 1 ? 3.8 : 4.6;
+  const double base_us = mb == 1 ? 2.33 : 2.55, even_us = mb == 1 ? 4.14 : 4.62;
   auto fixup_us = [&](int nw_, long long S) {
     if (S <= 1) return 0.0;
-    if (mb == 1) return (nw_ == 1 ? 0.4 : nw_ == 2 ? 0.95 : 0.8) + 0.08 * (double)S + (S > 8 ? 1.0 : 0.0);
-    return (nw_ == 1 ? 0.0 : nw_ == 2 ? 0.28 : 1.09) + 0.26 * (double)S + (S > 8 ? 0.34 : 0.0);
+    if (mb == 1) return (nw_ == 1 ? 0.0 : nw_ == 2 ? 0.36 : 0.68) + 0.137 * (double)S + (S > 8 ? 1.11 : 0.0);
+    return (nw_ == 1 ? -0.34 : nw_ == 2 ? 0.0 : 0.89) + 0.268 * (double)S + (S > 8 ? 0.51 : 0.0);
   };
   int even_nw = forced_nw ? forced_nw : 2;
   while (even_nw > 1 && N % (kChunkN * even_nw)) even_nw >>= 1;

@@ -62,6 +62,8 @@ MODES = [
     {"MARLIN_B200_CW": "12"}, {"MARLIN_B200_CW": "12", "MARLIN_B200_NW": "1", "MARLIN_B200_CLUSTER": "0"},
     {"MARLIN_B200_CW": "12", "MARLIN_B200_NW": "2", "MARLIN_B200_SPLIT": "0"}, {"MARLIN_B200_CW": "12", "MARLIN_B200_NW": "4"},
     {"MARLIN_B200_CW": "8"},
+    # the cluster exchange through the first CTA's stage ring (two cluster barriers) instead of a buffer behind the ring
+    {"MARLIN_B200_XBUF": "0"}, {"MARLIN_B200_XBUF": "0", "MARLIN_B200_CW": "12", "MARLIN_B200_NW": "2"},
 ]
 MODE_SHAPES = [(1, 4096, 4096, 128), (8, 2048, 1536, 128), (16, 1024, 768, -1), (13, 11008, 512, 128),
                (40, 4096, 4096, 128), (128, 2048, 1024, 128), (64, 8192, 8192, 128)]

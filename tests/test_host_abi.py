@@ -121,7 +121,8 @@ def test_stripe_partition_covers_every_unit_once(marlin, K, N, M, sms):
     (11008, 4096, 128, 128, "aligned"),    # 32 tiles x 4 k-ranges
     (2048, 8192, 64, 128, "aligned"),      # short K: one 64-column tile and all of K per CTA, no fix-up across CTAs
     (4096, 22016, 128, 148, "even"),       # 172 tiles do not divide 148 SMs: even stripes
-    (28672, 8192, 128, 148, "even"),       # long K: idle SMs would cost more than the late finishers
+    (28672, 8192, 128, 128, "aligned"),    # 64 tiles x 2 k-ranges of 112 stages (as fast as even stripes on 148 SMs)
+    (8192, 28672, 128, 148, "even"),       # 224 tiles: idle SMs would cost more than the late finishers
 ])
 def test_partition_chosen_for_the_layer_shapes_of_the_benchmarks(marlin, K, N, tile, workers, form):
     n_tile, w, bounds = marlin.plan_stripes(1, K, N, 148)
