@@ -5,6 +5,7 @@ The product is the C-ABI library ``libmarlin_b200.so`` declared in ``include/mar
 call loads the library and raises if it is missing (there is no CPU or eager fallback).
 """
 from .binding import (  # noqa: F401
+    Layer,
     MarlinError,
     gemm,
     gemm_sparse24,

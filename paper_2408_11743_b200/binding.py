@@ -477,6 +477,106 @@ def gemm_sparse24(A, w_packed, meta_packed, s_packed, K: int, N: int, group_size
     return out
 
 
+class Layer:
+    """A packed layer bound to its workspace: its buffers are checked once, here, so that a call only checks A,
+    reads three pointers and makes the one foreign call (marlin_gemm, marlin_gemm_sparse24, marlin_gemm_zp or
+    marlin_gemm_w8 by what the layer has).  Argument marshalling only, like the functions above.
+
+        layer = Layer(w_packed, s_packed, K, N, group_size, workspace)      # dense 4-bit
+        layer = Layer(..., meta_packed=meta)                                # 2:4
+        layer = Layer(..., z_packed=z)                                      # zero points
+        layer = Layer(..., w8=True)                                         # 8-bit codes
+        C = layer(A)            # or layer(A, out=C, stream=s)
+    """
+
+    def __init__(self, w_packed, s_packed, K: int, N: int, group_size: int, workspace, meta_packed=None, z_packed=None,
+                 w8: bool = False, max_M: Optional[int] = None):
+        torch = _torch()
+        L = lib()
+        if sum(x is not None for x in (meta_packed, z_packed)) + (1 if w8 else 0) > 1:
+            raise ValueError("a layer is one of: dense, 2:4 (meta_packed), zero points (z_packed), 8-bit (w8)")
+        self.K, self.N, self.G = int(K), int(N), int(group_size)
+        w = _dev(w_packed, torch.uint8, "w_packed")
+        sc = _dev(s_packed, torch.uint8, "s_packed")
+        ws = _dev(workspace, torch.uint8, "workspace")
+        wbytes = L.marlin_packed_weight_bytes_w8(K, N) if w8 else L.marlin_packed_weight_bytes(K, N, 1 if meta_packed is not None else 0)
+        sbytes = L.marlin_packed_scale_bytes(K, N, group_size)
+        if wbytes == 0 or sbytes == 0 or w.numel() != wbytes or sc.numel() != sbytes:
+            raise ValueError("packed buffer sizes do not match K, N, group_size")
+        self._keep = [w, sc, ws]
+        extra = None
+        if meta_packed is not None:
+            extra = _dev(meta_packed, torch.uint8, "meta_packed")
+            if extra.numel() != L.marlin_packed_meta_bytes(K, N):
+                raise ValueError("meta_packed does not match K, N")
+            self._fn, self._what = L.marlin_gemm_sparse24, "marlin_gemm_sparse24"
+        elif z_packed is not None:
+            extra = _dev(z_packed, torch.uint8, "z_packed")
+            if extra.numel() != sbytes:
+                raise ValueError("z_packed does not match K, N, group_size")
+            self._fn, self._what = L.marlin_gemm_zp, "marlin_gemm_zp"
+        elif w8:
+            self._fn, self._what = L.marlin_gemm_w8, "marlin_gemm_w8"
+        else:
+            self._fn, self._what = L.marlin_gemm, "marlin_gemm"
+        if extra is not None:
+            self._keep.append(extra)
+        self._kind = 1 if meta_packed is not None else (2 if z_packed is not None else 0)
+        self._w, self._s, self._x = w.data_ptr(), sc.data_ptr(), (extra.data_ptr() if extra is not None else 0)
+        self._ws, self._ws_bytes = ws.data_ptr(), ws.numel()
+        self._device = w.device
+        self._f16 = torch.float16
+        self._empty = torch.empty
+        self._current_stream = torch.cuda.current_stream
+        if max_M is not None and self._ws_bytes < L.marlin_workspace_bytes(max_M, K, N):
+            raise ValueError("workspace smaller than marlin_workspace_bytes(max_M, K, N)")
+
+    def __call__(self, A, out=None, stream=None):
+        if A.dtype != self._f16 or not A.is_cuda or not A.is_contiguous() or A.dim() != 2 or A.shape[1] != self.K:
+            raise ValueError("A must be a contiguous fp16 CUDA tensor [M, K]")
+        M = A.shape[0]
+        if out is None:
+            out = self._empty((M, self.N), dtype=self._f16, device=self._device)
+        elif out.dtype != self._f16 or not out.is_cuda or not out.is_contiguous() or tuple(out.shape) != (M, self.N):
+            raise ValueError("out must be a contiguous fp16 CUDA tensor [M, N]")
+        sp = (stream if stream is not None else self._current_stream()).cuda_stream
+        k = self._kind
+        if k == 0:
+            st = self._fn(A.data_ptr(), self._w, self._s, out.data_ptr(), M, self.K, self.N, self.G, self._ws, self._ws_bytes, sp)
+        elif k == 1:
+            st = self._fn(A.data_ptr(), self._w, self._x, self._s, out.data_ptr(), M, self.K, self.N, self.G, self._ws,
+                          self._ws_bytes, sp)
+        else:
+            st = self._fn(A.data_ptr(), self._w, self._s, self._x, out.data_ptr(), M, self.K, self.N, self.G, self._ws,
+                          self._ws_bytes, sp)
+        if st != 0:
+            raise MarlinError(st, self._what)
+        return out
+
+    def prepare(self, A, out=None, stream=None):
+        """Checks A and out once and returns a function of no arguments that makes the foreign call on exactly these
+        buffers and this stream and returns `out`: for callers that reuse fixed device buffers step after step."""
+        if A.dtype != self._f16 or not A.is_cuda or not A.is_contiguous() or A.dim() != 2 or A.shape[1] != self.K:
+            raise ValueError("A must be a contiguous fp16 CUDA tensor [M, K]")
+        M = A.shape[0]
+        if out is None:
+            out = self._empty((M, self.N), dtype=self._f16, device=self._device)
+        elif out.dtype != self._f16 or not out.is_cuda or not out.is_contiguous() or tuple(out.shape) != (M, self.N):
+            raise ValueError("out must be a contiguous fp16 CUDA tensor [M, N]")
+        sp = (stream if stream is not None else self._current_stream()).cuda_stream
+        head = (A.data_ptr(), self._w)
+        mid = (self._s,) if self._kind == 0 else ((self._x, self._s) if self._kind == 1 else (self._s, self._x))
+        args = head + mid + (out.data_ptr(), M, self.K, self.N, self.G, self._ws, self._ws_bytes, sp)
+        fn, what, keep = self._fn, self._what, (A, out, stream, self)
+
+        def call():
+            st = fn(*args)
+            if st != 0:
+                raise MarlinError(st, what)
+            return keep[1]
+        return call
+
+
 def read_status(workspace, stream=None) -> int:
     """marlin_read_status: synchronises the stream and returns the device-side status word."""
     torch = _torch()

@@ -341,3 +341,49 @@ def test_workspace_is_clean_after_large_batch_calls(marlin, oracle_lib):
         ws = to_host(layer.ws)
         assert np.all(ws[256:8192] == 0)                    # counters
         assert np.all(ws[-N * 128 * 4:] == 0)               # accumulation tiles (placed at the end)
+
+
+def test_layer_object_makes_the_same_calls(marlin, oracle_lib):
+    # Layer checks the packed buffers once and then makes the same foreign call as the functions: same results
+    # (bit for bit where the kernel's summation order is fixed), same errors for a bad A
+    import torch
+    from oracle import w8_ref, zp_ref
+    K, N, G, M = 1024, 512, 128, 8
+    case = inputs.make_dense(M, K, N, G, seed=5)
+    A = to_dev(case.A)
+    w, s = marlin.pack(to_dev(case.q_kpacked), to_dev(case.S), G)
+    ws = marlin.new_workspace(64, K, N)
+    dense = marlin.Layer(w, s, K, N, G, ws, max_M=64)
+    assert torch.equal(dense(A), marlin.gemm(A, w, s, K, N, G, ws))
+    out = torch.empty((M, N), dtype=torch.float16, device="cuda")
+    assert dense(A, out=out) is out
+    call = dense.prepare(A, out=out)           # buffers checked once, the same foreign call on every use
+    out.zero_()
+    assert call() is out and torch.equal(out, marlin.gemm(A, w, s, K, N, G, ws))
+    Z = np.random.default_rng(1).integers(0, 16, size=case.S.shape, dtype=np.uint8)
+    z = marlin.pack_zeros(to_dev(Z), K, N, G)
+    zp = marlin.Layer(w, s, K, N, G, ws, z_packed=z)
+    assert torch.equal(zp(A), marlin.gemm_zp(A, w, s, z, K, N, G, ws))
+    sp = inputs.make_sparse24(M, K, N, G, seed=6)
+    w2, meta, s2 = marlin.pack_sparse24(to_dev(sp.qc_kpacked), to_dev(sp.idx), to_dev(sp.S), sp.G)
+    sparse = marlin.Layer(w2, s2, K, N, G, ws, meta_packed=meta)
+    bad, worst, _ = oracle_lib.check_tolerance(to_host(sparse(to_dev(sp.A))),
+                                               oracle_lib.gemm_sparse24(sp.A, sp.qc_kpacked, sp.idx, sp.S, sp.G))
+    assert bad == 0, worst
+    rng = np.random.default_rng(7)
+    Q8 = rng.integers(0, 256, size=(K, N), dtype=np.uint8)
+    S8 = rng.uniform(0.0005, 0.002, size=(K // G, N)).astype(np.float16)
+    w8, s8 = marlin.pack_w8(to_dev(Q8), to_dev(S8), G)
+    eight = marlin.Layer(w8, s8, K, N, G, ws, w8=True)
+    bad, worst, _ = oracle_lib.check_tolerance(to_host(eight(A)), w8_ref.gemm_w8(case.A, Q8, S8, G))
+    assert bad == 0, worst
+    torch.cuda.synchronize()
+    assert marlin.read_status(ws) == 0
+    with pytest.raises(ValueError):
+        dense(A[:, :512])                       # wrong K (and not contiguous)
+    with pytest.raises(ValueError):
+        dense(A.float())
+    with pytest.raises(ValueError):
+        marlin.Layer(w, s, K, N, 64, ws)        # scale buffer does not match the group size
+    with pytest.raises(ValueError):
+        marlin.Layer(w, s, K, N, G, ws, max_M=100000)
