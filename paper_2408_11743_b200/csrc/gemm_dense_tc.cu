@@ -330,8 +330,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       }
     }
     if (p.cluster) {
-      // every thread of every CTA of the cluster takes part in the three barriers of the epilogue
-      cluster_sync_all();
+      // every thread of every CTA of the cluster takes part in the two barriers of the epilogue
       cluster_sync_all();
       cluster_sync_all();
     }
@@ -518,7 +517,8 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
       constexpr int R4 = MPAD / 4;              // blocks of four batch rows
       const int S = (int)p.split;
       const int r = (int)cluster_ctarank();
-      cluster_sync_all();                       // all CTAs of the tile are done with their stage rings
+      // (the partial tile goes into this CTA's OWN ring, which is quiet once its accumulators are complete: no
+      // barrier is needed before it; the others read it only after the barrier below)
       const uint32_t mine_s = smem_u32(stage0); // [block of four rows][256 columns] float4
 #pragma unroll 1
       for (int cc = 0; cc < MPAD / 32; ++cc) {
