@@ -673,6 +673,61 @@ def run_ours(args):
         torch.cuda.synchronize(dev)
         e2e_s = e0.elapsed_time(e1) * 1e-3 / args.steps
         torch.cuda.set_stream(torch.cuda.default_stream(dev))
+
+        # The same step as a caller with fixed buffers runs it: captured once through the same binding into a CUDA
+        # graph (copy in from the pinned buffer, the eight calls, copy out to a pinned buffer), three such graphs
+        # with buffer sets, workspaces and streams of their own replayed in turn, so that the copies of one step run
+        # under the kernels of the others.  Every step still moves its inputs in and its results out; the host makes
+        # two torch calls per step instead of a dozen, so a slow host no longer bounds the number.
+        NG = 3
+        g_streams = [torch.cuda.Stream(device=dev) for _ in range(NG)]
+        g_ws = [marlin.new_workspace(max(SWEEP), K_DIM, N_DIM) for _ in range(NG)]
+        g_A = [torch.empty((rows, K_DIM), dtype=torch.float16, device=dev) for _ in range(NG)]
+        g_C = [torch.empty((rows, N_DIM), dtype=torch.float16, device=dev) for _ in range(NG)]
+        g_Ch = [torch.empty((rows, N_DIM), dtype=torch.float16).pin_memory() for _ in range(NG)]
+        graphs = []
+        for gi in range(NG):
+            layers_g = [marlin.Layer(w, s, K_DIM, N_DIM, GROUP, g_ws[gi], max_M=max(SWEEP)) for w, s in packed]
+
+            def one_step(gi=gi, layers_g=layers_g):
+                g_A[gi].copy_(A_host, non_blocking=True)
+                r0 = 0
+                for j, M in enumerate(SWEEP):
+                    layers_g[(len(SWEEP) * gi + j) % copies](g_A[gi][r0:r0 + M], out=g_C[gi][r0:r0 + M], stream=g_streams[gi])
+                    r0 += M
+                g_Ch[gi].copy_(g_C[gi], non_blocking=True)
+            with torch.cuda.stream(g_streams[gi]):
+                one_step()
+            g_streams[gi].synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=g_streams[gi]):
+                one_step()
+            graphs.append(g)
+        torch.cuda.synchronize(dev)
+
+        def graph_step(i):
+            torch.cuda.set_stream(g_streams[i % NG])
+            graphs[i % NG].replay()
+        for i in range(2 * NG):
+            graph_step(i)
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(g_streams[0])
+        for i in range(args.steps):
+            graph_step(i)
+        for st in g_streams[1:]:
+            g_streams[0].wait_stream(st)
+        e1.record(g_streams[0])
+        e1.synchronize()
+        torch.cuda.synchronize(dev)
+        torch.cuda.set_stream(torch.cuda.default_stream(dev))
+        e2e_graph_s = e0.elapsed_time(e1) * 1e-3 / args.steps
+        for gi in range(NG):
+            if marlin.read_status(g_ws[gi]) != 0:
+                raise RuntimeError("device-side wait expired during the end-to-end run")
+        # the results that came back to the host are those of the eager pipeline's buffers (same inputs, same layer)
+        if not torch.equal(torch.nan_to_num(g_Ch[0][:16].float()), torch.nan_to_num(C_host[0][:16].float())):
+            raise RuntimeError("graph-replayed step and eager step returned different results for M <= 16")
         h2d = sum(2 * M * K_DIM for M in SWEEP)
         d2h = sum(2 * M * N_DIM for M in SWEEP)
 
@@ -715,8 +770,15 @@ def run_ours(args):
             "other_layers": extra,
             "cpu_baseline": {"value": round(cpu_v, 4), "unit": UNIT, "cores": cores, "kind": "oracle",
                              "sample": f"one whole step: the full layer at M in {list(CPU_SAMPLE_MS)} ({cpu_t:.1f} s on {cores} threads)"},
-            "e2e": {"value": round(world * step_wbytes / e2e_s / 1e9, 2), "unit": UNIT,
-                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_s * 1e3, 5)},
+            "e2e": {"value": round(world * step_wbytes / min(e2e_s, e2e_graph_s) / 1e9, 2), "unit": UNIT,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": round(min(e2e_s, e2e_graph_s) * 1e3, 5),
+                    "how": "the faster of two ways to run the step from pinned host buffers through the binding",
+                    "eager_ms_per_step": round(e2e_s * 1e3, 5),
+                    "eager": "a dozen torch calls and eight layer calls per step on three streams, two buffer sets",
+                    "graph_ms_per_step": round(e2e_graph_s * 1e3, 5),
+                    "graph": "the step (copy in, eight calls, copy out) captured once per buffer set, three graphs "
+                             "replayed in turn on three streams"},
             "gpu_launches": launches_per_step * args.steps,
             "clocks": clocks,
         }
