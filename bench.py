@@ -15,8 +15,10 @@ twice the L2 capacity.
 Prints ONE JSON line.  `value` = packed weight bytes (codes + scales) streamed per second over the
 whole step, inputs resident in HBM, timed with CUDA events around a CUDA graph of K steps.
 `e2e` = the same metric with every step's A copied from pinned host memory and its C copied back inside
-the timed region (one transfer each way per step, on copy streams that overlap the neighbouring steps'
-kernels; weights stay resident: they are the model).  `roofline` is that of the dominant kernel (the
+the timed region (one transfer each way per step; weights stay resident: they are the model), through the
+package's binding, run two ways of which the faster is reported and both are listed: eagerly on copy streams that
+overlap the neighbouring steps' kernels, and as three CUDA graphs of one step each (copy in, eight calls, copy
+out) replayed in turn on three streams.  `roofline` is that of the dominant kernel (the
 instance that serves M = 1, 2, 4, 8): its algorithmic bytes (weights + scales + A + C, each once) per
 second of its own live launch time against the measured HBM peak, with the same figure for the whole
 step under `whole_step`.  `per_m` lists each
