@@ -7,8 +7,8 @@ imports this file.
 Dense layout: the packed buffer is a sequence of 4096-byte chunks, one per (k-block kb = k/128,
 64-column block nb = n/64), ordered by super-columns of four chunks:
     chunk index = (nb/4) * 4 * (K/128) + kb * cs + nb % 4,   cs = min(4, N/64 - 4*(nb/4))
-Inside a chunk, 16-byte vector v = (2*j + b)*32 + lane (lane = 4*g + c) holds 32 codes of column
-    n = 64*nb + 16*j + 8*b + g;
+Inside a chunk, 16-byte vector v = (2*j + b)*32 + 4*g + slot holds 32 codes of column
+    n = 64*nb + 16*j + 8*b + g,   slot = (c + g/2) % 4 for c = 0..3;
 its word w = 2*h + u holds rows k = 128*kb + 64*h + 16*c + 8*u + o (o = 0..7), row offset o sitting in
 nibble (o >> 1) + 4*(o & 1) (bits 4p..4p+3 for nibble p).
 Scales: inside every run of 64 columns, packed position 8*g + 2*j + b holds column 16*j + 8*b + g; groups of 64 or
@@ -23,13 +23,14 @@ def pack_dense_weights(Q: np.ndarray) -> np.ndarray:
     """Codes Q[K, N] (uint8, 0..15) -> packed uint32 words (1-D, K*N/8)."""
     K, N = Q.shape
     assert K % 128 == 0 and N % 64 == 0
-    kb, nb, j, b, g, c, h, u, p = np.meshgrid(
+    kb, nb, j, b, g, slot, h, u, p = np.meshgrid(
         np.arange(K // 128), np.arange(N // 64), np.arange(4), np.arange(2), np.arange(8), np.arange(4),
         np.arange(2), np.arange(2), np.arange(8), indexing="ij")
+    c = (slot - g // 2) % 4     # the rows 16c.. of a column sit in slot (c + g/2) % 4
     o = 2 * (p & 3) + (p >> 2)  # row offset stored in nibble p
     n = 64 * nb + 16 * j + 8 * b + g
     k = 128 * kb + 64 * h + 16 * c + 8 * u + o
-    codes = Q[k, n].astype(np.uint32)  # [kb, nb, j, b, g, c, h, u, p]: already in word order inside a chunk
+    codes = Q[k, n].astype(np.uint32)  # [kb, nb, j, b, g, slot, h, u, p]: already in word order inside a chunk
     words = np.zeros(codes.shape[:-1], dtype=np.uint32)
     for pp in range(8):
         words |= codes[..., pp] << np.uint32(4 * pp)

@@ -449,7 +449,8 @@ gemm_dense_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a
           }
         }
       } else {
-      const uint32_t wp = st_s + G::A_BYTES + wn * G::CODE_CHUNK + lane * 16;
+      // lane (g, c) finds its vector in slot (c + g / 2) % 4 of its column's four
+      const uint32_t wp = st_s + G::A_BYTES + wn * G::CODE_CHUNK + (uint32_t)((lane & ~3) | ((lane + (lane >> 3)) & 3)) * 16;
       // codes of this lane: columns g (X) and g + 8 (Y) of each 16-column block j, its 32 rows of the k-block
       uint32_t X[4][4], Y[4][4];
 #pragma unroll

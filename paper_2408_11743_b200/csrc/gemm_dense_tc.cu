@@ -405,7 +405,7 @@ gemm_dense_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tma
         for (int c = 0; c < 8; ++c) v[c] = lds128(wbase + c * 256 * 16);  // codes of rows 16c .. 16c + 15 of this column
       } else if constexpr (!SP) {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) v[c] = lds128(wbase + c * 16);
+        for (int c = 0; c < 4; ++c) v[c] = lds128(wbase + (uint32_t)(((c + (g >> 1)) & 3) * 16));  // rows 16c.. sit in slot (c + g/2) % 4
       } else {
         v[0] = lds128(wbase);                        // kept values 0..31 of this column
         v[1] = lds128(wbase + 256 * 16);             // kept values 32..63

@@ -299,7 +299,7 @@ gemm_tcd_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tmap_a) 
       const uint32_t wbase = stage0_s + s * G::STAGE_BYTES + G::A_BYTES + vec_off;
       uint4 v[4];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) v[c] = lds128(wbase + c * 16);
+      for (int c = 0; c < 4; ++c) v[c] = lds128(wbase + (uint32_t)(((c + ((n128 & 7u) >> 1)) & 3u) * 16u));  // slot (c + g/2) % 4
       if (it >= (uint32_t)NSL) {
         // the slot was last read by the MMAs of k-block it - NSL
         const uint32_t jt = it - NSL;

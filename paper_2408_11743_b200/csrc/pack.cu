@@ -12,13 +12,15 @@
 //     chunk index = sc * 4 * (K/128) + kb * cs + (nb % 4)
 //   so the weights a CTA streams for a 256-column tile are one contiguous run of memory, k-block after
 //   k-block, and one k-block of a tile is a single 16 KB bulk copy.
-//   Inside a chunk, 16-byte vector number v = (2*j + b) * 32 + lane holds 32 codes of ONE column:
-//     column n = 64*nb + 16*j + 8*b + g        (lane = 4*g + c, g = lane / 4, c = lane % 4)
+//   Inside a chunk, 16-byte vector number v = (2*j + b) * 32 + 4*g + slot holds 32 codes of ONE column:
+//     column n = 64*nb + 16*j + 8*b + g        (g = 0..7; slot = (c + g/2) % 4, c = 0..3)
 //     rows   k = 128*kb + {16*c .. 16*c + 15} and 128*kb + 64 + {16*c .. 16*c + 15}
+//   (the four vectors of a column are rotated by g/2 so that the threads of the tcgen05 kernel, one column each
+//   and 64 bytes apart, hit different banks when they all read their vector of the same c)
 //   word w of the vector (w = 2*h + u) holds rows 128*kb + 64*h + 16*c + 8*u + o, o = 0..7, with
 //   row offset o in nibble (o >> 1) + 4*(o & 1): one AND+OR pulls out the two codes of rows (2i, 2i+1).
 //   Two readers use this order:
-//     - the warp-level MMA kernel: lane (g, c) reads the vectors of columns g and g + 8 of a 16-column
+//     - the warp-level MMA kernel: lane (g, c) reads the vectors (slot as above) of columns g and g + 8 of a 16-column
 //       block; one word of each gives the A-operand registers of two m16n8k16 steps (weights on the
 //       16-wide side), and the lane's activations for its rows are 16 contiguous fp16 per 64-row half;
 //     - the tcgen05 kernel: a thread owns one column and reads its four vectors (c = 0..3), i.e. all
@@ -35,7 +37,7 @@ namespace {
 // word `wi` (0..1023) of chunk (kb, nb), nibble p -> matrix position
 __device__ __forceinline__ void decode_position(int wi, int p, int kb, int nb, int* k, int* n) {
   int w = wi & 3, lane = (wi >> 2) & 31, i = wi >> 7;
-  int g = lane >> 2, c = lane & 3, j = i >> 1, b = i & 1;
+  int g = lane >> 2, c = ((lane & 3) - (g >> 1)) & 3, j = i >> 1, b = i & 1;  // slot = (c + g/2) % 4
   int o = 2 * (p & 3) + (p >> 2);
   *n = 64 * nb + 16 * j + 8 * b + g;
   *k = 128 * kb + 64 * (w >> 1) + 16 * c + 8 * (w & 1) + o;
@@ -95,7 +97,7 @@ __global__ void unpack_weights_kernel(const uint32_t* __restrict__ wq, uint32_t*
       int k = 8 * k8 + jn;
       int kb = k >> 7, h = (k >> 6) & 1, c = (k >> 4) & 3, u = (k >> 3) & 1, o = k & 7;
       int p = (o >> 1) + 4 * (o & 1);
-      int lane = 4 * g + c, i = 2 * j + b, w = 2 * h + u;
+      int lane = 4 * g + ((c + (g >> 1)) & 3), i = 2 * j + b, w = 2 * h + u;
       long long wi = ((chunk_index(kb, nb, K / 128, nb64) * 8 + i) * 32 + lane) * 4 + w;
       uint32_t code = (wq[wi] >> (4 * p)) & 15u;
       out |= code << (4 * jn);
