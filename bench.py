@@ -683,7 +683,7 @@ def run_ours(args):
         # two torch calls per step instead of a dozen, so a slow host no longer bounds the number.
         NG = 3
         g_streams = [torch.cuda.Stream(device=dev) for _ in range(NG)]
-        g_ws = [marlin.new_workspace(max(SWEEP), K_DIM, N_DIM) for _ in range(NG)]
+        g_ws = [marlin.new_workspace(max(SWEEP), K_DIM, N_DIM, device=dev) for _ in range(NG)]
         g_A = [torch.empty((rows, K_DIM), dtype=torch.float16, device=dev) for _ in range(NG)]
         g_C = [torch.empty((rows, N_DIM), dtype=torch.float16, device=dev) for _ in range(NG)]
         g_Ch = [torch.empty((rows, N_DIM), dtype=torch.float16).pin_memory() for _ in range(NG)]
