@@ -840,6 +840,11 @@ cudaError_t launch_gemm_dense_tc(GemmParams p, int sm_count, bool sparse24, cuda
     if (S == 8 && p.M > 64 && p.ncols > 8 && p.kb <= 120 && 4 * p.ncols * 100 >= workers * 40) {
       S = p.kb <= 56 ? 4 : 6;
       chosen = true;
+    } else if (S == 8 && p.M > 32 && p.ncols > 8 && p.kb <= 32 && 4 * p.ncols * 100 >= workers * 40) {
+      // 33-64 rows: the same on the shortest layers (2:4, 4096 x 4096 at 64 rows: 7.6 us with four k-ranges in
+      // clusters, 8.9 with eight through the L2; the dense layer runs 10.1 and 10.0)
+      S = 4;
+      chosen = true;
     }
     if (e && atoi(e) >= 2 && atoi(e) <= 8 && atoi(e) <= workers / p.ncols) {  // tuning knob: 2..8 k-ranges per tile
       S = atoi(e);
